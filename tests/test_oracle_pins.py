@@ -1,0 +1,433 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU).
+
+Each test is chosen so that a plausible mistake in the oracle (dropped term, wrong sign or
+index, transposed operand, wrong mask bit) fails it.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import glance_oracle as O
+from paper_2609_00355_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ------------------------------------------------------------------ Eq. 1 / Eq. 2: printed values
+
+def _golden_rows():
+    rows = []
+    with open(os.path.join(GOLDEN, "eq2_printed_values.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            kind, arg, L, val, dec = line.split()
+            rows.append((kind, float(arg), int(L), float(val), int(dec)))
+    return rows
+
+
+def test_eq2_printed_values():
+    """Eq. 2 / Lemma 1: the closed form reproduces every number the paper prints for it."""
+    sig = lambda z: 1.0 / (1.0 + math.exp(-z))
+    seen = set()
+    for kind, arg, L, val, dec in _golden_rows():
+        half = 0.5 * 10.0 ** (-dec) + 1e-12
+        seen.add(kind)
+        if kind == "trunc_err":
+            p = arg
+            trunc = O.expected_accept(p, L)
+            untr = p / (1.0 - p)
+            assert abs((untr - trunc) / untr - val) <= half
+            assert abs(p ** L - val) <= half
+        elif kind == "sup_mean":
+            assert abs(O.expected_accept(sig(arg), L) - val) <= half
+        elif kind == "geo_cap":
+            p = sig(arg)
+            assert abs(p / (1 - p) - val) <= half and abs(math.exp(arg) - val) <= half
+        elif kind == "rel_gap_bound":
+            for p in np.linspace(0.05, arg, 16):
+                untr = p / (1 - p)
+                assert (untr - O.expected_accept(float(p), L)) / untr < val
+    assert seen == {"trunc_err", "sup_mean", "geo_cap", "rel_gap_bound"}
+
+
+def test_eq2_closed_form_and_eq1():
+    for p in (0.3, 0.5, 0.8, 0.9):
+        for L in (1, 3, 7, 15):
+            assert abs(O.expected_accept(p, L) - p * (1 - p ** L) / (1 - p)) < 1e-12
+    assert O.mean_accept_tokens([0, 0, 0]) == 1.0          # autoregressive decoding has tau = 1
+    assert O.mean_accept_tokens([2, 4]) == 4.0
+
+
+# ------------------------------------------------------------------ model pieces
+
+def test_rmsnorm_closed_form():
+    x = torch.tensor([[3.0, -4.0, 0.0, 0.0]])
+    g = torch.tensor([1.0, 2.0, 1.0, 1.0])
+    y = O.rmsnorm(x, g, 0.0)
+    rms = math.sqrt(25.0 / 4.0)
+    assert torch.allclose(y, torch.tensor([[3.0 / rms, -8.0 / rms, 0.0, 0.0]]), atol=1e-6)
+    c = torch.full((2, 8), 5.0)
+    assert torch.allclose(O.rmsnorm(c, torch.ones(8), 0.0), torch.ones(2, 8), atol=1e-6)
+
+
+def test_rope_pairs_and_relative_position():
+    # d = 2: one pair (0, 1), frequency theta^0 = 1: (1, 0) at position p -> (cos p, sin p)
+    x = torch.tensor([[[1.0, 0.0]]])
+    y = O.rope(x, torch.tensor([2]), 1e6)
+    assert torch.allclose(y, torch.tensor([[[math.cos(2.0), math.sin(2.0)]]]), atol=1e-6)
+    # d = 4: pairs are (0, 2) and (1, 3); second pair rotates by p * theta^(-1/2)
+    x = torch.tensor([[[0.0, 1.0, 0.0, 0.0]]])
+    y = O.rope(x, torch.tensor([3]), 100.0)
+    assert torch.allclose(y, torch.tensor([[[0.0, math.cos(0.3), 0.0, math.sin(0.3)]]]), atol=1e-6)
+    # position 0 is the identity; rotation preserves norms; scores depend on position differences only
+    g = torch.Generator().manual_seed(0)
+    q = torch.randn(1, 3, 16, generator=g)
+    k = torch.randn(1, 3, 16, generator=g)
+    assert torch.allclose(O.rope(q, torch.tensor([0]), 1e4), q)
+    assert torch.allclose(O.rope(q, torch.tensor([77]), 1e4).norm(dim=-1), q.norm(dim=-1), atol=1e-5)
+    s1 = (O.rope(q, torch.tensor([40]), 1e4) * O.rope(k, torch.tensor([33]), 1e4)).sum(-1)
+    s2 = (O.rope(q, torch.tensor([12]), 1e4) * O.rope(k, torch.tensor([5]), 1e4)).sum(-1)
+    s3 = (O.rope(q, torch.tensor([12]), 1e4) * O.rope(k, torch.tensor([6]), 1e4)).sum(-1)
+    assert torch.allclose(s1, s2, atol=1e-4)
+    assert not torch.allclose(s1, s3, atol=1e-3)
+
+
+def test_attention_matches_library_sdpa():
+    g = torch.Generator().manual_seed(1)
+    n, m, Hq, Hkv, d = 9, 23, 6, 2, 16
+    q = torch.randn(n, Hq, d, generator=g)
+    K = torch.randn(m, Hkv, d, generator=g)
+    V = torch.randn(m, Hkv, d, generator=g)
+    mask = torch.rand(n, m, generator=g) < 0.6
+    mask[:, 0] = True
+    got = O.attention(q, K, V, mask)
+    Kr = K.repeat_interleave(Hq // Hkv, dim=1)
+    Vr = V.repeat_interleave(Hq // Hkv, dim=1)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        q.transpose(0, 1)[None], Kr.transpose(0, 1)[None], Vr.transpose(0, 1)[None], attn_mask=mask[None, None])
+    assert torch.allclose(got, ref[0].transpose(0, 1), atol=1e-5)
+
+
+def test_topk_logprobs_matches_library_and_breaks_ties_low():
+    g = torch.Generator().manual_seed(2)
+    logits = torch.randn(5, 300, generator=g) * 3
+    logits[2, 17] = logits[2, 250] = logits[2].max() + 1.0       # exact tie for rank 0 of offset 2
+    ids, lp = O.topk_logprobs(logits, 4)
+    assert ids.shape == (4, 4)
+    for j in range(1, 5):
+        tv, ti = torch.topk(logits[j], 4)
+        lse = torch.logsumexp(logits[j].double(), dim=-1)
+        assert np.allclose(lp[j - 1], (tv.double() - lse).numpy(), atol=1e-5)
+        if j != 2:
+            assert list(ids[j - 1]) == ti.tolist()
+        assert np.all(np.diff(lp[j - 1]) <= 0) and np.all(lp[j - 1] <= 0)
+    assert list(ids[1][:2]) == [17, 250]
+    # probabilities of the full vocabulary sum to one
+    ids_all, lp_all = O.topk_logprobs(logits[:2], 300)
+    assert abs(np.exp(lp_all[0].astype(np.float64)).sum() - 1.0) < 1e-4
+
+
+def test_argmax_lowest_id_on_ties():
+    x = torch.tensor([[1.0, 5.0, 5.0, 2.0], [7.0, 1.0, 7.0, 7.0]])
+    assert list(O.argmax_lowest(x)) == [1, 0]
+
+
+# ------------------------------------------------------------------ candidate tree
+
+def _assert_tree_equal(a: O.Tree, b: O.Tree):
+    assert a.n_nodes == b.n_nodes
+    for f in ("token", "parent", "depth", "rank"):
+        assert np.array_equal(getattr(a, f), getattr(b, f)), f
+    assert np.array_equal(a.score.view(np.uint32), b.score.view(np.uint32))
+    assert np.array_equal(a.anc, b.anc)
+
+
+@pytest.mark.parametrize("L,k,N", [(3, 2, 8), (3, 2, 16), (4, 3, 32), (7, 4, 32), (5, 8, 64), (2, 2, 64)])
+@pytest.mark.parametrize("ties", [False, True])
+def test_best_first_equals_bruteforce_sort(L, k, N, ties):
+    """Algorithm 1 line 2: best-first search returns exactly the sorted top N-1 prefixes."""
+    rng = np.random.default_rng(100 * L + k + (7 if ties else 0))
+    if k ** L > 40000:
+        pytest.skip("enumeration too large")
+    for _ in range(3):
+        ids, lp = synth.random_topk(L, k, 5000, rng, ties=ties)
+        _assert_tree_equal(O.build_tree(11, ids, lp, N), O.build_tree_bruteforce(11, ids, lp, N))
+
+
+def test_best_first_on_controlled_marginals_with_exact_score_ties():
+    # identical marginals at every depth: commuted sums tie exactly, the path key decides
+    lp = synth.controlled_marginals(0.8, 4, 6)
+    ids = np.arange(24, dtype=np.int32).reshape(6, 4)
+    bf, bb = O.build_tree(3, ids, lp, 64), O.build_tree_bruteforce(3, ids, lp, 64)
+    _assert_tree_equal(bf, bb)
+    sc = bf.score[1:bf.n_nodes]
+    assert len(np.unique(sc)) < len(sc)
+
+
+def test_tree_invariants():
+    """Section 3.3: the kept set is prefix-closed; no prefix scores below its extensions."""
+    rng = np.random.default_rng(5)
+    ids, lp = synth.random_topk(15, 8, 152064, rng)
+    t = O.build_tree(9, ids, lp, 64)
+    assert t.n_nodes == 64 and t.parent[0] == -1 and t.depth[0] == 0
+    for i in range(1, t.n_nodes):
+        p = t.parent[i]
+        assert 0 <= p < i and t.depth[i] == t.depth[p] + 1
+        assert t.score[i] <= t.score[p]
+        assert t.token[i] == ids[t.depth[i] - 1][t.rank[i]]
+        assert np.float32(t.score[p] + lp[t.depth[i] - 1][t.rank[i]]) == t.score[i]
+    assert np.all(np.diff(t.score[1:t.n_nodes]) <= 0)
+    # fewer candidates than rows: n_nodes reported, padding rows see only themselves
+    ids2, lp2 = synth.random_topk(2, 2, 100, rng)
+    t2 = O.build_tree(1, ids2, lp2, 16)
+    assert t2.n_nodes == 1 + 2 + 4
+    for i in range(t2.n_nodes, 16):
+        assert t2.parent[i] == -1 and int(t2.anc[i, 0]) == 1 << i
+
+
+EX_PARENT = [-1, 0, 0, 1, 1, 2, 3, 4]
+EX_DEPTH = [0, 1, 1, 2, 2, 2, 3, 3]
+EX_TOKEN = [7, 11, 12, 21, 22, 23, 31, 32]
+
+
+def test_ancestor_mask_hand_example():
+    # hand-derived: node 6 -> ancestors 3, 1, 0 -> bits {0,1,3,6} = 0x4B, node 7 -> {0,1,4,7} = 0x93
+    t = O.tree_from_arrays(EX_TOKEN, EX_PARENT, EX_DEPTH)
+    assert [int(x) for x in t.anc[:, 0]] == [0x01, 0x03, 0x05, 0x0B, 0x13, 0x25, 0x4B, 0x93]
+    big = O.chain_tree(1, list(range(2, 72)), 128)             # second mask word
+    assert int(big.anc[70, 1]) == (1 << 7) - 1 and int(big.anc[70, 0]) == (1 << 64) - 1
+    assert int(big.anc[100, 0]) == 0 and int(big.anc[100, 1]) == 1 << 36
+
+
+def test_walk_hand_examples():
+    """Algorithm 1 lines 5-12 on a hand-made tree."""
+    t = O.tree_from_arrays(EX_TOKEN, EX_PARENT, EX_DEPTH)
+    am = np.array([11, 22, 0, 0, 99, 0, 0, 0])
+    assert O.walk(t, am) == (2, [0, 1, 4], [11, 22], 99)
+    am = np.array([12, 0, 23, 0, 0, 5, 0, 0])                  # node 5 is a leaf: stop there
+    assert O.walk(t, am) == (2, [0, 2, 5], [12, 23], 5)
+    am = np.array([13, 0, 0, 0, 0, 0, 0, 0])
+    assert O.walk(t, am) == (0, [0], [], 13)
+    am = np.array([11, 21, 0, 31, 0, 0, 44, 0])                # full depth
+    assert O.walk(t, am) == (3, [0, 1, 3, 6], [11, 21, 31], 44)
+    # a padding row can never be entered even if its token matches
+    tp = O.tree_from_arrays(EX_TOKEN[:3], EX_PARENT[:3], EX_DEPTH[:3], N=8)
+    assert O.walk(tp, np.array([0, 0, 0, 0, 0, 0, 0, 0])) == (0, [0], [], 0)
+
+
+def test_masks_chain_is_causal_and_star_sees_root_and_self():
+    P = 5
+    ch = O.chain_tree(1, [2, 3, 4, 5], 5)
+    m = O.visibility(ch, P)
+    assert torch.equal(m[:, :P], torch.ones(5, P, dtype=torch.bool))
+    assert torch.equal(m[:, P:], torch.tril(torch.ones(5, 5, dtype=torch.bool)))
+    star = O.tree_from_arrays([1, 2, 3, 4], [-1, 0, 0, 0], [0, 1, 1, 1])
+    ms = O.visibility(star, 0)
+    expect = torch.eye(4, dtype=torch.bool)
+    expect[:, 0] = True
+    assert torch.equal(ms, expect)
+
+
+# ------------------------------------------------------------------ the round on the tiny config
+
+class Tiny:
+    pass
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    torch.manual_seed(0)
+    cfg = synth.CONFIGS["tiny"]
+    tw_b, hw_b = synth.make_weights(cfg)
+    img, ids = synth.make_context(cfg)
+    t = Tiny()
+    t.cfg, t.sh = cfg, O.Shape.of(cfg)
+    t.tw, t.hw = O.widen(tw_b), O.widen(hw_b)
+    t.ctx = O.context_embeddings(t.tw, img, ids.numpy())
+    t.n_new = 40
+    t.Y, t.margins = O.greedy_ar_cachefree(t.sh, t.tw, t.ctx, t.n_new)
+    t.cap = cfg.ctx + t.n_new + cfg.tree_N + 64
+    return t
+
+
+def _fresh(t):
+    return O.prefill(t.sh, t.tw, t.hw, t.ctx, t.cap)
+
+
+def test_prefill_root_is_first_greedy_token(tiny):
+    st = _fresh(tiny)
+    assert st.P == tiny.cfg.ctx and st.root == tiny.Y[0]
+    print("smallest top-2 margin met by plain greedy decoding:", min(tiny.margins))
+
+
+def test_verify_rows_equal_plain_chain(tiny):
+    """Definition 1: the row of node y_1:d is p(. | x o b o y_1:d), for every node of small trees."""
+    rng = np.random.default_rng(3)
+    st = _fresh(tiny)
+    for n_nodes in (8, 5):
+        tok, par, dep = synth.random_tree(n_nodes, tiny.cfg.L, tiny.cfg.vocab, rng)
+        tok[0] = st.root
+        tree = O.tree_from_arrays(tok, par, dep, N=8)
+        logits, hidden = O.verify_tree(tiny.sh, tiny.tw, st, tree)
+        scale = float(logits.abs().max())
+        for s, i in O.tree_paths(tree).items():
+            ref_l, ref_h = O.chain_row(tiny.sh, tiny.tw, tiny.ctx, st.root, s)
+            assert float((logits[i] - ref_l).abs().max()) <= 1e-4 * scale
+            assert float((hidden[i] - ref_h).abs().max()) <= 1e-4 * float(hidden.abs().max())
+        ref_l, _ = O.chain_row(tiny.sh, tiny.tw, tiny.ctx, st.root, ())
+        assert float((logits[0] - ref_l).abs().max()) <= 1e-4 * scale
+
+
+def test_mask_errors_are_visible_in_attention():
+    """A wrong mask bit must change the output by O(1): one-hot values, strongly separated keys."""
+    n = 6
+    K = torch.eye(n)[:, None, :] * 30.0
+    V = torch.eye(n)[:, None, :]
+    q = torch.ones(n, 1, n)
+    tree = O.tree_from_arrays([0] * n, [-1, 0, 0, 1, 1, 2], [0, 1, 1, 2, 2, 2])
+    out = O.attention(q, K, V, O.visibility(tree, 0))[:, 0, :]
+    for i in range(n):
+        vis = [(int(tree.anc[i, 0]) >> j) & 1 for j in range(n)]
+        expect = torch.tensor(vis, dtype=torch.float32) / sum(vis)
+        assert torch.allclose(out[i], expect, atol=1e-6)
+
+
+def test_chain_tree_verify_equals_causal_chunk(tiny):
+    st = _fresh(tiny)
+    chain = O.chain_tree(st.root, tiny.Y[1:8], 8)
+    logits, hidden = O.verify_tree(tiny.sh, tiny.tw, st, chain)
+    x = torch.cat([tiny.ctx, tiny.tw["embed"][torch.tensor(tiny.Y[:8])]], dim=0)
+    ref_l, ref_h = O.full_causal_forward(tiny.sh, tiny.tw, x)
+    assert float((logits - ref_l[-8:]).abs().max()) <= 1e-4 * float(ref_l.abs().max())
+    assert float((hidden - ref_h[-8:]).abs().max()) <= 1e-4 * float(ref_h.abs().max())
+    # and the whole chain is accepted: a = 7 = min(L-limit of the chain, matches)
+    a, path, out, new_root = O.walk(chain, O.argmax_lowest(logits))
+    assert (a, path, out, new_root) == (7, list(range(8)), tiny.Y[1:8], tiny.Y[8])
+
+
+def _run_rounds(t, tree_fn, n_rounds):
+    st = _fresh(t)
+    accepts = []
+    for _ in range(n_rounds):
+        done = len(st.tokens)
+        Yrest = t.Y[done + 1:]
+        tree = tree_fn(st, Yrest)
+        if len(Yrest) < t.cfg.L + 2:
+            break
+        info = O.spec_round(t.sh, t.tw, t.hw, st, t.cfg.block_B, t.cfg.topk, t.cfg.tree_N, tree=tree)
+        assert info["a"] == O.accepted_length_bruteforce(info["tree"], Yrest)     # Definition 1
+        accepts.append(info["a"])
+    emitted = st.tokens + [st.root]
+    assert emitted == t.Y[:len(emitted)]                                         # Theorem 1
+    return st, accepts
+
+
+def test_lossless_with_drafted_best_first_trees(tiny):
+    st, acc = _run_rounds(tiny, lambda st, Y: None, 8)
+    assert len(acc) == 8
+
+
+def test_lossless_with_random_trees_planted_continuation(tiny):
+    rng = np.random.default_rng(11)
+
+    def tree_fn(st, Y):
+        def pref(parent, depth):
+            # plant the true continuation along first children with probability 0.7
+            return int(Y[depth - 1]) if rng.random() < 0.7 and depth - 1 < len(Y) else None
+        tok, par, dep = synth.random_tree(8, tiny.cfg.L, tiny.cfg.vocab, rng, tokens_for=pref)
+        tok[0] = st.root
+        return O.tree_from_arrays(tok, par, dep, N=8)
+
+    st, acc = _run_rounds(tiny, tree_fn, 10)
+    assert max(acc) >= 1 and min(acc) == 0 or len(set(acc)) > 1
+
+
+def test_lossless_with_garbage_trees_and_chain_and_single_node(tiny):
+    rng = np.random.default_rng(12)
+
+    def garbage(st, Y):
+        tok, par, dep = synth.random_tree(8, tiny.cfg.L, tiny.cfg.vocab, rng)
+        tok[0] = st.root
+        return O.tree_from_arrays(tok, par, dep, N=8)
+
+    _run_rounds(tiny, garbage, 5)
+    st, acc = _run_rounds(tiny, lambda st, Y: O.chain_tree(st.root, Y[:3], 8), 6)
+    assert acc == [3] * len(acc)                      # a true chain of depth L is accepted whole
+    st, acc = _run_rounds(tiny, lambda st, Y: O.chain_tree(st.root, [], 1), 6)
+    assert acc == [0] * len(acc) and O.mean_accept_tokens(acc) == 1.0    # N = 1 is plain AR, tau = 1
+
+
+def test_kv_state_after_rounds_equals_fresh_prefill(tiny):
+    rng = np.random.default_rng(13)
+
+    def tree_fn(st, Y):
+        def pref(parent, depth):
+            return int(Y[depth - 1]) if rng.random() < 0.8 else None
+        tok, par, dep = synth.random_tree(8, tiny.cfg.L, tiny.cfg.vocab, rng, tokens_for=pref)
+        tok[0] = st.root
+        return O.tree_from_arrays(tok, par, dep, N=8)
+
+    st, acc = _run_rounds(tiny, tree_fn, 6)
+    assert sum(acc) > 0
+    x = torch.cat([tiny.ctx, tiny.tw["embed"][torch.tensor(st.tokens)]], dim=0)
+    ref = O.prefill(tiny.sh, tiny.tw, tiny.hw, x, tiny.cap)
+    assert ref.P == st.P and ref.root == st.root
+    for l in range(tiny.sh.n_layers):
+        assert float((ref.K[l][:st.P] - st.K[l][:st.P]).abs().max()) < 1e-4
+        assert float((ref.V[l][:st.P] - st.V[l][:st.P]).abs().max()) < 1e-4
+    assert float((ref.hK[:st.P] - st.hK[:st.P]).abs().max()) < 1e-4
+    assert float((ref.hV[:st.P] - st.hV[:st.P]).abs().max()) < 1e-4
+    assert float((ref.feat[:st.P] - st.feat[:st.P]).abs().max()) < 1e-4 * float(ref.feat.abs().max())
+
+
+def test_commit_moves_rows_in_ascending_order_hazard_case(tiny):
+    """Path (0,2,5): cache row P+2 is read by step 1 and overwritten by step 2."""
+    st = _fresh(tiny)
+    P = st.P
+    for l in range(tiny.sh.n_layers):
+        for i in range(8):
+            st.K[l][P + i] = float(100 * l + i)
+            st.V[l][P + i] = float(-100 * l - i)
+    hidden = torch.arange(8, dtype=torch.float32)[:, None].repeat(1, tiny.sh.hidden)
+    O.commit(tiny.sh, tiny.hw, st, [0, 2, 5], hidden, [12, 23], 5)
+    assert st.P == P + 3 and st.root == 5
+    for l in range(tiny.sh.n_layers):
+        assert [float(st.K[l][P + i, 0, 0]) for i in range(3)] == [100 * l + 0, 100 * l + 2, 100 * l + 5]
+        assert [float(st.V[l][P + i, 1, 3]) for i in range(3)] == [-100 * l - 0, -100 * l - 2, -100 * l - 5]
+    assert [float(st.feat[P + i, 0]) for i in range(3)] == [0.0, 2.0, 5.0]
+
+
+def test_draft_block_internal_consistency(tiny):
+    """The head definition is unpinned by the paper; these are consistency checks only."""
+    st = _fresh(tiny)
+    dl = O.draft_block(tiny.sh, tiny.tw, tiny.hw, st, tiny.cfg.block_B)
+    assert dl.shape == (tiny.cfg.block_B, tiny.cfg.vocab)
+    # bidirectional block: changing the root token changes every slot's output
+    st2 = _fresh(tiny)
+    st2.root = (st.root + 1) % tiny.cfg.vocab
+    dl2 = O.draft_block(tiny.sh, tiny.tw, tiny.hw, st2, tiny.cfg.block_B)
+    assert all(float((dl[j] - dl2[j]).abs().max()) > 0 for j in range(tiny.cfg.block_B))
+    # masked slots differ only through their rotary positions
+    assert float((dl[1] - dl[2]).abs().max()) > 0
+
+
+def test_controlled_match_acceptance_statistics(tiny):
+    """Measured mean accepted length under controlled per-depth match probability sits on Eq. 2."""
+    rng = np.random.default_rng(21)
+    cfg = tiny.cfg
+    L, k, p = 15, 8, 0.8
+    lp = synth.controlled_marginals(p, k, L)
+    Y = list(np.random.default_rng(5).integers(0, 50000, size=L + 1))
+    acc = []
+    for _ in range(600):
+        ids = synth.controlled_candidates(Y[:L], p, k, L, 50000, rng)
+        tree = O.build_tree(1, ids, lp, 64)
+        acc.append(O.accepted_length_bruteforce(tree, Y))
+    mean, sd = np.mean(acc), np.std(acc) / math.sqrt(len(acc))
+    # the rank-0 chain reaches depth 15 inside a 64-node tree at p = 0.8
+    assert abs(mean - O.expected_accept(p, L)) < 4 * sd + 0.05
