@@ -1,0 +1,509 @@
+// C ABI of the GLANCE round library: context, workspace carving, and the stream-ordered sequence of
+// kernels behind each entry point declared in glance.h.
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "kernels.cuh"
+
+using namespace glance;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// split-K factor of a weight-streaming GEMM: enough CTAs to cover the SMs, at least 8 k-tiles per split
+int choose_split(int Nout, int K) {
+    const int tiles = (Nout + 127) / 128;
+    const int ktiles = K / 64;
+    int s = (148 + tiles - 1) / tiles;
+    s = std::min(s, std::max(1, ktiles / 8));
+    return std::max(1, std::min(s, 16));
+}
+
+struct Workspace {
+    float *x;            // [Rmax][H] residual stream
+    bf16 *xn;            // [Rmax][H]
+    float *part;         // split-K planes
+    bf16 *q;             // [Rmax][Hq d]
+    bf16 *attn;          // [Rmax][Hq d]
+    bf16 *act;           // [Rmax][F]
+    float *logits;       // [Rlog][V]
+    float *att_o;        // attention split partials
+    float *att_ml;
+    int32_t *att_ctr;
+    int32_t *walk_ctr;
+    int32_t *row_seq, *row_pos, *row_kvslot;
+    float *rope_cos, *rope_sin;
+    uint64_t *chain_anc;   // [N][W] prefill chain mask
+    bf16 *hidden_tmp;      // [N][H] prefill hidden
+    int32_t *argmax_tmp;   // [N]
+    int32_t *status;
+    size_t part_elems;
+    size_t total;
+};
+
+struct Dims {
+    int Rmax, Rlog, qkv_out, qd, S_qkv, S_o, S_d, S_att, q_tiles_max, W;
+};
+
+Dims make_dims(const glance_config &c) {
+    Dims d;
+    d.Rmax = c.max_batch * std::max(c.tree_N, 2 * c.block_B);
+    d.Rmax = std::max(d.Rmax, c.tree_N);
+    d.Rlog = c.max_batch * std::max(c.tree_N, c.block_B);
+    d.qkv_out = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
+    d.qd = c.n_q_heads * c.head_dim;
+    d.S_qkv = choose_split(d.qkv_out, c.hidden);
+    d.S_o = choose_split(c.hidden, d.qd);
+    d.S_d = choose_split(c.hidden, c.ffn);
+    const int G = c.n_q_heads / c.n_kv_heads;
+    d.q_tiles_max = attention_q_tiles(std::max(c.tree_N, c.block_B), G);
+    int ctas = attention_q_tiles(c.tree_N, G) * c.n_kv_heads * c.max_batch;
+    d.S_att = std::max(1, std::min(16, (2 * 148 + ctas - 1) / ctas));
+    d.W = (c.tree_N + 63) / 64;
+    return d;
+}
+
+// carve (or just size, when base == nullptr) the workspace
+Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
+    Workspace w;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        unsigned char *p = base ? base + off : nullptr;
+        off = align_up(off + bytes, 256);
+        return p;
+    };
+    const size_t R = d.Rmax, H = c.hidden;
+    w.x = (float *)take(R * H * 4);
+    w.xn = (bf16 *)take(R * H * 2);
+    size_t pe = std::max({(size_t)d.S_qkv * R * d.qkv_out, (size_t)d.S_o * R * H, (size_t)R * 2 * c.ffn,
+                          (size_t)d.S_d * R * H});
+    w.part_elems = pe;
+    w.part = (float *)take(pe * 4);
+    w.q = (bf16 *)take(R * d.qd * 2);
+    w.attn = (bf16 *)take(R * d.qd * 2);
+    w.act = (bf16 *)take(R * (size_t)c.ffn * 2);
+    w.logits = (float *)take((size_t)d.Rlog * c.vocab * 4);
+    const size_t att_rows = (size_t)c.max_batch * c.n_kv_heads * d.q_tiles_max * 64;
+    w.att_o = (float *)take(att_rows * d.S_att * c.head_dim * 4);
+    w.att_ml = (float *)take(att_rows * d.S_att * 2 * 4);
+    w.att_ctr = (int32_t *)take((size_t)c.max_batch * c.n_kv_heads * d.q_tiles_max * 4);
+    w.walk_ctr = (int32_t *)take((size_t)c.max_batch * 4);
+    w.row_seq = (int32_t *)take(R * 4);
+    w.row_pos = (int32_t *)take(R * 4);
+    w.row_kvslot = (int32_t *)take(R * 4);
+    w.rope_cos = (float *)take(R * (c.head_dim / 2) * 4);
+    w.rope_sin = (float *)take(R * (c.head_dim / 2) * 4);
+    w.chain_anc = (uint64_t *)take((size_t)c.tree_N * d.W * 8);
+    w.hidden_tmp = (bf16 *)take((size_t)c.tree_N * H * 2);
+    w.argmax_tmp = (int32_t *)take((size_t)c.tree_N * 4);
+    w.status = (int32_t *)take(256);
+    w.total = off;
+    return w;
+}
+
+bool config_ok(const glance_config *c) {
+    if (!c) return false;
+    if (c->n_layers < 1 || c->hidden < 64 || c->hidden % 64 || c->ffn < 64 || c->ffn % 64) return false;
+    if (c->head_dim != 64 && c->head_dim != 128) return false;
+    if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return false;
+    if (c->vocab < 2) return false;
+    if (c->block_B < 2 || c->block_B > kMaxBlock || c->topk < 1 || c->topk > kMaxTopk) return false;
+    if (c->tree_N < 1 || c->tree_N > kMaxTreeN) return false;
+    if (c->page_size != kPage || c->max_batch < 1 || c->max_batch > 64 || c->max_pages_per_seq < 1) return false;
+    if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
+    return true;
+}
+
+}  // namespace
+
+struct glance_ctx {
+    glance_config cfg;
+    Dims dims;
+    Workspace ws;
+    cudaStream_t stream;
+    const bf16 *embed, *lm_head, *final_norm;
+    std::vector<const bf16 *> ln1, wqkv, wo, ln2, wgu, wd;
+    glance_head_weights head;
+    int64_t launches;
+};
+
+namespace {
+
+#define LAUNCH(ctx, call) \
+    do {                  \
+        call;             \
+        (ctx)->launches++; \
+    } while (0)
+
+struct LayerW {
+    const bf16 *ln2, *wqkv, *wo, *wgu, *wd;
+};
+
+struct PassInfo {
+    int R;                 // rows entering the layer
+    int Rq;                // rows that continue after the K/V write (queries)
+    int batch, T;          // attention: T query rows / extra keys per sequence
+    const uint64_t *anc;   // or nullptr
+    const glance_seqs *seqs;
+    int seq_off;           // first sequence (prefill of one sequence of a batch)
+};
+
+KvGeom geom_of(const glance_ctx *ctx, const glance_seqs *s) {
+    KvGeom g;
+    g.n_pages = s->n_pages;
+    g.n_kv_heads = ctx->cfg.n_kv_heads;
+    g.head_dim = ctx->cfg.head_dim;
+    g.max_pages_per_seq = ctx->cfg.max_pages_per_seq;
+    return g;
+}
+
+RowMeta meta_of(const glance_ctx *ctx) {
+    RowMeta m;
+    m.seq = ctx->ws.row_seq;
+    m.pos = ctx->ws.row_pos;
+    m.kvslot = ctx->ws.row_kvslot;
+    m.rope_cos = ctx->ws.rope_cos;
+    m.rope_sin = ctx->ws.rope_sin;
+    return m;
+}
+
+// One decoder layer over the rows of a pass.  On entry ws.xn holds the normalised input rows; on exit
+// ws.x holds the new residual stream and ws.xn the rows normalised with `next_gain`.
+void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInfo &ps, const bf16 *next_gain,
+               bf16 *hidden_out) {
+    const glance_config &c = ctx->cfg;
+    const Dims &d = ctx->dims;
+    Workspace &ws = ctx->ws;
+    cudaStream_t st = ctx->stream;
+    const KvGeom geom = geom_of(ctx, ps.seqs);
+    const int32_t *page_table = ps.seqs->page_table + (size_t)ps.seq_off * c.max_pages_per_seq;
+    const int32_t *seq_len = ps.seqs->seq_len + ps.seq_off;
+    // QKV projection, split-K planes
+    size_t ss = (size_t)ps.R * d.qkv_out;
+    LAUNCH(ctx, launch_gemm(w.wqkv, ws.xn, ws.part, d.qkv_out, c.hidden, ps.R, d.qkv_out, ss, d.S_qkv, st));
+    RopeKv rk;
+    rk.R = ps.R; rk.Rq = ps.Rq; rk.Hq = c.n_q_heads; rk.Hkv = c.n_kv_heads; rk.d = c.head_dim;
+    rk.part = ws.part; rk.S = d.S_qkv; rk.split_stride = ss; rk.ldy = d.qkv_out;
+    rk.meta = meta_of(ctx); rk.q = ws.q; rk.pool_layer = pool_layer; rk.geom = geom; rk.page_table = page_table;
+    rk.status = ws.status;
+    LAUNCH(ctx, launch_rope_kv(rk, st));
+    if (ps.Rq == 0) return;
+    AttnParams ap;
+    ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
+    ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
+    ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn; ap.S = d.S_att; ap.part_o = ws.att_o;
+    ap.part_ml = ws.att_ml; ap.counters = ws.att_ctr; ap.status = ws.status;
+    LAUNCH(ctx, launch_attention(ap, st));
+    const int R = ps.Rq;
+    // output projection + residual + norm
+    ss = (size_t)R * c.hidden;
+    LAUNCH(ctx, launch_gemm(w.wo, ws.attn, ws.part, c.hidden, d.qd, R, c.hidden, ss, d.S_o, st));
+    LAUNCH(ctx, launch_norm(ws.x, ws.part, d.S_o, ss, c.hidden, R, c.hidden, w.ln2, nullptr, R, c.rms_eps, ws.xn,
+                            nullptr, st));
+    // SwiGLU MLP
+    LAUNCH(ctx, launch_gemm(w.wgu, ws.xn, ws.part, 2 * c.ffn, c.hidden, R, 2 * c.ffn, 0, 1, st));
+    LAUNCH(ctx, launch_swiglu(ws.part, 2 * c.ffn, R, c.ffn, ws.act, st));
+    LAUNCH(ctx, launch_gemm(w.wd, ws.act, ws.part, c.hidden, c.ffn, R, c.hidden, ss, d.S_d, st));
+    LAUNCH(ctx, launch_norm(ws.x, ws.part, d.S_d, ss, c.hidden, R, c.hidden, next_gain, nullptr, R, c.rms_eps,
+                            ws.xn, hidden_out, st));
+}
+
+// all target layers + final norm (+ LM head and argmax) over rows already set up in ws.x
+void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *logits, int32_t *argmax) {
+    const glance_config &c = ctx->cfg;
+    Workspace &ws = ctx->ws;
+    cudaStream_t st = ctx->stream;
+    const KvGeom geom = geom_of(ctx, ps.seqs);
+    LAUNCH(ctx, launch_norm(ws.x, nullptr, 0, 0, c.hidden, ps.R, c.hidden, ctx->ln1[0], nullptr, ps.R, c.rms_eps,
+                            ws.xn, nullptr, st));
+    for (int l = 0; l < c.n_layers; ++l) {
+        LayerW w{ctx->ln2[l], ctx->wqkv[l], ctx->wo[l], ctx->wgu[l], ctx->wd[l]};
+        const bool last = (l + 1 == c.n_layers);
+        bf16 *pool_layer = (bf16 *)ps.seqs->kv_pool + (size_t)l * geom.layer_stride();
+        run_layer(ctx, w, pool_layer, ps, last ? ctx->final_norm : ctx->ln1[l + 1], last ? hidden_out : nullptr);
+    }
+    if (argmax) {
+        LAUNCH(ctx, launch_gemm(ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, ps.R, c.vocab, 0, 1, st));
+        LAUNCH(ctx, launch_argmax(logits, ps.R, c.vocab, argmax, st));
+    }
+}
+
+int32_t check_seqs(const glance_ctx *ctx, const glance_seqs *s) {
+    if (!ctx || !s) return GLANCE_E_INVALID_ARG;
+    if (s->batch < 1 || s->batch > ctx->cfg.max_batch || s->n_pages < 1) return GLANCE_E_INVALID_ARG;
+    if (!s->seq_len || !s->root || !s->page_table || !s->kv_pool || !s->head_kv_pool || !s->feat || !s->feat_count)
+        return GLANCE_E_INVALID_ARG;
+    return GLANCE_OK;
+}
+
+int32_t finish(glance_ctx *ctx) { return cudaPeekAtLastError() == cudaSuccess ? GLANCE_OK : GLANCE_E_CUDA; }
+
+__global__ void set_seq_kernel(int32_t *seq_len, int32_t *root, int32_t len, int32_t r) {
+    *seq_len = len;
+    *root = r;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *glance_status_string(int32_t status) {
+    switch (status) {
+        case GLANCE_OK: return "ok";
+        case GLANCE_E_INVALID_ARG: return "invalid argument";
+        case GLANCE_E_SHAPE: return "unsupported shape";
+        case GLANCE_E_CAPACITY: return "capacity exceeded";
+        case GLANCE_E_CUDA: return "CUDA error";
+        case GLANCE_E_TIMEOUT: return "device wait timed out";
+        case GLANCE_E_BOUNDS: return "device index out of bounds";
+        case GLANCE_E_STATE: return "invalid call order";
+        default: return "unknown status";
+    }
+}
+
+size_t glance_workspace_bytes(const glance_config *cfg) {
+    if (!config_ok(cfg)) return 0;
+    return carve(*cfg, make_dims(*cfg), nullptr).total;
+}
+
+int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, const glance_head_weights *h,
+                      void *workspace, size_t workspace_bytes, void *cuda_stream, glance_ctx **out) {
+    if (!cfg || !t || !h || !workspace || !out) return GLANCE_E_INVALID_ARG;
+    if (!config_ok(cfg)) return GLANCE_E_SHAPE;
+    if (((uintptr_t)workspace & 255) != 0) return GLANCE_E_INVALID_ARG;
+    if (!t->embed || !t->lm_head || !t->final_norm || !t->ln1 || !t->wqkv || !t->wo || !t->ln2 || !t->wgu || !t->wd)
+        return GLANCE_E_INVALID_ARG;
+    if (!h->mask_embed || !h->ctx_norm || !h->ln1 || !h->wqkv || !h->wo || !h->ln2 || !h->wgu || !h->wd ||
+        !h->final_norm)
+        return GLANCE_E_INVALID_ARG;
+    const Dims d = make_dims(*cfg);
+    Workspace ws = carve(*cfg, d, (unsigned char *)workspace);
+    if (ws.total > workspace_bytes) return GLANCE_E_CAPACITY;
+    glance_ctx *ctx = new (std::nothrow) glance_ctx();
+    if (!ctx) return GLANCE_E_INVALID_ARG;
+    ctx->cfg = *cfg;
+    ctx->dims = d;
+    ctx->ws = ws;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->embed = (const bf16 *)t->embed;
+    ctx->lm_head = (const bf16 *)t->lm_head;
+    ctx->final_norm = (const bf16 *)t->final_norm;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        if (!t->ln1[l] || !t->wqkv[l] || !t->wo[l] || !t->ln2[l] || !t->wgu[l] || !t->wd[l]) {
+            delete ctx;
+            return GLANCE_E_INVALID_ARG;
+        }
+        ctx->ln1.push_back((const bf16 *)t->ln1[l]);
+        ctx->wqkv.push_back((const bf16 *)t->wqkv[l]);
+        ctx->wo.push_back((const bf16 *)t->wo[l]);
+        ctx->ln2.push_back((const bf16 *)t->ln2[l]);
+        ctx->wgu.push_back((const bf16 *)t->wgu[l]);
+        ctx->wd.push_back((const bf16 *)t->wd[l]);
+    }
+    ctx->head = *h;
+    ctx->launches = 0;
+    // counters and the status word start at zero
+    if (cudaMemsetAsync(ws.att_ctr, 0, (size_t)cfg->max_batch * cfg->n_kv_heads * d.q_tiles_max * 4, ctx->stream) !=
+            cudaSuccess ||
+        cudaMemsetAsync(ws.walk_ctr, 0, (size_t)cfg->max_batch * 4, ctx->stream) != cudaSuccess ||
+        cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess) {
+        delete ctx;
+        return GLANCE_E_CUDA;
+    }
+    *out = ctx;
+    return GLANCE_OK;
+}
+
+int32_t glance_destroy(glance_ctx *ctx) {
+    if (!ctx) return GLANCE_E_INVALID_ARG;
+    delete ctx;
+    return GLANCE_OK;
+}
+
+int32_t glance_prefill(glance_ctx *ctx, const glance_seqs *seqs, int32_t seq, const void *embeds, const int32_t *ids,
+                       int32_t count) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    if (seq < 0 || seq >= seqs->batch || count < 1) return GLANCE_E_INVALID_ARG;
+    if ((embeds == nullptr) == (ids == nullptr)) return GLANCE_E_INVALID_ARG;
+    const glance_config &c = ctx->cfg;
+    Workspace &ws = ctx->ws;
+    cudaStream_t st = ctx->stream;
+    const int N = c.tree_N;
+    for (int done = 0; done < count; done += N) {
+        const int n = std::min(N, count - done);
+        const bool last = (done + n == count);
+        VerifySetup vs;
+        vs.batch = 1; vs.N = N; vs.H = c.hidden; vs.d = c.head_dim; vs.theta = c.rope_theta;
+        vs.seq_len = seqs->seq_len + seq; vs.token = nullptr; vs.depth = nullptr;
+        vs.row_embeds = embeds ? (const bf16 *)embeds + (size_t)done * c.hidden : nullptr;
+        vs.row_ids = ids ? ids + done : nullptr;
+        vs.count = n; vs.chain_anc = ws.chain_anc; vs.embed = ctx->embed; vs.vocab = c.vocab;
+        vs.capacity = c.max_pages_per_seq * kPage; vs.x = ws.x; vs.meta = meta_of(ctx); vs.status = ws.status;
+        LAUNCH(ctx, launch_setup_verify(vs, st));
+        PassInfo ps{N, N, 1, N, ws.chain_anc, seqs, seq};
+        run_target(ctx, ps, ws.hidden_tmp, ws.logits, last ? ws.argmax_tmp : nullptr);
+        // head context K/V of the new positions (Section 3.2: keys and values are the target's hidden states)
+        DraftSetup ds;
+        ds.batch = 1; ds.B = c.block_B; ds.FR = N; ds.H = c.hidden; ds.d = c.head_dim; ds.theta = c.rope_theta;
+        ds.seq_len = seqs->seq_len + seq; ds.root = seqs->root + seq; ds.feat = ws.hidden_tmp; ds.feat_count = nullptr;
+        ds.count_const = n; ds.n_block = 0; ds.embed = ctx->embed; ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
+        ds.vocab = c.vocab; ds.capacity = c.max_pages_per_seq * kPage; ds.x = ws.x; ds.meta = meta_of(ctx);
+        ds.status = ws.status;
+        LAUNCH(ctx, launch_setup_draft(ds, st));
+        LAUNCH(ctx, launch_norm(ws.x, nullptr, 0, 0, c.hidden, N, c.hidden, (const bf16 *)ctx->head.ctx_norm, nullptr, N,
+                                c.rms_eps, ws.xn, nullptr, st));
+        LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
+                  (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
+        PassInfo hp{N, 0, 1, N, nullptr, seqs, seq};
+        run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, hp, nullptr, nullptr);
+        LAUNCH(ctx, launch_prefill_advance(seqs->seq_len + seq, seqs->root + seq, seqs->feat_count + seq,
+                                           last ? ws.argmax_tmp : nullptr, n, st));
+    }
+    return finish(ctx);
+}
+
+int32_t glance_seq_truncate(glance_ctx *ctx, const glance_seqs *seqs, int32_t seq, int32_t new_len, int32_t new_root) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    if (seq < 0 || seq >= seqs->batch || new_len < 0 || new_root < 0 || new_root >= ctx->cfg.vocab)
+        return GLANCE_E_INVALID_ARG;
+    LAUNCH(ctx, (set_seq_kernel<<<1, 1, 0, ctx->stream>>>(seqs->seq_len + seq, seqs->root + seq, new_len, new_root)));
+    return finish(ctx);
+}
+
+int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *topk_ids, float *topk_lp,
+                           float *logits_dbg) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    if (!topk_ids || !topk_lp) return GLANCE_E_INVALID_ARG;
+    const glance_config &c = ctx->cfg;
+    Workspace &ws = ctx->ws;
+    cudaStream_t st = ctx->stream;
+    const int batch = seqs->batch, B = c.block_B;
+    const int R1 = batch * B, R = 2 * R1;
+    DraftSetup ds;
+    ds.batch = batch; ds.B = B; ds.FR = B; ds.H = c.hidden; ds.d = c.head_dim; ds.theta = c.rope_theta;
+    ds.seq_len = seqs->seq_len; ds.root = seqs->root; ds.feat = (const bf16 *)seqs->feat;
+    ds.feat_count = seqs->feat_count; ds.count_const = 0; ds.n_block = B; ds.embed = ctx->embed;
+    ds.mask_embed = (const bf16 *)ctx->head.mask_embed; ds.vocab = c.vocab;
+    ds.capacity = c.max_pages_per_seq * kPage; ds.x = ws.x; ds.meta = meta_of(ctx); ds.status = ws.status;
+    LAUNCH(ctx, launch_setup_draft(ds, st));
+    // block rows use the head's input norm, feature rows the context norm
+    LAUNCH(ctx, launch_norm(ws.x, nullptr, 0, 0, c.hidden, R, c.hidden, (const bf16 *)ctx->head.ln1,
+                            (const bf16 *)ctx->head.ctx_norm, R1, c.rms_eps, ws.xn, nullptr, st));
+    LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
+              (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
+    PassInfo ps{R, R1, batch, B, nullptr, seqs, 0};
+    run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, ps, (const bf16 *)ctx->head.final_norm, nullptr);
+    float *logits = logits_dbg ? logits_dbg : ws.logits;
+    LAUNCH(ctx, launch_gemm(ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, R1, c.vocab, 0, 1, st));
+    LAUNCH(ctx, launch_topk(logits, batch, B, c.vocab, c.topk, topk_ids, topk_lp, st));
+    return finish(ctx);
+}
+
+int32_t glance_build_tree(glance_ctx *ctx, int32_t batch, const int32_t *root, const int32_t *topk_ids,
+                          const float *topk_lp, const glance_tree *out) {
+    if (!ctx || !root || !topk_ids || !topk_lp || !out) return GLANCE_E_INVALID_ARG;
+    if (batch < 1 || batch > ctx->cfg.max_batch) return GLANCE_E_INVALID_ARG;
+    if (!out->token || !out->parent || !out->depth || !out->rank || !out->score || !out->anc || !out->n_nodes)
+        return GLANCE_E_INVALID_ARG;
+    const glance_config &c = ctx->cfg;
+    LAUNCH(ctx, launch_build_tree(batch, c.tree_N, c.block_B - 1, c.topk, root, topk_ids, topk_lp, *out, ctx->stream));
+    return finish(ctx);
+}
+
+int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, int32_t *argmax,
+                           void *hidden, float *logits_dbg) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    if (!tree || !tree->token || !tree->depth || !tree->anc || !argmax || !hidden) return GLANCE_E_INVALID_ARG;
+    const glance_config &c = ctx->cfg;
+    Workspace &ws = ctx->ws;
+    const int batch = seqs->batch, N = c.tree_N;
+    VerifySetup vs;
+    vs.batch = batch; vs.N = N; vs.H = c.hidden; vs.d = c.head_dim; vs.theta = c.rope_theta;
+    vs.seq_len = seqs->seq_len; vs.token = tree->token; vs.depth = tree->depth; vs.row_embeds = nullptr;
+    vs.row_ids = nullptr; vs.count = 0; vs.chain_anc = nullptr; vs.embed = ctx->embed; vs.vocab = c.vocab;
+    vs.capacity = c.max_pages_per_seq * kPage; vs.x = ws.x; vs.meta = meta_of(ctx); vs.status = ws.status;
+    LAUNCH(ctx, launch_setup_verify(vs, ctx->stream));
+    PassInfo ps{batch * N, batch * N, batch, N, tree->anc, seqs, 0};
+    run_target(ctx, ps, (bf16 *)hidden, logits_dbg ? logits_dbg : ws.logits, argmax);
+    return finish(ctx);
+}
+
+static int32_t commit_common(glance_ctx *ctx, const glance_seqs *seqs, WalkCommit &wc, const void *hidden) {
+    const glance_config &c = ctx->cfg;
+    wc.batch = seqs->batch; wc.N = c.tree_N; wc.B = c.block_B; wc.H = c.hidden; wc.n_layers = c.n_layers;
+    wc.hidden = (const bf16 *)hidden; wc.kv_pool = (bf16 *)seqs->kv_pool; wc.geom = geom_of(ctx, seqs);
+    wc.page_table = seqs->page_table; wc.seq_len = seqs->seq_len; wc.root = seqs->root;
+    wc.feat_count = seqs->feat_count; wc.feat = (bf16 *)seqs->feat; wc.counters = ctx->ws.walk_ctr;
+    wc.status = ctx->ws.status;
+    LAUNCH(ctx, launch_walk_commit(wc, ctx->stream));
+    return finish(ctx);
+}
+
+int32_t glance_accept_commit(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, const int32_t *argmax,
+                             const void *hidden, int32_t *accept_len, int32_t *path, int32_t *out_tokens) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    if (!tree || !tree->token || !tree->parent || !tree->n_nodes || !argmax || !hidden || !accept_len || !path ||
+        !out_tokens)
+        return GLANCE_E_INVALID_ARG;
+    WalkCommit wc{};
+    wc.token = tree->token; wc.parent = tree->parent; wc.n_nodes = tree->n_nodes; wc.argmax = argmax;
+    wc.accept_len = accept_len; wc.path = path; wc.out_tokens = out_tokens;
+    return commit_common(ctx, seqs, wc, hidden);
+}
+
+int32_t glance_commit_forced(glance_ctx *ctx, const glance_seqs *seqs, const void *hidden, const int32_t *path,
+                             const int32_t *path_len, const int32_t *new_root) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    if (!hidden || !path || !path_len || !new_root) return GLANCE_E_INVALID_ARG;
+    WalkCommit wc{};
+    wc.forced_path = path; wc.forced_len = path_len; wc.forced_root = new_root;
+    return commit_common(ctx, seqs, wc, hidden);
+}
+
+int32_t glance_poll_status(glance_ctx *ctx, int32_t *device_status) {
+    if (!ctx || !device_status) return GLANCE_E_INVALID_ARG;
+    int32_t v = 0;
+    if (cudaMemcpyAsync(&v, ctx->ws.status, 4, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return GLANCE_E_CUDA;
+    if (cudaMemsetAsync(ctx->ws.status, 0, 4, ctx->stream) != cudaSuccess) return GLANCE_E_CUDA;
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return GLANCE_E_CUDA;
+    *device_status = v;
+    return GLANCE_OK;
+}
+
+int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t layer, const void *q,
+                               const uint64_t *anc, int32_t T, void *out) {
+    int32_t rc = check_seqs(ctx, seqs);
+    if (rc) return rc;
+    const glance_config &c = ctx->cfg;
+    if (!q || !out || layer < 0 || layer >= c.n_layers || T < 1 || T > std::max(c.tree_N, c.block_B))
+        return GLANCE_E_INVALID_ARG;
+    const KvGeom geom = geom_of(ctx, seqs);
+    AttnParams ap;
+    ap.batch = seqs->batch; ap.T = T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
+    ap.q = (const bf16 *)q; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
+    ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
+    ap.out = (bf16 *)out; ap.S = ctx->dims.S_att; ap.part_o = ctx->ws.att_o; ap.part_ml = ctx->ws.att_ml;
+    ap.counters = ctx->ws.att_ctr; ap.status = ctx->ws.status;
+    LAUNCH(ctx, launch_attention(ap, ctx->stream));
+    return finish(ctx);
+}
+
+int32_t glance_debug_gemm(glance_ctx *ctx, const void *W, const void *X, float *Y, int32_t Nout, int32_t K,
+                          int32_t R, int32_t S) {
+    if (!ctx || !W || !X || !Y) return GLANCE_E_INVALID_ARG;
+    if (Nout < 1 || K < 64 || K % 64 || R < 1 || R > 128 || S < 1 || S > 16) return GLANCE_E_INVALID_ARG;
+    LAUNCH(ctx, launch_gemm((const bf16 *)W, (const bf16 *)X, Y, Nout, K, R, Nout, (size_t)R * Nout, S, ctx->stream));
+    return finish(ctx);
+}
+
+int64_t glance_launch_count(const glance_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

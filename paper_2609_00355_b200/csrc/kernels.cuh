@@ -1,0 +1,125 @@
+// Launch wrappers of the round's kernels (definitions in the .cu files beside this header).
+#pragma once
+#include "common.cuh"
+
+namespace glance {
+
+// ---- setup (kernels_small.cu) -------------------------------------------------------------
+struct VerifySetup {
+    // rows r = s*N + i
+    int batch, N, H, d;
+    float theta;
+    const int32_t *seq_len;     // [batch]
+    const int32_t *token;       // [batch][N] tree tokens (mode tree) or nullptr
+    const int32_t *depth;       // [batch][N] (mode tree) or nullptr (chain: depth = i)
+    const bf16 *row_embeds;     // prefill: [count][H] or nullptr
+    const int32_t *row_ids;     // prefill: [count] or nullptr
+    int count;                  // prefill: valid rows
+    uint64_t *chain_anc;        // prefill: [N][W] written with the causal chain mask
+    const bf16 *embed;          // [V][H]
+    int vocab;
+    int capacity;               // max_pages_per_seq * page
+    float *x;                   // [R][H] fp32 residual stream (out)
+    RowMeta meta;
+    int32_t *status;
+};
+void launch_setup_verify(const VerifySetup &p, cudaStream_t st);
+
+struct DraftSetup {
+    // block rows r = s*B + j (R1 = batch*n_block rows), then feature rows r = R1 + s*FR + i
+    int batch, B, FR, H, d;
+    float theta;
+    const int32_t *seq_len, *root;
+    const bf16 *feat;           // [batch][FR][H]: FR = B (round) or tree_N (prefill head-context update)
+    const int32_t *feat_count;  // [batch] or nullptr (then count_const rows, appended at seq_len)
+    int count_const;
+    int n_block;                // B (round) or 0 (prefill: only feature rows)
+    const bf16 *embed, *mask_embed;
+    int vocab;
+    int capacity;
+    float *x;
+    RowMeta meta;
+    int32_t *status;
+};
+void launch_setup_draft(const DraftSetup &p, cudaStream_t st);
+
+// ---- reductions / elementwise (kernels_small.cu) -----------------------------------------
+// x[r] += sum_s part[s][r][0..H) (fixed order); optional hidden_out = bf16(x); xn = bf16(rms(x) * gain)
+// rows >= split_row use gain_b.
+void launch_norm(float *x, const float *part, int S, size_t part_split_stride, int ldp, int R, int H,
+                 const bf16 *gain_a, const bf16 *gain_b, int split_row, float eps, bf16 *xn, bf16 *hidden_out,
+                 cudaStream_t st);
+
+struct RopeKv {
+    int R, Rq;                  // rows in the pass; rows < Rq also emit q
+    int Hq, Hkv, d;
+    const float *part;          // [S][Rld][ldy] QKV partial sums
+    int S;
+    size_t split_stride;
+    int ldy;
+    RowMeta meta;
+    bf16 *q;                    // [Rq][Hq*d]
+    bf16 *pool_layer;           // base of this layer's pages
+    KvGeom geom;
+    const int32_t *page_table;  // [batch][max_pages_per_seq]
+    int32_t *status;
+};
+void launch_rope_kv(const RopeKv &p, cudaStream_t st);
+
+void launch_swiglu(const float *part, int ldp, int R, int F, bf16 *act, cudaStream_t st);
+void launch_argmax(const float *logits, int R, int V, int32_t *out, cudaStream_t st);
+// rows (s, j), j = 1..L of logits [batch*B][V] -> ids/lp [batch][L][k]
+void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *ids, float *lp, cudaStream_t st);
+
+// ---- tree + walk (tree_walk.cu) -----------------------------------------------------------
+void launch_build_tree(int batch, int N, int L, int k, const int32_t *root, const int32_t *ids, const float *lp,
+                       const glance_tree &out, cudaStream_t st);
+
+struct WalkCommit {
+    int batch, N, B, H, n_layers;
+    const int32_t *token, *parent, *n_nodes;   // tree (walk mode) or nullptr
+    const int32_t *argmax;                      // [batch][N] (walk mode)
+    const int32_t *forced_path, *forced_len, *forced_root;   // forced mode (argmax == nullptr)
+    const bf16 *hidden;                         // [batch][N][H]
+    bf16 *kv_pool;
+    KvGeom geom;
+    const int32_t *page_table;
+    int32_t *seq_len, *root, *feat_count;
+    bf16 *feat;                                 // [batch][B][H]
+    int32_t *accept_len, *path, *out_tokens;    // outputs (may be nullptr in forced mode)
+    int32_t *counters;                          // [batch], zero between calls
+    int32_t *status;
+};
+void launch_walk_commit(const WalkCommit &p, cudaStream_t st);
+
+// prefill bookkeeping: seq_len += count, root = argmax[count-1], feat_count = 0
+void launch_prefill_advance(int32_t *seq_len, int32_t *root, int32_t *feat_count, const int32_t *argmax, int count,
+                            cudaStream_t st);
+
+// ---- attention (attention.cu) -------------------------------------------------------------
+struct AttnParams {
+    int batch, T, Hq, Hkv, d;    // T = query rows per sequence = extra (uncommitted) keys per sequence
+    const bf16 *q;               // [batch*T][Hq*d]
+    const bf16 *pool_layer;
+    KvGeom geom;
+    const int32_t *page_table;
+    const int32_t *seq_len;
+    const uint64_t *anc;         // [batch][T][W] or nullptr (all T extra keys visible)
+    int W;
+    bf16 *out;                   // [batch*T][Hq*d]
+    int S;                       // key splits
+    float *part_o;               // [batch][Hkv][PR][S][d]
+    float *part_ml;              // [batch][Hkv][PR][S][2]
+    int32_t *counters;           // [batch][Hkv][q_tiles], zero between calls
+    int32_t *status;
+};
+void launch_attention(const AttnParams &p, cudaStream_t st);
+int attention_q_tiles(int T, int G);
+
+// ---- weight-streaming GEMM (gemm_mma.cu) --------------------------------------------------
+// Y[s][r][f] = sum over the K range of split s of X[r][k] * W[f][k];  X bf16 [R][K], W bf16 [Nout][K],
+// Y fp32 [S][.][ldy] with split stride `split_stride` elements.  K must be a multiple of 64.
+void launch_gemm(const bf16 *W, const bf16 *X, float *Y, int Nout, int K, int R, int ldy, size_t split_stride,
+                 int S, cudaStream_t st);
+
+}  // namespace glance

@@ -1,0 +1,307 @@
+"""GPU parity tests: the CUDA library, called through its C ABI, against the CPU oracle."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import glance_oracle as O
+from paper_2609_00355_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def harness():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from tests import parity_harness
+    return parity_harness
+
+
+@pytest.fixture(scope="module")
+def tiny_run(harness):
+    return harness.ParityRun(synth.CONFIGS["tiny"])
+
+
+def make_engine(cfg, batch=1, max_len=None):
+    """An engine on random weights without any oracle state (kernel-level tests)."""
+    from paper_2609_00355_b200.binding import Engine
+    tw, hw = synth.make_weights(cfg, "cuda")
+    return Engine(cfg, tw, hw, batch=batch, max_len=max_len)
+
+
+# ------------------------------------------------------------------ GEMM alone
+
+@pytest.mark.parametrize("Nout,K,R,S", [(256, 256, 8, 1), (512, 256, 64, 2), (1408, 256, 16, 1), (1000, 704, 37, 3),
+                                        (4608, 3584, 64, 5), (3584, 18944, 64, 6), (640, 1024, 128, 4), (130, 64, 1, 1)])
+def test_gemm_matches_matmul(tiny_run, Nout, K, R, S):
+    eng = tiny_run.eng
+    g = torch.Generator(device="cuda").manual_seed(Nout + K + R)
+    W = (torch.randn(Nout, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    X = torch.randn(R, K, generator=g, device="cuda").to(torch.bfloat16)
+    Y = torch.full((S, R, Nout), float("nan"), device="cuda")
+    eng.glance_debug_gemm(W, X, Y, S)
+    eng.check_device_status()
+    ref = X.double().cpu() @ W.double().cpu().T
+    got = Y.double().sum(0).cpu()
+    scale = float(ref.abs().max())
+    assert float((got - ref).abs().max()) <= 1e-4 * scale + 1e-5
+    # run-to-run bit reproducibility
+    Y2 = torch.zeros_like(Y)
+    eng.glance_debug_gemm(W, X, Y2, S)
+    assert torch.equal(Y, Y2)
+
+
+# ------------------------------------------------------------------ attention alone
+
+def _fill_cache(eng, seq, layer, K, V):
+    """Write logical rows K,V [n,Hkv,d] of one sequence/layer into the paged pool."""
+    page = eng.cfg.page_size
+    n = K.shape[0]
+    pos = torch.arange(n, device=eng.device)
+    pages = eng.page_table[seq].long()[pos // page]
+    eng.kv_pool[layer, pages, 0, :, pos % page, :] = K.to(torch.bfloat16)
+    eng.kv_pool[layer, pages, 1, :, pos % page, :] = V.to(torch.bfloat16)
+
+
+def test_attention_mask_bits_one_hot(harness):
+    """Every (row, key) mask bit changes the output by O(1): tree keys dominate, values are one-hot."""
+    cfg = synth.CONFIGS["tiny"].replace(tree_N=64, vocab=256, n_layers=2)
+    eng = make_engine(cfg, max_len=320)
+    rng = np.random.default_rng(3)
+    N, Hq, Hkv, d = 64, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    for P in (0, 3, 64, 70):
+        tok, par, dep = synth.random_tree(N, 15, 1000, rng)
+        tree = O.tree_from_arrays(tok, par, dep)
+        n = P + N
+        # context keys score 0, tree key j scores 5 on every query (q = 1): visible tree keys dominate the
+        # softmax, and value j is one-hot at dim j mod d, so each output dim reports one tree key's weight
+        K = torch.zeros(n, Hkv, d)
+        V = torch.zeros(n, Hkv, d)
+        for j in range(P, n):
+            K[j, :, j % d] = 5.0 * math.sqrt(d)
+            V[j, :, j % d] = 1.0
+        V[:P, :, 0] = -1.0
+        q = torch.ones(N, Hq, d)
+        eng.seq_len[0] = P
+        # poison the rows after the last key: they must never contribute
+        Kp = torch.cat([K, torch.full((8, Hkv, d), float("nan"))])
+        Vp = torch.cat([V, torch.full((8, Hkv, d), float("nan"))])
+        _fill_cache(eng, 0, 1, Kp.cuda(), Vp.cuda())
+        out = torch.zeros(N, Hq * d, dtype=torch.bfloat16, device="cuda")
+        anc = torch.from_numpy(tree.anc.view(np.int64)).cuda()[None].contiguous()
+        eng.glance_debug_attention(1, q.to(torch.bfloat16).cuda().reshape(N, Hq * d).contiguous(), anc, N, out)
+        eng.check_device_status()
+        vis = O.visibility(tree, P)
+        ref = O.attention(q, K, V, vis)
+        got = out.float().cpu().reshape(N, Hq, d)
+        assert torch.isfinite(got).all()
+        assert float((got - ref).abs().max()) < 0.01
+        # any single flipped tree-key bit would move the reference by far more than the tolerance
+        for (i, j) in [(N - 1, 1), (5, 5), (17, 3), (40, 40)]:
+            m2 = vis.clone()
+            m2[i, P + j] = ~m2[i, P + j]
+            if m2[i, P:].any():
+                assert float((O.attention(q, K, V, m2) - ref).abs().max()) > 0.04
+
+
+@pytest.mark.parametrize("name,P,T", [("tiny", 300, 8), ("small", 704, 32), ("7b", 1536, 64), ("7b", 100, 128)])
+def test_attention_random_inputs(harness, name, P, T):
+    base = synth.CONFIGS[name]
+    cfg = base.replace(n_layers=1, vocab=256, ffn=64, hidden=64, tree_N=T, n_img=2, n_txt=1, rounds=1)
+    eng = make_engine(cfg, batch=2, max_len=P + T + 64)
+    rng = np.random.default_rng(P + T)
+    g = torch.Generator().manual_seed(P)
+    Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    Ps = [P, max(1, P // 3)]
+    qs, refs, ancs = [], [], []
+    for s in range(2):
+        tok, par, dep = synth.random_tree(T, 15, 1000, rng)
+        tree = O.tree_from_arrays(tok, par, dep)
+        K = torch.randn(Ps[s] + T, Hkv, d, generator=g).to(torch.bfloat16)
+        V = torch.randn(Ps[s] + T, Hkv, d, generator=g).to(torch.bfloat16)
+        q = (torch.randn(T, Hq, d, generator=g) * 1.5).to(torch.bfloat16)
+        eng.seq_len[s] = Ps[s]
+        _fill_cache(eng, s, 0, K.cuda(), V.cuda())
+        refs.append(O.attention(q.float(), K.float(), V.float(), O.visibility(tree, Ps[s])))
+        qs.append(q.reshape(T, Hq * d))
+        ancs.append(torch.from_numpy(tree.anc.view(np.int64)))
+    out = torch.zeros(2 * T, Hq * d, dtype=torch.bfloat16, device="cuda")
+    eng.glance_debug_attention(0, torch.cat(qs).cuda().contiguous(), torch.stack(ancs).cuda().contiguous(), T, out)
+    eng.check_device_status()
+    out2 = torch.zeros_like(out)
+    eng.glance_debug_attention(0, torch.cat(qs).cuda().contiguous(), torch.stack(ancs).cuda().contiguous(), T, out2)
+    assert torch.equal(out, out2)                       # split merge is order-fixed: run-to-run identical
+    for s in range(2):
+        got = out[s * T:(s + 1) * T].float().cpu().reshape(T, Hq, d)
+        assert float((got - refs[s]).abs().max()) <= 2e-2 * float(refs[s].abs().max())
+    # no mask = every extra key visible (the draft block's bidirectional attention)
+    eng.glance_debug_attention(0, torch.cat(qs).cuda().contiguous(), None, T, out)
+    for s in range(2):
+        full = torch.ones(T, Ps[s] + T, dtype=torch.bool)
+        Kf, Vf = eng.gather_kv(s, 0, Ps[s] + T)
+        ref = O.attention(qs[s].float().reshape(T, Hq, d), Kf.float().cpu(), Vf.float().cpu(), full)
+        got = out[s * T:(s + 1) * T].float().cpu().reshape(T, Hq, d)
+        assert float((got - ref).abs().max()) <= 2e-2 * float(ref.abs().max())
+
+
+# ------------------------------------------------------------------ tree builder (bit-exact)
+
+@pytest.mark.parametrize("name", ["tiny", "small", "7b", "long"])
+def test_build_tree_bit_exact(harness, tiny_run, name):
+    base = synth.CONFIGS[name]
+    cfg = synth.CONFIGS["tiny"].replace(block_B=base.block_B, topk=base.topk, tree_N=base.tree_N, n_img=2, n_txt=1,
+                                        rounds=1, vocab=256)
+    eng = make_engine(cfg, batch=3)
+    rng = np.random.default_rng(17)
+    L, k, N = cfg.L, cfg.topk, cfg.tree_N
+    for trial in range(6):
+        ids = np.zeros((3, L, k), dtype=np.int32)
+        lp = np.zeros((3, L, k), dtype=np.float32)
+        for s in range(3):
+            if trial % 3 == 2:
+                lp[s] = synth.controlled_marginals([0.3, 0.6, 0.9][s], k, L)
+                ids[s] = rng.integers(0, 1000, size=(L, k))
+            else:
+                ids[s], lp[s] = synth.random_topk(L, k, 1000, rng, ties=(trial % 3 == 1))
+        roots = torch.tensor([5, 6, 7], dtype=torch.int32, device="cuda")
+        eng.glance_build_tree(torch.from_numpy(ids).cuda(), torch.from_numpy(lp).cuda(), root=roots)
+        eng.check_device_status()
+        for s in range(3):
+            harness.assert_tree_bits(harness.tree_from_device(eng.tree, s), O.build_tree(5 + s, ids[s], lp[s], N))
+
+
+# ------------------------------------------------------------------ walk + commit (bit-exact)
+
+def test_walk_commit_examples_and_compaction_hazard(harness):
+    cfg = synth.CONFIGS["tiny"]
+    run = harness.ParityRun(cfg, ctx_lens=[(40, 9)])
+    eng = run.eng
+    ex_parent = [-1, 0, 0, 1, 1, 2, 3, 4]
+    ex_depth = [0, 1, 1, 2, 2, 2, 3, 3]
+    ex_token = [7, 11, 12, 21, 22, 23, 31, 32]
+    tree = O.tree_from_arrays(ex_token, ex_parent, ex_depth)
+    harness.tree_to_device(eng, [tree])
+    cases = [([11, 22, 0, 0, 99, 0, 0, 0], (2, [0, 1, 4], [11, 22], 99)),
+             ([12, 0, 23, 0, 0, 5, 0, 0], (2, [0, 2, 5], [12, 23], 5)),       # row P+2: source, then destination
+             ([13, 0, 0, 0, 0, 0, 0, 0], (0, [0], [], 13)),
+             ([11, 21, 0, 31, 0, 0, 44, 0], (3, [0, 1, 3, 6], [11, 21, 31], 44))]
+    for am, expect in cases:
+        assert O.walk(tree, np.array(am)) == expect
+        P = int(eng.seq_len[0])
+        # distinct recognisable bytes in every scratch row
+        for i in range(8):
+            pos = P + i
+            pg = int(eng.page_table[0, pos // 64])
+            eng.kv_pool[:, pg, :, :, pos % 64, :] = float(i + 1)
+        eng.hidden.copy_(torch.arange(8, device="cuda")[None, :, None].expand_as(eng.hidden).to(torch.bfloat16))
+        before = eng.kv_pool.clone()
+        eng.argmax.copy_(torch.tensor([am], dtype=torch.int32))
+        eng.glance_accept_commit()
+        eng.check_device_status()
+        a, path, out, new_root = expect
+        assert int(eng.accept_len[0]) == a
+        assert eng.path[0, :a + 1].tolist() == path and eng.path[0, a + 1:].tolist() == [-1] * (cfg.block_B - a - 1)
+        assert eng.out_tokens[0, :a + 1].tolist() == out + [new_root]
+        assert int(eng.seq_len[0]) == P + a + 1 and int(eng.root[0]) == new_root and int(eng.feat_count[0]) == a + 1
+        run._check_compaction(0, P, path, before)
+        assert eng.feat[0, :a + 1, 0].float().tolist() == [float(v) for v in path]
+
+
+def test_commit_forced_and_bad_path_is_reported(harness):
+    cfg = synth.CONFIGS["tiny"]
+    run = harness.ParityRun(cfg, ctx_lens=[(20, 5)])
+    eng = run.eng
+    P = int(eng.seq_len[0])
+    before = eng.kv_pool.clone()
+    path = torch.tensor([[0, 3, 7, -1]], dtype=torch.int32, device="cuda")
+    eng.glance_commit_forced(path, torch.tensor([3], dtype=torch.int32, device="cuda"),
+                             torch.tensor([42], dtype=torch.int32, device="cuda"))
+    eng.check_device_status()
+    assert int(eng.seq_len[0]) == P + 3 and int(eng.root[0]) == 42
+    run._check_compaction(0, P, [0, 3, 7], before)
+    # a non-increasing path is rejected by the device-side check (status word, no fault)
+    bad = torch.tensor([[0, 5, 2, -1]], dtype=torch.int32, device="cuda")
+    eng.glance_commit_forced(bad, torch.tensor([3], dtype=torch.int32, device="cuda"),
+                             torch.tensor([1], dtype=torch.int32, device="cuda"))
+    assert eng.glance_poll_status() == -6
+    assert eng.glance_poll_status() == 0
+
+
+def test_capacity_overflow_sets_status_not_fault(harness):
+    cfg = synth.CONFIGS["tiny"]
+    run = harness.ParityRun(cfg, ctx_lens=[(20, 5)])
+    eng = run.eng
+    eng.seq_len[0] = eng.pages_per_seq * 64 - 2          # P + N exceeds the page budget
+    eng.glance_verify_tree()
+    assert eng.glance_poll_status() in (-3, -6)
+
+
+# ------------------------------------------------------------------ the whole round, stage by stage
+
+def test_prefill_state_tiny(tiny_run):
+    tiny_run.check_state()
+    tiny_run.check_head_state()
+
+
+def test_rounds_tiny_drafted_trees(tiny_run):
+    """Tiny config, trees from the library's own draft (random head: short accepts)."""
+    for _ in range(4):
+        tiny_run.round()
+    tiny_run.check_head_state()
+
+
+def test_rounds_tiny_controlled_match(tiny_run):
+    """Tiny config, 16 rounds at p_m = 0.7: accepted paths, compaction and state after every round."""
+    for _ in range(16):
+        tiny_run.round(p_m=0.7)
+    tiny_run.check_head_state()
+    st = tiny_run.stats
+    print("tiny parity stats:", st)
+    assert st["accepted"] > 0
+    assert st["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_tiny_single_node_is_plain_ar(harness):
+    """tree_N = 1 rounds commit exactly one token each (tau = 1) and follow the oracle's greedy stream."""
+    cfg = synth.CONFIGS["tiny"].replace(tree_N=1)
+    run = harness.ParityRun(cfg, ctx_lens=[(50, 14)])
+    for _ in range(6):
+        run.round(check_draft=False)
+    assert run.stats["accepted"] == 0 and run.stats["rounds"] == 6
+
+
+@pytest.mark.parametrize("p_m", [0.3, 0.6, 0.9])
+def test_rounds_small(harness, p_m):
+    cfg = synth.CONFIGS["small"]
+    run = harness.ParityRun(cfg)
+    run.check_state()
+    run.check_head_state()
+    for r in range(6):
+        run.round(p_m=p_m, check_draft=(r < 2))
+    run.check_head_state()
+    print("small parity stats p_m", p_m, run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_batch3_ragged(harness):
+    """Three sequences with different context lengths and trees in one call (ragged accepts)."""
+    cfg = synth.CONFIGS["tiny"].replace(tree_N=16, block_B=6, topk=3)
+    run = harness.ParityRun(cfg, batch=3, ctx_lens=[(100, 30), (17, 3), (200, 57)])
+    run.check_state()
+    for _ in range(5):
+        run.round(p_m=0.75)
+    run.check_head_state()
+    print("batch parity stats:", run.stats)
+
+
+def test_round_7b_shape_one_layer_slice(harness):
+    """Full 7B widths (hidden 3584, 28/4 heads of 128, FFN 18944, N 64) on 2 layers and a reduced vocabulary:
+    the launch configuration of the benchmark's per-layer kernels, small enough for the oracle."""
+    cfg = synth.CONFIGS["7b"].replace(n_layers=2, vocab=4096, n_img=150, n_txt=43, rounds=4)
+    run = harness.ParityRun(cfg)
+    run.check_state()
+    for r in range(3):
+        run.round(p_m=0.8, check_draft=(r == 0))
+    print("7b-slice parity stats:", run.stats)
