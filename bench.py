@@ -1,0 +1,418 @@
+#!/usr/bin/env python
+"""Benchmark of the GLANCE speculative round on B200: committed tokens/s at the 7B-shape config.
+
+One step = one speculative round (glance_draft_block -> glance_build_tree -> glance_verify_tree ->
+glance_accept_commit) over one batch of synthetic input.  Candidate trees are generated at a controlled
+per-depth match probability p_m against the model's own greedy continuation, which an untimed look-ahead
+(single-node rounds, then a state rollback) obtains before every round.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 7b] [--impl reference]
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2609_00355_b200 import synth
+
+METRIC = "committed_tokens_per_s"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return float(p["hbm_gbs"]), "measured (MEASURED_PEAKS.json, sustained copy)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+def round_algorithmic_bytes(cfg) -> float:
+    """Bytes one round must move: every weight once per pass, context K/V read once per layer, tree K/V written."""
+    H, F, V, d = cfg.hidden, cfg.ffn, cfg.vocab, cfg.head_dim
+    qkv = (cfg.n_q_heads + 2 * cfg.n_kv_heads) * d
+    layer = 2.0 * (qkv * H + H * cfg.n_q_heads * d + 2 * F * H + H * F)
+    P = cfg.ctx
+    kv_layer = 2.0 * P * cfg.n_kv_heads * d * 2
+    target = cfg.n_layers * (layer + kv_layer + 2.0 * cfg.tree_N * cfg.n_kv_heads * d * 2) + 2.0 * V * H
+    head = layer + kv_layer + 2.0 * V * H
+    return target + head
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.gpu_index)],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, mx = [], set(), None
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    mx = float(parts[2])
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=mx, samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def to_device(w, dev):
+    if isinstance(w, dict):
+        return {k: to_device(v, dev) for k, v in w.items()}
+    if isinstance(w, list):
+        return [to_device(v, dev) for v in w]
+    return w.to(dev)
+
+
+class RoundBench:
+    """Drives rounds of the library at controlled p_m.  All method arithmetic runs in the CUDA library."""
+
+    def __init__(self, cfg, device, rank=0, weights=None):
+        from paper_2609_00355_b200.binding import Engine, TreeBuffers
+        self.cfg, self.dev = cfg, device
+        self.tw, self.hw = weights if weights is not None else synth.make_weights(cfg, device)
+        self.eng = Engine(cfg, self.tw, self.hw, batch=cfg.batch)
+        eng = self.eng
+        lens = [cfg.ctx] * cfg.batch
+        if cfg.batch > 1:
+            lens = synth.batch_context_lengths(cfg)
+            self.p_ms = synth.batch_match_probs(cfg)
+        else:
+            self.p_ms = [cfg.p_m]
+        for s in range(cfg.batch):
+            n_img = cfg.n_img if cfg.batch == 1 else int(lens[s] * 0.75)
+            n_txt = lens[s] - n_img
+            img, ids = synth.make_context(cfg, device, seed=1 + s + 100 * rank, n_img=n_img, n_txt=n_txt)
+            eng.prefill_context(s, img, ids)
+        eng.check_device_status()
+        # single-node trees for the look-ahead (plain greedy steps through the same library)
+        self.ar_tree = TreeBuffers(cfg.batch, cfg.tree_N, device)
+        N, W = cfg.tree_N, (cfg.tree_N + 63) // 64
+        anc = np.zeros((N, W), dtype=np.uint64)
+        for i in range(N):
+            anc[i, i >> 6] = np.uint64(1) << np.uint64(i & 63)
+        self.ar_tree.anc.copy_(torch.from_numpy(anc.view(np.int64))[None].expand(cfg.batch, N, W))
+        self.rng = np.random.default_rng(3 + rank)
+        L, k = cfg.L, cfg.topk
+        self.lp_host = torch.from_numpy(np.stack([synth.controlled_marginals(p, k, L) for p in self.p_ms])).pin_memory()
+        self.ids_host = torch.zeros(cfg.batch, L, k, dtype=torch.int32).pin_memory()
+        self.cand_ids = torch.zeros(cfg.batch, L, k, dtype=torch.int32, device=device)
+        self.cand_lp = self.lp_host.to(device)
+        self.res_host = torch.zeros(cfg.batch, 1 + cfg.block_B, dtype=torch.int32).pin_memory()
+        self.res_dev = torch.zeros(cfg.batch, 1 + cfg.block_B, dtype=torch.int32, device=device)
+
+    def lookahead(self):
+        """Untimed: the next L greedy tokens after the pending root (single-node rounds, then rollback)."""
+        eng, cfg = self.eng, self.cfg
+        snap = eng.snapshot_state()
+        ys = []
+        for _ in range(cfg.L):
+            self.ar_tree.token[:, 0].copy_(eng.root)
+            eng.glance_verify_tree(tree=self.ar_tree)
+            eng.glance_accept_commit(tree=self.ar_tree)
+            ys.append(eng.root.clone())
+        eng.restore_state(snap)
+        return torch.stack(ys, dim=1).cpu().numpy()      # [batch][L]
+
+    def make_candidates(self, Y):
+        cfg = self.cfg
+        for s in range(cfg.batch):
+            self.ids_host[s] = torch.from_numpy(
+                synth.controlled_candidates(list(Y[s]), self.p_ms[s], cfg.topk, cfg.L, cfg.vocab, self.rng))
+
+    def round_device(self):
+        """The four calls of one round, inputs already on the device."""
+        eng = self.eng
+        eng.glance_draft_block()
+        eng.glance_build_tree(self.cand_ids, self.cand_lp)
+        eng.glance_verify_tree()
+        eng.glance_accept_commit()
+
+    def round_e2e(self):
+        """Same round with this step's inputs copied from pinned host memory and the result read back."""
+        eng = self.eng
+        self.cand_ids.copy_(self.ids_host, non_blocking=True)
+        self.cand_lp.copy_(self.lp_host, non_blocking=True)
+        self.round_device()
+        self.res_dev[:, 0].copy_(eng.accept_len)
+        self.res_dev[:, 1:].copy_(eng.out_tokens)
+        self.res_host.copy_(self.res_dev, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return self.res_host[:, 0].clone()
+
+
+class OracleSample:
+    """Times the CPU oracle (as it stands) on a bounded sample of one round and scales to the full depth.
+
+    Sample: one draft pass (full head layer + LM head over the block) + verify passes over the first `layers_a`
+    and `layers_b` target layers (N rows, full LM head, argmax, walk) against a context of the configured
+    length filled with random K/V.  Per-layer cost = (t_b - t_a) / (layers_b - layers_a); the round estimate
+    adds the remaining layers at that cost.
+    """
+
+    def __init__(self, cfg, tw_any, hw_any, layers_a=1, layers_b=2):
+        from oracle import glance_oracle as O
+        self.O, self.cfg = O, cfg
+        self.sh = O.Shape.of(cfg)
+        self.lb = min(layers_b, cfg.n_layers)
+        self.la = min(layers_a, self.lb)
+        cpu = lambda t: t.detach().to("cpu").float()
+        self.tw = {"embed": cpu(tw_any["embed"]), "lm_head": cpu(tw_any["lm_head"]), "final_norm": cpu(tw_any["final_norm"]),
+                   "layers": [{k: cpu(v) for k, v in lw.items()} for lw in tw_any["layers"][:self.lb]]}
+        self.hw = {k: cpu(v) for k, v in hw_any.items()}
+        P, N = cfg.ctx, cfg.tree_N
+        g = torch.Generator().manual_seed(0)
+        cap = P + N + 16
+        mk = lambda: torch.randn(cap, cfg.n_kv_heads, cfg.head_dim, generator=g) * 0.3
+        self.st = O.SeqState(P, 1, [mk() for _ in range(self.lb)], [mk() for _ in range(self.lb)], mk(), mk(),
+                             torch.randn(cap, cfg.hidden, generator=g))
+        self.ids, self.lp = synth.random_topk(cfg.L, cfg.topk, cfg.vocab, np.random.default_rng(0))
+        self.desc = (f"1 round = draft pass (full) + verify of {self.la} and {self.lb} of {cfg.n_layers} layers with full LM "
+                     f"head, N={N}, ctx={P} random K/V; per-layer cost extrapolated to {cfg.n_layers} layers")
+        self.threads = torch.get_num_threads()
+
+    def _verify(self, n_layers, tree):
+        O, sh = self.O, self.sh
+        sub = dict(self.tw, layers=self.tw["layers"][:n_layers])
+        sh_n = O.Shape(n_layers, sh.hidden, sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.ffn, sh.vocab, sh.rms_eps, sh.rope_theta)
+        t = time.perf_counter()
+        logits, hidden = O.verify_tree(sh_n, sub, self.st, tree)
+        O.walk(tree, O.argmax_lowest(logits))
+        return time.perf_counter() - t
+
+    def round_seconds(self) -> float:
+        O, cfg = self.O, self.cfg
+        t0 = time.perf_counter()
+        dl = O.draft_block(self.sh, self.tw, self.hw, self.st, cfg.block_B)
+        O.topk_logprobs(dl, cfg.topk)
+        tree = O.build_tree(1, self.ids, self.lp, cfg.tree_N)
+        t_draft = time.perf_counter() - t0
+        tb = self._verify(self.lb, tree)
+        if self.lb > self.la:
+            ta = self._verify(self.la, tree)
+            per_layer = max((tb - ta) / (self.lb - self.la), 0.0)
+        else:
+            per_layer = tb / self.lb
+        return t_draft + tb + per_layer * (cfg.n_layers - self.lb)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=48)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="7b")
+    ap.add_argument("--impl", default="glance", choices=["glance", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = synth.CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    warmup = max(args.warmup, 3) if args.impl == "glance" else args.warmup
+    expected_tau = 1.0 + sum(cfg.p_m ** l for l in range(1, cfg.L + 1))
+    config = {"workload": f"{cfg.name}: {cfg.n_layers}L h{cfg.hidden} {cfg.n_q_heads}q/{cfg.n_kv_heads}kv d{cfg.head_dim} "
+                          f"ffn{cfg.ffn} V{cfg.vocab}; ctx {cfg.n_img} image + {cfg.n_txt} text; B={cfg.block_B} k={cfg.topk} "
+                          f"N={cfg.tree_N} p_m={cfg.p_m} batch {cfg.batch}",
+              "l2": "inputs larger than L2: every round streams all weights (~15 GB at the 7B shape) and an untimed "
+                    "look-ahead of L verify passes runs between timed rounds",
+              "replicas": world}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        torch.manual_seed(0)
+        tw, hw = synth.make_weights(cfg.replace(n_layers=min(cfg.n_layers, 2)), "cpu")
+        sample = OracleSample(cfg, tw, hw)
+        desc, threads = sample.desc, sample.threads
+        times = []
+        for i in range(args.warmup + args.steps):
+            t = sample.round_seconds()
+            if i >= args.warmup:
+                times.append(t)
+        t_round = sum(times) / max(len(times), 1)
+        value = expected_tau / t_round
+        line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_round * 1e3, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                 "sample": desc + f"; committed tokens per round taken as the closed form tau = {expected_tau:.3f}"},
+                "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    from paper_2609_00355_b200 import build as glance_build
+    glance_build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist_mod.init_process_group("nccl", device_id=dev)
+        dist = dist_mod
+    torch.manual_seed(0)
+    bench = RoundBench(cfg, dev, rank)
+    eng = bench.eng
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident arm -------------------------------------------------------------------
+    round_ms, committed = [], 0
+    sampler = ClockSampler(local_rank)
+    for step in range(warmup + args.steps):
+        Y = bench.lookahead()
+        bench.make_candidates(Y)
+        bench.cand_ids.copy_(bench.ids_host)
+        if step == warmup:
+            barrier()
+            sampler.start()
+        torch.cuda.synchronize()
+        if step >= warmup:
+            eng.glance_profile_enable(True)      # per-launch GEMM events, timed rounds only
+        start.record()
+        bench.round_device()
+        stop.record()
+        torch.cuda.synchronize()
+        eng.glance_profile_enable(False)
+        if step >= warmup:
+            round_ms.append(start.elapsed_time(stop))
+            committed += int(eng.accept_len.sum().item()) + cfg.batch
+    barrier()
+    clocks = sampler.stop()
+    gemm_ms, gemm_bytes, gemm_launches = eng.glance_profile_read()
+    eng.check_device_status()
+    # launches inside the timed regions only (look-ahead launches excluded): measure one round's count
+    l0 = eng.glance_launch_count()
+    bench.cand_ids.copy_(bench.ids_host)
+    snap = eng.snapshot_state()
+    bench.round_device()
+    launches_per_round = eng.glance_launch_count() - l0
+    eng.restore_state(snap)
+
+    # ---- end-to-end arm: host buffers, copies inside the timed region ----------------------------
+    e2e_s, e2e_committed = 0.0, 0
+    for step in range(warmup + args.steps):
+        Y = bench.lookahead()
+        bench.make_candidates(Y)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        acc = bench.round_e2e()
+        dt = time.perf_counter() - t0
+        if step >= warmup:
+            e2e_s += dt
+            e2e_committed += int(acc.sum()) + cfg.batch
+    eng.check_device_status()
+
+    total_ms = sum(round_ms)
+    stats = torch.tensor([total_ms, float(committed), e2e_s, float(e2e_committed)], dtype=torch.float64, device=dev)
+    if dist is not None:
+        mx = stats.clone()
+        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+        sm = stats.clone()
+        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+        total_ms, e2e_s = float(mx[0]), float(mx[2])
+        committed, e2e_committed = float(sm[1]), float(sm[3])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    value = committed / (total_ms * 1e-3)
+    ms_per_step = total_ms / args.steps
+    peak, peak_src = load_peaks()
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+    round_bytes = round_algorithmic_bytes(cfg)
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": config,
+        "round_us": {"mean": 1e3 * ms_per_step, "median": 1e3 * statistics.median(round_ms)},
+        "tau": committed / (args.steps * cfg.batch * world), "tau_expected": expected_tau,
+        "round_hbm": {"algorithmic_gb": round_bytes / 1e9, "achieved_gbs": round_bytes / (ms_per_step * 1e-3) / 1e9,
+                      "frac_of_measured_peak": round_bytes / (ms_per_step * 1e-3) / 1e9 / peak},
+        "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections, MLP, LM head)",
+                     "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
+                     "traffic": None, "peak_source": peak_src, "launches_timed": gemm_launches,
+                     "avg_launch_us": 1e3 * gemm_ms / max(gemm_launches, 1),
+                     "algorithmic_bytes_per_launch": gemm_bytes / max(gemm_launches, 1),
+                     "share_of_round_time": gemm_ms / total_ms if world == 1 else None},
+        "e2e": {"value": e2e_committed / e2e_s, "unit": UNIT,
+                "h2d_bytes_per_step": int(bench.ids_host.numel() * 4 + bench.lp_host.numel() * 4),
+                "d2h_bytes_per_step": int(bench.res_host.numel() * 4)},
+        "gpu_launches": int(launches_per_round * args.steps),
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+    }
+    if not args.no_cpu_baseline and world == 1:
+        sample = OracleSample(cfg, bench.tw, bench.hw)
+        t_round, desc, threads = sample.round_seconds(), sample.desc, sample.threads
+        tau = line["tau"]
+        line["cpu_baseline"] = {"value": tau / t_round, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": desc + f"; committed tokens per round = the GPU run's measured {tau:.3f}",
+                                "s_per_round": t_round}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

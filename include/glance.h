@@ -175,6 +175,15 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
 int32_t glance_debug_gemm(glance_ctx *ctx, const void *W, const void *X, float *Y, int32_t Nout, int32_t K,
                           int32_t R, int32_t S);
 
+/* Measurement aid.  While enabled, every launch of the weight-streaming GEMM kernel is bracketed by a pair
+ * of CUDA events on the context's stream (the pairs are created when profiling is enabled, so the round
+ * calls still allocate nothing).  glance_profile_read synchronises the stream, returns the summed device
+ * time of those launches in milliseconds, their summed algorithmic bytes (weights once + activations in +
+ * results out) and their count, and resets the tally.  Disabling only pauses the tally.  At most 8192
+ * launches are tallied per read. */
+int32_t glance_profile_enable(glance_ctx *ctx, int32_t on);
+int32_t glance_profile_read(glance_ctx *ctx, double *gemm_ms, double *gemm_bytes, int64_t *gemm_launches);
+
 /* Number of kernel launches enqueued by this context since creation (host counter). */
 int64_t glance_launch_count(const glance_ctx *ctx);
 

@@ -18,7 +18,7 @@ EXPORTS = [
     "glance_status_string", "glance_workspace_bytes", "glance_create", "glance_destroy", "glance_prefill",
     "glance_seq_truncate", "glance_draft_block", "glance_build_tree", "glance_verify_tree",
     "glance_accept_commit", "glance_commit_forced", "glance_poll_status", "glance_launch_count",
-    "glance_debug_attention", "glance_debug_gemm",
+    "glance_debug_attention", "glance_debug_gemm", "glance_profile_enable", "glance_profile_read",
 ]
 
 
@@ -94,6 +94,10 @@ def load_library() -> C.CDLL:
     lib.glance_debug_gemm.restype = C.c_int32
     lib.glance_debug_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                       C.c_int32]
+    lib.glance_profile_enable.restype = C.c_int32
+    lib.glance_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+    lib.glance_profile_read.restype = C.c_int32
+    lib.glance_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.glance_launch_count.restype = C.c_int64
     lib.glance_launch_count.argtypes = [C.c_void_p]
     _lib = lib
@@ -257,6 +261,14 @@ class Engine:
     def glance_debug_gemm(self, W: torch.Tensor, X: torch.Tensor, Y: torch.Tensor, S: int):
         _check(self.lib.glance_debug_gemm(self.ctx, _ptr(W), _ptr(X), _ptr(Y), W.shape[0], W.shape[1], X.shape[0], S),
                "glance_debug_gemm")
+
+    def glance_profile_enable(self, on: bool):
+        _check(self.lib.glance_profile_enable(self.ctx, 1 if on else 0), "glance_profile_enable")
+
+    def glance_profile_read(self):
+        ms, by, n = C.c_double(0), C.c_double(0), C.c_int64(0)
+        _check(self.lib.glance_profile_read(self.ctx, C.byref(ms), C.byref(by), C.byref(n)), "glance_profile_read")
+        return ms.value, by.value, n.value
 
     def glance_launch_count(self) -> int:
         return int(self.lib.glance_launch_count(self.ctx))

@@ -127,6 +127,11 @@ struct glance_ctx {
     std::vector<const bf16 *> ln1, wqkv, wo, ln2, wgu, wd;
     glance_head_weights head;
     int64_t launches;
+    // optional per-launch timing of the GEMM kernel
+    bool profiling = false;
+    std::vector<cudaEvent_t> ev;      // 2 per tallied launch
+    std::vector<double> ev_bytes;
+    size_t ev_used = 0;
 };
 
 namespace {
@@ -136,6 +141,22 @@ namespace {
         call;             \
         (ctx)->launches++; \
     } while (0)
+
+constexpr size_t kMaxProfiled = 8192;
+
+// the weight-streaming GEMM, optionally bracketed by events
+void gemm(glance_ctx *ctx, const bf16 *W, const bf16 *X, float *Y, int Nout, int K, int R, int ldy, size_t split_stride,
+          int S) {
+    const bool prof = ctx->profiling && ctx->ev_used < kMaxProfiled;
+    if (prof) cudaEventRecord(ctx->ev[2 * ctx->ev_used], ctx->stream);
+    launch_gemm(W, X, Y, Nout, K, R, ldy, split_stride, S, ctx->stream);
+    ctx->launches++;
+    if (prof) {
+        cudaEventRecord(ctx->ev[2 * ctx->ev_used + 1], ctx->stream);
+        ctx->ev_bytes[ctx->ev_used] = 2.0 * Nout * K + 2.0 * R * K + 4.0 * S * R * Nout;
+        ctx->ev_used++;
+    }
+}
 
 struct LayerW {
     const bf16 *ln2, *wqkv, *wo, *wgu, *wd;
@@ -182,7 +203,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     const int32_t *seq_len = ps.seqs->seq_len + ps.seq_off;
     // QKV projection, split-K planes
     size_t ss = (size_t)ps.R * d.qkv_out;
-    LAUNCH(ctx, launch_gemm(w.wqkv, ws.xn, ws.part, d.qkv_out, c.hidden, ps.R, d.qkv_out, ss, d.S_qkv, st));
+    gemm(ctx, w.wqkv, ws.xn, ws.part, d.qkv_out, c.hidden, ps.R, d.qkv_out, ss, d.S_qkv);
     RopeKv rk;
     rk.R = ps.R; rk.Rq = ps.Rq; rk.Hq = c.n_q_heads; rk.Hkv = c.n_kv_heads; rk.d = c.head_dim;
     rk.part = ws.part; rk.S = d.S_qkv; rk.split_stride = ss; rk.ldy = d.qkv_out;
@@ -199,13 +220,13 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     const int R = ps.Rq;
     // output projection + residual + norm
     ss = (size_t)R * c.hidden;
-    LAUNCH(ctx, launch_gemm(w.wo, ws.attn, ws.part, c.hidden, d.qd, R, c.hidden, ss, d.S_o, st));
+    gemm(ctx, w.wo, ws.attn, ws.part, c.hidden, d.qd, R, c.hidden, ss, d.S_o);
     LAUNCH(ctx, launch_norm(ws.x, ws.part, d.S_o, ss, c.hidden, R, c.hidden, w.ln2, nullptr, R, c.rms_eps, ws.xn,
                             nullptr, st));
     // SwiGLU MLP
-    LAUNCH(ctx, launch_gemm(w.wgu, ws.xn, ws.part, 2 * c.ffn, c.hidden, R, 2 * c.ffn, 0, 1, st));
+    gemm(ctx, w.wgu, ws.xn, ws.part, 2 * c.ffn, c.hidden, R, 2 * c.ffn, 0, 1);
     LAUNCH(ctx, launch_swiglu(ws.part, 2 * c.ffn, R, c.ffn, ws.act, st));
-    LAUNCH(ctx, launch_gemm(w.wd, ws.act, ws.part, c.hidden, c.ffn, R, c.hidden, ss, d.S_d, st));
+    gemm(ctx, w.wd, ws.act, ws.part, c.hidden, c.ffn, R, c.hidden, ss, d.S_d);
     LAUNCH(ctx, launch_norm(ws.x, ws.part, d.S_d, ss, c.hidden, R, c.hidden, next_gain, nullptr, R, c.rms_eps,
                             ws.xn, hidden_out, st));
 }
@@ -225,7 +246,7 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
         run_layer(ctx, w, pool_layer, ps, last ? ctx->final_norm : ctx->ln1[l + 1], last ? hidden_out : nullptr);
     }
     if (argmax) {
-        LAUNCH(ctx, launch_gemm(ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, ps.R, c.vocab, 0, 1, st));
+        gemm(ctx, ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, ps.R, c.vocab, 0, 1);
         LAUNCH(ctx, launch_argmax(logits, ps.R, c.vocab, argmax, st));
     }
 }
@@ -318,6 +339,7 @@ int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, 
 
 int32_t glance_destroy(glance_ctx *ctx) {
     if (!ctx) return GLANCE_E_INVALID_ARG;
+    for (auto &e : ctx->ev) cudaEventDestroy(e);
     delete ctx;
     return GLANCE_OK;
 }
@@ -399,7 +421,7 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
     PassInfo ps{R, R1, batch, B, nullptr, seqs, 0};
     run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, ps, (const bf16 *)ctx->head.final_norm, nullptr);
     float *logits = logits_dbg ? logits_dbg : ws.logits;
-    LAUNCH(ctx, launch_gemm(ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, R1, c.vocab, 0, 1, st));
+    gemm(ctx, ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, R1, c.vocab, 0, 1);
     LAUNCH(ctx, launch_topk(logits, batch, B, c.vocab, c.topk, topk_ids, topk_lp, st));
     return finish(ctx);
 }
@@ -500,8 +522,37 @@ int32_t glance_debug_gemm(glance_ctx *ctx, const void *W, const void *X, float *
                           int32_t R, int32_t S) {
     if (!ctx || !W || !X || !Y) return GLANCE_E_INVALID_ARG;
     if (Nout < 1 || K < 64 || K % 64 || R < 1 || R > 128 || S < 1 || S > 16) return GLANCE_E_INVALID_ARG;
-    LAUNCH(ctx, launch_gemm((const bf16 *)W, (const bf16 *)X, Y, Nout, K, R, Nout, (size_t)R * Nout, S, ctx->stream));
+    gemm(ctx, (const bf16 *)W, (const bf16 *)X, Y, Nout, K, R, Nout, (size_t)R * Nout, S);
     return finish(ctx);
+}
+
+int32_t glance_profile_enable(glance_ctx *ctx, int32_t on) {
+    if (!ctx) return GLANCE_E_INVALID_ARG;
+    if (on && ctx->ev.empty()) {
+        ctx->ev.resize(2 * kMaxProfiled);
+        ctx->ev_bytes.resize(kMaxProfiled);
+        for (auto &e : ctx->ev)
+            if (cudaEventCreate(&e) != cudaSuccess) return GLANCE_E_CUDA;
+    }
+    ctx->profiling = on != 0;     // the tally survives pauses; glance_profile_read resets it
+    return GLANCE_OK;
+}
+
+int32_t glance_profile_read(glance_ctx *ctx, double *gemm_ms, double *gemm_bytes, int64_t *gemm_launches) {
+    if (!ctx || !gemm_ms || !gemm_bytes || !gemm_launches) return GLANCE_E_INVALID_ARG;
+    if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return GLANCE_E_CUDA;
+    double ms = 0.0, bytes = 0.0;
+    for (size_t i = 0; i < ctx->ev_used; ++i) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, ctx->ev[2 * i], ctx->ev[2 * i + 1]) != cudaSuccess) return GLANCE_E_CUDA;
+        ms += t;
+        bytes += ctx->ev_bytes[i];
+    }
+    *gemm_ms = ms;
+    *gemm_bytes = bytes;
+    *gemm_launches = (int64_t)ctx->ev_used;
+    ctx->ev_used = 0;
+    return GLANCE_OK;
 }
 
 int64_t glance_launch_count(const glance_ctx *ctx) { return ctx ? ctx->launches : 0; }
