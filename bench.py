@@ -123,6 +123,7 @@ class RoundBench:
     def __init__(self, cfg, device, rank=0, weights=None):
         from paper_2609_00355_b200.binding import Engine, TreeBuffers
         self.cfg, self.dev = cfg, device
+        self.no_lookahead = False
         self.tw, self.hw = weights if weights is not None else synth.make_weights(cfg, device)
         self.eng = Engine(cfg, self.tw, self.hw, batch=cfg.batch)
         eng = self.eng
@@ -157,6 +158,8 @@ class RoundBench:
     def lookahead(self):
         """Untimed: the next L greedy tokens after the pending root (single-node rounds, then rollback)."""
         eng, cfg = self.eng, self.cfg
+        if self.no_lookahead:
+            return self.rng.integers(0, cfg.vocab, size=(cfg.batch, cfg.L))
         snap = eng.snapshot_state()
         ys = []
         for _ in range(cfg.L):
@@ -257,8 +260,14 @@ def main():
     ap.add_argument("--config", default="7b")
     ap.add_argument("--impl", default="glance", choices=["glance", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of target layers (profiling captures)")
+    ap.add_argument("--no-lookahead", action="store_true",
+                    help="random candidates instead of the look-ahead (profiling captures: fewer launches)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end arm (profiling captures)")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.config]
+    if args.layers > 0:
+        cfg = cfg.replace(n_layers=args.layers, name=f"{cfg.name}-{args.layers}layers")
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -307,6 +316,7 @@ def main():
         dist = dist_mod
     torch.manual_seed(0)
     bench = RoundBench(cfg, dev, rank)
+    bench.no_lookahead = args.no_lookahead
     eng = bench.eng
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -338,7 +348,8 @@ def main():
             committed += int(eng.accept_len.sum().item()) + cfg.batch
     barrier()
     clocks = sampler.stop()
-    gemm_ms, gemm_bytes, gemm_launches = eng.glance_profile_read()
+    prof = eng.glance_profile_read()
+    gemm_ms, gemm_bytes, gemm_launches = prof["gemm"]
     eng.check_device_status()
     # launches inside the timed regions only (look-ahead launches excluded): measure one round's count
     l0 = eng.glance_launch_count()
@@ -350,7 +361,7 @@ def main():
 
     # ---- end-to-end arm: host buffers, copies inside the timed region ----------------------------
     e2e_s, e2e_committed = 0.0, 0
-    for step in range(warmup + args.steps):
+    for step in range(0 if args.no_e2e else warmup + args.steps):
         Y = bench.lookahead()
         bench.make_candidates(Y)
         torch.cuda.synchronize()
@@ -395,7 +406,9 @@ def main():
                      "avg_launch_us": 1e3 * gemm_ms / max(gemm_launches, 1),
                      "algorithmic_bytes_per_launch": gemm_bytes / max(gemm_launches, 1),
                      "share_of_round_time": gemm_ms / total_ms if world == 1 else None},
-        "e2e": {"value": e2e_committed / e2e_s, "unit": UNIT,
+        "kernel_time_share": {k: (v[0] / total_ms if world == 1 else None) for k, v in prof.items()},
+        "kernel_avg_us": {k: (1e3 * v[0] / v[2] if v[2] else None) for k, v in prof.items()},
+        "e2e": {"value": e2e_committed / e2e_s if e2e_s > 0 else None, "unit": UNIT,
                 "h2d_bytes_per_step": int(bench.ids_host.numel() * 4 + bench.lp_host.numel() * 4),
                 "d2h_bytes_per_step": int(bench.res_host.numel() * 4)},
         "gpu_launches": int(launches_per_round * args.steps),

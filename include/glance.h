@@ -170,19 +170,22 @@ int32_t glance_poll_status(glance_ctx *ctx, int32_t *device_status);
 int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t layer, const void *q,
                                const uint64_t *anc, int32_t T, void *out);
 
-/* Test hook: the weight-streaming GEMM alone.  Y[s][r][f] = sum over split s of X[r][k] W[f][k];
- * W (device [Nout][K] bf16), X (device [R][K] bf16), Y (device [S][R][Nout] fp32), K % 64 == 0, R <= 128. */
-int32_t glance_debug_gemm(glance_ctx *ctx, const void *W, const void *X, float *Y, int32_t Nout, int32_t K,
-                          int32_t R, int32_t S);
+/* Test hook: the weight-streaming GEMM kernel alone (K % 64 == 0).  mode 0: Y[s][r][f] fp32 planes (S splits);
+ * mode 1: W = [2F][K] (gate rows then up rows), act (device [R][F] bf16) = silu(gate) * up;
+ * mode 2: argmax (device [R] int32) over f of X W^T with ties to the lowest f, Y (device [R][Nout] fp32) optional. */
+int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const void *X, float *Y, void *act,
+                             int32_t *argmax, int32_t Nout, int32_t K, int32_t R, int32_t S);
 
-/* Measurement aid.  While enabled, every launch of the weight-streaming GEMM kernel is bracketed by a pair
- * of CUDA events on the context's stream (the pairs are created when profiling is enabled, so the round
- * calls still allocate nothing).  glance_profile_read synchronises the stream, returns the summed device
- * time of those launches in milliseconds, their summed algorithmic bytes (weights once + activations in +
- * results out) and their count, and resets the tally.  Disabling only pauses the tally.  At most 8192
- * launches are tallied per read. */
+/* Measurement aid.  While enabled, every kernel launch is bracketed by a pair of CUDA events on the context's
+ * stream (the pairs are created when profiling is first enabled, so the round calls still allocate nothing).
+ * glance_profile_read synchronises the stream and fills three arrays of GLANCE_PROFILE_KINDS entries, indexed by
+ * kernel kind (0 weight-streaming GEMM, 1 attention, 2 residual+norm, 3 rotary + K/V write, 4 everything
+ * else): summed device time in milliseconds, summed algorithmic bytes (GEMM only: weights once +
+ * activations in + results out) and launch count; then it resets the tally.  Disabling only pauses the
+ * tally.  At most 32768 launches are tallied per read. */
+#define GLANCE_PROFILE_KINDS 5
 int32_t glance_profile_enable(glance_ctx *ctx, int32_t on);
-int32_t glance_profile_read(glance_ctx *ctx, double *gemm_ms, double *gemm_bytes, int64_t *gemm_launches);
+int32_t glance_profile_read(glance_ctx *ctx, double *ms, double *bytes, int64_t *launches);
 
 /* Number of kernel launches enqueued by this context since creation (host counter). */
 int64_t glance_launch_count(const glance_ctx *ctx);

@@ -92,8 +92,8 @@ def load_library() -> C.CDLL:
     lib.glance_debug_attention.argtypes = [C.c_void_p, C.POINTER(Seqs), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
                                            C.c_void_p]
     lib.glance_debug_gemm.restype = C.c_int32
-    lib.glance_debug_gemm.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
-                                      C.c_int32]
+    lib.glance_debug_gemm.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_int32, C.c_int32, C.c_int32, C.c_int32]
     lib.glance_profile_enable.restype = C.c_int32
     lib.glance_profile_enable.argtypes = [C.c_void_p, C.c_int32]
     lib.glance_profile_read.restype = C.c_int32
@@ -258,17 +258,19 @@ class Engine:
         _check(self.lib.glance_debug_attention(self.ctx, C.byref(self.seqs), layer, _ptr(q), _ptr(anc), T, _ptr(out)),
                "glance_debug_attention")
 
-    def glance_debug_gemm(self, W: torch.Tensor, X: torch.Tensor, Y: torch.Tensor, S: int):
-        _check(self.lib.glance_debug_gemm(self.ctx, _ptr(W), _ptr(X), _ptr(Y), W.shape[0], W.shape[1], X.shape[0], S),
-               "glance_debug_gemm")
+    def glance_debug_gemm(self, mode: int, W, X, Y=None, act=None, argmax=None, S: int = 1):
+        _check(self.lib.glance_debug_gemm(self.ctx, mode, _ptr(W), _ptr(X), _ptr(Y), _ptr(act), _ptr(argmax),
+                                             W.shape[0], W.shape[1], X.shape[0], S), "glance_debug_gemm")
 
     def glance_profile_enable(self, on: bool):
         _check(self.lib.glance_profile_enable(self.ctx, 1 if on else 0), "glance_profile_enable")
 
     def glance_profile_read(self):
-        ms, by, n = C.c_double(0), C.c_double(0), C.c_int64(0)
-        _check(self.lib.glance_profile_read(self.ctx, C.byref(ms), C.byref(by), C.byref(n)), "glance_profile_read")
-        return ms.value, by.value, n.value
+        """Per kernel kind (gemm, attention, norm, rope_kv, other): (ms, algorithmic bytes, launches)."""
+        ms, by, n = (C.c_double * 5)(), (C.c_double * 5)(), (C.c_int64 * 5)()
+        _check(self.lib.glance_profile_read(self.ctx, ms, by, n), "glance_profile_read")
+        names = ("gemm", "attention", "norm", "rope_kv", "other")
+        return {names[i]: (ms[i], by[i], n[i]) for i in range(5)}
 
     def glance_launch_count(self) -> int:
         return int(self.lib.glance_launch_count(self.ctx))

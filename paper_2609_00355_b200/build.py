@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libglance.so")
-SOURCES = ["glance_api.cu", "kernels_small.cu", "tree_walk.cu", "attention.cu", "gemm_mma.cu"]
+SOURCES = ["glance_api.cu", "kernels_small.cu", "tree_walk.cu", "attention.cu", "gemm_tc.cu"]
 
 
 def _stale() -> bool:
@@ -28,7 +28,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-o", LIB]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-lcuda"]
+    cmd += [os.path.join(CSRC, s) for s in SOURCES] 
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

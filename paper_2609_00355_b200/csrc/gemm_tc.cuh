@@ -1,0 +1,35 @@
+// Interface of the tcgen05 weight-streaming GEMM (definitions in gemm_tc.cu).
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace glance {
+
+struct TcGemmArgs {
+    int Nout, K, R, S;          // W [Nout][K], X [R][K]; S = split-K factor (mode 0 only; 1 otherwise)
+    // mode 0: fp32 planes Y[split][r][f]; mode 2: optional fp32 logits Y[r][f] (may be nullptr)
+    float *Y;
+    int ldy;
+    size_t split_stride;
+    // mode 1 (SwiGLU): W holds F gate rows then F up rows; act[r][f] = silu(gate) * up
+    bf16 *act;
+    int F;
+    // mode 2 (arg-max over f): keys[r] packed (value, id) merged with atomicMax; the last CTA writes argmax[r]
+    unsigned long long *keys;
+    int32_t *argmax;
+    int32_t *counter;
+    int32_t *status;
+    // filled by launch_gemm_tc
+    int np, stages;
+    uint32_t tmem_cols;
+};
+
+// 2-D bf16 tensor map {inner = K, rows}, box {64, box_rows}, 128-byte swizzle.  Host call, no device work.
+bool tc_make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows);
+// activation rows per CTA, padded to the UMMA N granularity (box_rows of the X map)
+int tc_row_pad(int R);
+// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max.  map_w box_rows must be 128, map_x box_rows tc_row_pad(R).
+cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, const CUtensorMap &map_x, cudaStream_t st);
+
+}  // namespace glance

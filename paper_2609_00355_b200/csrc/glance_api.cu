@@ -1,9 +1,12 @@
 // C ABI of the GLANCE round library: context, workspace carving, and the stream-ordered sequence of
 // kernels behind each entry point declared in glance.h.
 #include <algorithm>
+#include <map>
 #include <new>
+#include <tuple>
 #include <vector>
 
+#include "gemm_tc.cuh"
 #include "kernels.cuh"
 
 using namespace glance;
@@ -12,11 +15,12 @@ namespace {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// split-K factor of a weight-streaming GEMM: enough CTAs to cover the SMs, at least 8 k-tiles per split
+// split-K factor of a weight-streaming GEMM: as many CTAs as fit one wave of the 148 SMs, at least 8 k-tiles
+// per split
 int choose_split(int Nout, int K) {
     const int tiles = (Nout + 127) / 128;
     const int ktiles = K / 64;
-    int s = (148 + tiles - 1) / tiles;
+    int s = 148 / tiles;
     s = std::min(s, std::max(1, ktiles / 8));
     return std::max(1, std::min(s, 16));
 }
@@ -39,6 +43,10 @@ struct Workspace {
     bf16 *hidden_tmp;      // [N][H] prefill hidden
     int32_t *argmax_tmp;   // [N]
     int32_t *status;
+    unsigned long long *am_keys;   // [Rlog] packed arg-max keys, zero between launches
+    int32_t *am_counter;
+    unsigned long long *topk_cand; // [batch*L][warps][k]
+    float *topk_ml;                // [batch*L][warps][2]
     size_t part_elems;
     size_t total;
 };
@@ -60,7 +68,7 @@ Dims make_dims(const glance_config &c) {
     const int G = c.n_q_heads / c.n_kv_heads;
     d.q_tiles_max = attention_q_tiles(std::max(c.tree_N, c.block_B), G);
     int ctas = attention_q_tiles(c.tree_N, G) * c.n_kv_heads * c.max_batch;
-    d.S_att = std::max(1, std::min(16, (2 * 148 + ctas - 1) / ctas));
+    d.S_att = std::max(1, std::min(8, 148 / ctas));
     d.W = (c.tree_N + 63) / 64;
     return d;
 }
@@ -77,8 +85,7 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     const size_t R = d.Rmax, H = c.hidden;
     w.x = (float *)take(R * H * 4);
     w.xn = (bf16 *)take(R * H * 2);
-    size_t pe = std::max({(size_t)d.S_qkv * R * d.qkv_out, (size_t)d.S_o * R * H, (size_t)R * 2 * c.ffn,
-                          (size_t)d.S_d * R * H});
+    size_t pe = std::max({(size_t)d.S_qkv * R * d.qkv_out, (size_t)d.S_o * R * H, (size_t)d.S_d * R * H});
     w.part_elems = pe;
     w.part = (float *)take(pe * 4);
     w.q = (bf16 *)take(R * d.qd * 2);
@@ -99,6 +106,11 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.hidden_tmp = (bf16 *)take((size_t)c.tree_N * H * 2);
     w.argmax_tmp = (int32_t *)take((size_t)c.tree_N * 4);
     w.status = (int32_t *)take(256);
+    w.am_keys = (unsigned long long *)take((size_t)d.Rlog * 8);
+    w.am_counter = (int32_t *)take(256);
+    const size_t trows = (size_t)c.max_batch * (c.block_B - 1) * topk_warps(c.vocab);
+    w.topk_cand = (unsigned long long *)take(trows * c.topk * 8);
+    w.topk_ml = (float *)take(trows * 2 * 4);
     w.total = off;
     return w;
 }
@@ -127,35 +139,75 @@ struct glance_ctx {
     std::vector<const bf16 *> ln1, wqkv, wo, ln2, wgu, wd;
     glance_head_weights head;
     int64_t launches;
-    // optional per-launch timing of the GEMM kernel
+    // optional per-launch timing (event pairs created when profiling is first enabled)
     bool profiling = false;
     std::vector<cudaEvent_t> ev;      // 2 per tallied launch
     std::vector<double> ev_bytes;
+    std::vector<int> ev_kind;
     size_t ev_used = 0;
+    // TMA descriptors, keyed by (base, inner extent, rows, box rows); built on first use by a host-only call
+    std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;
+    bool map_error = false;
 };
 
 namespace {
 
-#define LAUNCH(ctx, call) \
-    do {                  \
-        call;             \
-        (ctx)->launches++; \
-    } while (0)
+enum { KIND_GEMM = 0, KIND_ATTN = 1, KIND_NORM = 2, KIND_ROPE = 3, KIND_OTHER = 4, KIND_COUNT = 5 };
 
-constexpr size_t kMaxProfiled = 8192;
+constexpr size_t kMaxProfiled = 32768;
 
-// the weight-streaming GEMM, optionally bracketed by events
-void gemm(glance_ctx *ctx, const bf16 *W, const bf16 *X, float *Y, int Nout, int K, int R, int ldy, size_t split_stride,
-          int S) {
+inline bool prof_begin(glance_ctx *ctx) {
     const bool prof = ctx->profiling && ctx->ev_used < kMaxProfiled;
     if (prof) cudaEventRecord(ctx->ev[2 * ctx->ev_used], ctx->stream);
-    launch_gemm(W, X, Y, Nout, K, R, ldy, split_stride, S, ctx->stream);
+    return prof;
+}
+inline void prof_end(glance_ctx *ctx, bool prof, int kind, double bytes) {
     ctx->launches++;
-    if (prof) {
-        cudaEventRecord(ctx->ev[2 * ctx->ev_used + 1], ctx->stream);
-        ctx->ev_bytes[ctx->ev_used] = 2.0 * Nout * K + 2.0 * R * K + 4.0 * S * R * Nout;
-        ctx->ev_used++;
+    if (!prof) return;
+    cudaEventRecord(ctx->ev[2 * ctx->ev_used + 1], ctx->stream);
+    ctx->ev_bytes[ctx->ev_used] = bytes;
+    ctx->ev_kind[ctx->ev_used] = kind;
+    ctx->ev_used++;
+}
+
+#define LAUNCH(ctx, kind, call)                  \
+    do {                                         \
+        const bool prof_ = prof_begin(ctx);      \
+        call;                                    \
+        prof_end(ctx, prof_, kind, 0.0);         \
+    } while (0)
+
+const CUtensorMap *get_map(glance_ctx *ctx, const void *base, int inner, int rows, int box_rows) {
+    auto key = std::make_tuple(base, inner, rows, box_rows);
+    auto it = ctx->maps.find(key);
+    if (it != ctx->maps.end()) return &it->second;
+    CUtensorMap m;
+    if (!tc_make_map(&m, base, (uint64_t)inner, (uint64_t)rows, (uint32_t)box_rows)) {
+        ctx->map_error = true;
+        return nullptr;
     }
+    return &ctx->maps.emplace(key, m).first->second;
+}
+
+// The weight-streaming GEMM.  mode 0: fp32 split-K planes Y[s][r][f]; mode 1: SwiGLU into act (W = gate rows
+// then up rows, Nout = 2F); mode 2: arg-max over f into `argmax` (optional fp32 logits in Y).
+// x_rows = rows allocated behind X (rows of its tensor map).
+void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, int Nout, int K, int R, int S, float *Y,
+          int ldy, size_t split_stride, bf16 *act, int32_t *argmax) {
+    const CUtensorMap *mw = get_map(ctx, W, K, Nout, 128);
+    const CUtensorMap *mx = get_map(ctx, X, K, x_rows, tc_row_pad(R));
+    if (!mw || !mx) return;
+    TcGemmArgs a{};
+    a.Nout = Nout; a.K = K; a.R = R; a.S = mode == 0 ? S : 1; a.Y = Y; a.ldy = ldy; a.split_stride = split_stride;
+    a.act = act; a.F = Nout / 2; a.keys = ctx->ws.am_keys; a.argmax = argmax; a.counter = ctx->ws.am_counter;
+    a.status = ctx->ws.status;
+    const bool prof = prof_begin(ctx);
+    if (launch_gemm_tc(mode, a, *mw, *mx, ctx->stream) != cudaSuccess) ctx->map_error = true;
+    double bytes = 2.0 * Nout * K + 2.0 * R * K;
+    if (mode == 0) bytes += 4.0 * a.S * R * Nout;
+    else if (mode == 1) bytes += 2.0 * R * (Nout / 2);
+    else bytes += 4.0 * R + (Y ? 4.0 * R * Nout : 0.0);
+    prof_end(ctx, prof, KIND_GEMM, bytes);
 }
 
 struct LayerW {
@@ -201,34 +253,34 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     const KvGeom geom = geom_of(ctx, ps.seqs);
     const int32_t *page_table = ps.seqs->page_table + (size_t)ps.seq_off * c.max_pages_per_seq;
     const int32_t *seq_len = ps.seqs->seq_len + ps.seq_off;
-    // QKV projection, split-K planes
+    const int xr = d.Rmax;                             // rows allocated behind every activation buffer
+    // QKV projection (split-K planes), reduced by the rotary / K-V write kernel
     size_t ss = (size_t)ps.R * d.qkv_out;
-    gemm(ctx, w.wqkv, ws.xn, ws.part, d.qkv_out, c.hidden, ps.R, d.qkv_out, ss, d.S_qkv);
+    gemm(ctx, 0, w.wqkv, ws.xn, xr, d.qkv_out, c.hidden, ps.R, d.S_qkv, ws.part, d.qkv_out, ss, nullptr, nullptr);
     RopeKv rk;
     rk.R = ps.R; rk.Rq = ps.Rq; rk.Hq = c.n_q_heads; rk.Hkv = c.n_kv_heads; rk.d = c.head_dim;
     rk.part = ws.part; rk.S = d.S_qkv; rk.split_stride = ss; rk.ldy = d.qkv_out;
     rk.meta = meta_of(ctx); rk.q = ws.q; rk.pool_layer = pool_layer; rk.geom = geom; rk.page_table = page_table;
     rk.status = ws.status;
-    LAUNCH(ctx, launch_rope_kv(rk, st));
+    LAUNCH(ctx, KIND_ROPE, launch_rope_kv(rk, st));
     if (ps.Rq == 0) return;
     AttnParams ap;
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
     ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn; ap.S = d.S_att; ap.part_o = ws.att_o;
     ap.part_ml = ws.att_ml; ap.counters = ws.att_ctr; ap.status = ws.status;
-    LAUNCH(ctx, launch_attention(ap, st));
+    LAUNCH(ctx, KIND_ATTN, launch_attention(ap, st));
     const int R = ps.Rq;
-    // output projection + residual + norm
+    // output projection (split-K planes), reduced by residual + norm
     ss = (size_t)R * c.hidden;
-    gemm(ctx, w.wo, ws.attn, ws.part, c.hidden, d.qd, R, c.hidden, ss, d.S_o);
-    LAUNCH(ctx, launch_norm(ws.x, ws.part, d.S_o, ss, c.hidden, R, c.hidden, w.ln2, nullptr, R, c.rms_eps, ws.xn,
-                            nullptr, st));
-    // SwiGLU MLP
-    gemm(ctx, w.wgu, ws.xn, ws.part, 2 * c.ffn, c.hidden, R, 2 * c.ffn, 0, 1);
-    LAUNCH(ctx, launch_swiglu(ws.part, 2 * c.ffn, R, c.ffn, ws.act, st));
-    gemm(ctx, w.wd, ws.act, ws.part, c.hidden, c.ffn, R, c.hidden, ss, d.S_d);
-    LAUNCH(ctx, launch_norm(ws.x, ws.part, d.S_d, ss, c.hidden, R, c.hidden, next_gain, nullptr, R, c.rms_eps,
-                            ws.xn, hidden_out, st));
+    gemm(ctx, 0, w.wo, ws.attn, xr, c.hidden, d.qd, R, d.S_o, ws.part, c.hidden, ss, nullptr, nullptr);
+    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, ws.part, d.S_o, ss, c.hidden, R, c.hidden, w.ln2, nullptr, R, c.rms_eps,
+                                       ws.xn, nullptr, st));
+    // SwiGLU MLP: gate/up GEMM with the activation fused into its epilogue, then down projection
+    gemm(ctx, 1, w.wgu, ws.xn, xr, 2 * c.ffn, c.hidden, R, 1, nullptr, 0, 0, ws.act, nullptr);
+    gemm(ctx, 0, w.wd, ws.act, xr, c.hidden, c.ffn, R, d.S_d, ws.part, c.hidden, ss, nullptr, nullptr);
+    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, ws.part, d.S_d, ss, c.hidden, R, c.hidden, next_gain, nullptr, R,
+                                       c.rms_eps, ws.xn, hidden_out, st));
 }
 
 // all target layers + final norm (+ LM head and argmax) over rows already set up in ws.x
@@ -237,18 +289,16 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
     Workspace &ws = ctx->ws;
     cudaStream_t st = ctx->stream;
     const KvGeom geom = geom_of(ctx, ps.seqs);
-    LAUNCH(ctx, launch_norm(ws.x, nullptr, 0, 0, c.hidden, ps.R, c.hidden, ctx->ln1[0], nullptr, ps.R, c.rms_eps,
-                            ws.xn, nullptr, st));
+    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, nullptr, 0, 0, c.hidden, ps.R, c.hidden, ctx->ln1[0], nullptr, ps.R,
+                                       c.rms_eps, ws.xn, nullptr, st));
     for (int l = 0; l < c.n_layers; ++l) {
         LayerW w{ctx->ln2[l], ctx->wqkv[l], ctx->wo[l], ctx->wgu[l], ctx->wd[l]};
         const bool last = (l + 1 == c.n_layers);
         bf16 *pool_layer = (bf16 *)ps.seqs->kv_pool + (size_t)l * geom.layer_stride();
         run_layer(ctx, w, pool_layer, ps, last ? ctx->final_norm : ctx->ln1[l + 1], last ? hidden_out : nullptr);
     }
-    if (argmax) {
-        gemm(ctx, ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, ps.R, c.vocab, 0, 1);
-        LAUNCH(ctx, launch_argmax(logits, ps.R, c.vocab, argmax, st));
-    }
+    if (argmax)   // LM head with the arg-max fused into its epilogue; logits are stored only on request
+        gemm(ctx, 2, ctx->lm_head, ws.xn, ctx->dims.Rmax, c.vocab, c.hidden, ps.R, 1, logits, c.vocab, 0, nullptr, argmax);
 }
 
 int32_t check_seqs(const glance_ctx *ctx, const glance_seqs *s) {
@@ -259,7 +309,13 @@ int32_t check_seqs(const glance_ctx *ctx, const glance_seqs *s) {
     return GLANCE_OK;
 }
 
-int32_t finish(glance_ctx *ctx) { return cudaPeekAtLastError() == cudaSuccess ? GLANCE_OK : GLANCE_E_CUDA; }
+int32_t finish(glance_ctx *ctx) {
+    if (ctx->map_error) {
+        ctx->map_error = false;
+        return GLANCE_E_CUDA;
+    }
+    return cudaPeekAtLastError() == cudaSuccess ? GLANCE_OK : GLANCE_E_CUDA;
+}
 
 __global__ void set_seq_kernel(int32_t *seq_len, int32_t *root, int32_t len, int32_t r) {
     *seq_len = len;
@@ -329,7 +385,9 @@ int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, 
     if (cudaMemsetAsync(ws.att_ctr, 0, (size_t)cfg->max_batch * cfg->n_kv_heads * d.q_tiles_max * 4, ctx->stream) !=
             cudaSuccess ||
         cudaMemsetAsync(ws.walk_ctr, 0, (size_t)cfg->max_batch * 4, ctx->stream) != cudaSuccess ||
-        cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess) {
+        cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess ||
+        cudaMemsetAsync(ws.am_keys, 0, (size_t)d.Rlog * 8, ctx->stream) != cudaSuccess ||
+        cudaMemsetAsync(ws.am_counter, 0, 256, ctx->stream) != cudaSuccess) {
         delete ctx;
         return GLANCE_E_CUDA;
     }
@@ -364,9 +422,9 @@ int32_t glance_prefill(glance_ctx *ctx, const glance_seqs *seqs, int32_t seq, co
         vs.row_ids = ids ? ids + done : nullptr;
         vs.count = n; vs.chain_anc = ws.chain_anc; vs.embed = ctx->embed; vs.vocab = c.vocab;
         vs.capacity = c.max_pages_per_seq * kPage; vs.x = ws.x; vs.meta = meta_of(ctx); vs.status = ws.status;
-        LAUNCH(ctx, launch_setup_verify(vs, st));
+        LAUNCH(ctx, KIND_OTHER, launch_setup_verify(vs, st));
         PassInfo ps{N, N, 1, N, ws.chain_anc, seqs, seq};
-        run_target(ctx, ps, ws.hidden_tmp, ws.logits, last ? ws.argmax_tmp : nullptr);
+        run_target(ctx, ps, ws.hidden_tmp, nullptr, last ? ws.argmax_tmp : nullptr);
         // head context K/V of the new positions (Section 3.2: keys and values are the target's hidden states)
         DraftSetup ds;
         ds.batch = 1; ds.B = c.block_B; ds.FR = N; ds.H = c.hidden; ds.d = c.head_dim; ds.theta = c.rope_theta;
@@ -374,14 +432,14 @@ int32_t glance_prefill(glance_ctx *ctx, const glance_seqs *seqs, int32_t seq, co
         ds.count_const = n; ds.n_block = 0; ds.embed = ctx->embed; ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
         ds.vocab = c.vocab; ds.capacity = c.max_pages_per_seq * kPage; ds.x = ws.x; ds.meta = meta_of(ctx);
         ds.status = ws.status;
-        LAUNCH(ctx, launch_setup_draft(ds, st));
-        LAUNCH(ctx, launch_norm(ws.x, nullptr, 0, 0, c.hidden, N, c.hidden, (const bf16 *)ctx->head.ctx_norm, nullptr, N,
+        LAUNCH(ctx, KIND_OTHER, launch_setup_draft(ds, st));
+        LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, nullptr, 0, 0, c.hidden, N, c.hidden, (const bf16 *)ctx->head.ctx_norm, nullptr, N,
                                 c.rms_eps, ws.xn, nullptr, st));
         LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
                   (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
         PassInfo hp{N, 0, 1, N, nullptr, seqs, seq};
         run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, hp, nullptr, nullptr);
-        LAUNCH(ctx, launch_prefill_advance(seqs->seq_len + seq, seqs->root + seq, seqs->feat_count + seq,
+        LAUNCH(ctx, KIND_OTHER, launch_prefill_advance(seqs->seq_len + seq, seqs->root + seq, seqs->feat_count + seq,
                                            last ? ws.argmax_tmp : nullptr, n, st));
     }
     return finish(ctx);
@@ -392,7 +450,7 @@ int32_t glance_seq_truncate(glance_ctx *ctx, const glance_seqs *seqs, int32_t se
     if (rc) return rc;
     if (seq < 0 || seq >= seqs->batch || new_len < 0 || new_root < 0 || new_root >= ctx->cfg.vocab)
         return GLANCE_E_INVALID_ARG;
-    LAUNCH(ctx, (set_seq_kernel<<<1, 1, 0, ctx->stream>>>(seqs->seq_len + seq, seqs->root + seq, new_len, new_root)));
+    LAUNCH(ctx, KIND_OTHER, (set_seq_kernel<<<1, 1, 0, ctx->stream>>>(seqs->seq_len + seq, seqs->root + seq, new_len, new_root)));
     return finish(ctx);
 }
 
@@ -412,17 +470,22 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
     ds.feat_count = seqs->feat_count; ds.count_const = 0; ds.n_block = B; ds.embed = ctx->embed;
     ds.mask_embed = (const bf16 *)ctx->head.mask_embed; ds.vocab = c.vocab;
     ds.capacity = c.max_pages_per_seq * kPage; ds.x = ws.x; ds.meta = meta_of(ctx); ds.status = ws.status;
-    LAUNCH(ctx, launch_setup_draft(ds, st));
+    LAUNCH(ctx, KIND_OTHER, launch_setup_draft(ds, st));
     // block rows use the head's input norm, feature rows the context norm
-    LAUNCH(ctx, launch_norm(ws.x, nullptr, 0, 0, c.hidden, R, c.hidden, (const bf16 *)ctx->head.ln1,
+    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, nullptr, 0, 0, c.hidden, R, c.hidden, (const bf16 *)ctx->head.ln1,
                             (const bf16 *)ctx->head.ctx_norm, R1, c.rms_eps, ws.xn, nullptr, st));
     LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
               (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
     PassInfo ps{R, R1, batch, B, nullptr, seqs, 0};
     run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, ps, (const bf16 *)ctx->head.final_norm, nullptr);
     float *logits = logits_dbg ? logits_dbg : ws.logits;
-    gemm(ctx, ctx->lm_head, ws.xn, logits, c.vocab, c.hidden, R1, c.vocab, 0, 1);
-    LAUNCH(ctx, launch_topk(logits, batch, B, c.vocab, c.topk, topk_ids, topk_lp, st));
+    gemm(ctx, 0, ctx->lm_head, ws.xn, ctx->dims.Rmax, c.vocab, c.hidden, R1, 1, logits, c.vocab, 0, nullptr, nullptr);
+    {
+        const bool prof = prof_begin(ctx);
+        launch_topk(logits, batch, B, c.vocab, c.topk, topk_ids, topk_lp, ws.topk_cand, ws.topk_ml, st);
+        ctx->launches++;                              // two kernels
+        prof_end(ctx, prof, KIND_OTHER, 0.0);
+    }
     return finish(ctx);
 }
 
@@ -433,7 +496,7 @@ int32_t glance_build_tree(glance_ctx *ctx, int32_t batch, const int32_t *root, c
     if (!out->token || !out->parent || !out->depth || !out->rank || !out->score || !out->anc || !out->n_nodes)
         return GLANCE_E_INVALID_ARG;
     const glance_config &c = ctx->cfg;
-    LAUNCH(ctx, launch_build_tree(batch, c.tree_N, c.block_B - 1, c.topk, root, topk_ids, topk_lp, *out, ctx->stream));
+    LAUNCH(ctx, KIND_OTHER, launch_build_tree(batch, c.tree_N, c.block_B - 1, c.topk, root, topk_ids, topk_lp, *out, ctx->stream));
     return finish(ctx);
 }
 
@@ -450,9 +513,9 @@ int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glanc
     vs.seq_len = seqs->seq_len; vs.token = tree->token; vs.depth = tree->depth; vs.row_embeds = nullptr;
     vs.row_ids = nullptr; vs.count = 0; vs.chain_anc = nullptr; vs.embed = ctx->embed; vs.vocab = c.vocab;
     vs.capacity = c.max_pages_per_seq * kPage; vs.x = ws.x; vs.meta = meta_of(ctx); vs.status = ws.status;
-    LAUNCH(ctx, launch_setup_verify(vs, ctx->stream));
+    LAUNCH(ctx, KIND_OTHER, launch_setup_verify(vs, ctx->stream));
     PassInfo ps{batch * N, batch * N, batch, N, tree->anc, seqs, 0};
-    run_target(ctx, ps, (bf16 *)hidden, logits_dbg ? logits_dbg : ws.logits, argmax);
+    run_target(ctx, ps, (bf16 *)hidden, logits_dbg, argmax);
     return finish(ctx);
 }
 
@@ -463,7 +526,7 @@ static int32_t commit_common(glance_ctx *ctx, const glance_seqs *seqs, WalkCommi
     wc.page_table = seqs->page_table; wc.seq_len = seqs->seq_len; wc.root = seqs->root;
     wc.feat_count = seqs->feat_count; wc.feat = (bf16 *)seqs->feat; wc.counters = ctx->ws.walk_ctr;
     wc.status = ctx->ws.status;
-    LAUNCH(ctx, launch_walk_commit(wc, ctx->stream));
+    LAUNCH(ctx, KIND_OTHER, launch_walk_commit(wc, ctx->stream));
     return finish(ctx);
 }
 
@@ -514,15 +577,17 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
     ap.out = (bf16 *)out; ap.S = ctx->dims.S_att; ap.part_o = ctx->ws.att_o; ap.part_ml = ctx->ws.att_ml;
     ap.counters = ctx->ws.att_ctr; ap.status = ctx->ws.status;
-    LAUNCH(ctx, launch_attention(ap, ctx->stream));
+    LAUNCH(ctx, KIND_ATTN, launch_attention(ap, ctx->stream));
     return finish(ctx);
 }
 
-int32_t glance_debug_gemm(glance_ctx *ctx, const void *W, const void *X, float *Y, int32_t Nout, int32_t K,
-                          int32_t R, int32_t S) {
-    if (!ctx || !W || !X || !Y) return GLANCE_E_INVALID_ARG;
-    if (Nout < 1 || K < 64 || K % 64 || R < 1 || R > 128 || S < 1 || S > 16) return GLANCE_E_INVALID_ARG;
-    gemm(ctx, (const bf16 *)W, (const bf16 *)X, Y, Nout, K, R, Nout, (size_t)R * Nout, S);
+int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const void *X, float *Y, void *act,
+                             int32_t *argmax, int32_t Nout, int32_t K, int32_t R, int32_t S) {
+    if (!ctx || !W || !X || mode < 0 || mode > 2) return GLANCE_E_INVALID_ARG;
+    if (Nout < 1 || K < 64 || K % 64 || R < 1 || R > ctx->dims.Rlog || S < 1 || S > 16) return GLANCE_E_INVALID_ARG;
+    if ((mode == 0 && !Y) || (mode == 1 && (!act || Nout % 2)) || (mode == 2 && !argmax)) return GLANCE_E_INVALID_ARG;
+    gemm(ctx, mode, (const bf16 *)W, (const bf16 *)X, R, Nout, K, R, S, Y, Nout, (size_t)R * Nout, (bf16 *)act, argmax);
+    ctx->maps.clear();          // the hook's operands are transient: do not keep their descriptors
     return finish(ctx);
 }
 
@@ -531,6 +596,7 @@ int32_t glance_profile_enable(glance_ctx *ctx, int32_t on) {
     if (on && ctx->ev.empty()) {
         ctx->ev.resize(2 * kMaxProfiled);
         ctx->ev_bytes.resize(kMaxProfiled);
+        ctx->ev_kind.resize(kMaxProfiled);
         for (auto &e : ctx->ev)
             if (cudaEventCreate(&e) != cudaSuccess) return GLANCE_E_CUDA;
     }
@@ -538,19 +604,18 @@ int32_t glance_profile_enable(glance_ctx *ctx, int32_t on) {
     return GLANCE_OK;
 }
 
-int32_t glance_profile_read(glance_ctx *ctx, double *gemm_ms, double *gemm_bytes, int64_t *gemm_launches) {
-    if (!ctx || !gemm_ms || !gemm_bytes || !gemm_launches) return GLANCE_E_INVALID_ARG;
+int32_t glance_profile_read(glance_ctx *ctx, double *ms, double *bytes, int64_t *launches) {
+    if (!ctx || !ms || !bytes || !launches) return GLANCE_E_INVALID_ARG;
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return GLANCE_E_CUDA;
-    double ms = 0.0, bytes = 0.0;
+    for (int k = 0; k < KIND_COUNT; ++k) { ms[k] = 0.0; bytes[k] = 0.0; launches[k] = 0; }
     for (size_t i = 0; i < ctx->ev_used; ++i) {
         float t = 0.f;
         if (cudaEventElapsedTime(&t, ctx->ev[2 * i], ctx->ev[2 * i + 1]) != cudaSuccess) return GLANCE_E_CUDA;
-        ms += t;
-        bytes += ctx->ev_bytes[i];
+        const int k = ctx->ev_kind[i];
+        ms[k] += t;
+        bytes[k] += ctx->ev_bytes[i];
+        launches[k]++;
     }
-    *gemm_ms = ms;
-    *gemm_bytes = bytes;
-    *gemm_launches = (int64_t)ctx->ev_used;
     ctx->ev_used = 0;
     return GLANCE_OK;
 }

@@ -66,10 +66,11 @@ struct RopeKv {
 };
 void launch_rope_kv(const RopeKv &p, cudaStream_t st);
 
-void launch_swiglu(const float *part, int ldp, int R, int F, bf16 *act, cudaStream_t st);
-void launch_argmax(const float *logits, int R, int V, int32_t *out, cudaStream_t st);
-// rows (s, j), j = 1..L of logits [batch*B][V] -> ids/lp [batch][L][k]
-void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *ids, float *lp, cudaStream_t st);
+// rows (s, j), j = 1..L of logits [batch*B][V] -> ids/lp [batch][L][k]; scratch: cand [rows][topk_warps(V)][k],
+// ml [rows][topk_warps(V)][2].  Two launches.
+int topk_warps(int V);
+void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *ids, float *lp,
+                 unsigned long long *cand, float *ml, cudaStream_t st);
 
 // ---- tree + walk (tree_walk.cu) -----------------------------------------------------------
 void launch_build_tree(int batch, int N, int L, int k, const int32_t *root, const int32_t *ids, const float *lp,
@@ -115,11 +116,5 @@ struct AttnParams {
 };
 void launch_attention(const AttnParams &p, cudaStream_t st);
 int attention_q_tiles(int T, int G);
-
-// ---- weight-streaming GEMM (gemm_mma.cu) --------------------------------------------------
-// Y[s][r][f] = sum over the K range of split s of X[r][k] * W[f][k];  X bf16 [R][K], W bf16 [Nout][K],
-// Y fp32 [S][.][ldy] with split stride `split_stride` elements.  K must be a multiple of 64.
-void launch_gemm(const bf16 *W, const bf16 *X, float *Y, int Nout, int K, int R, int ldy, size_t split_stride,
-                 int S, cudaStream_t st);
 
 }  // namespace glance

@@ -125,121 +125,122 @@ void launch_setup_draft(const DraftSetup &p, cudaStream_t st) {
 // ------------------------------------------------------------------------------------------
 // residual add (split-K partials, fixed order) + RMSNorm -> bf16
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) norm_kernel(float *x, const float *part, int S, size_t split_stride, int ldp,
-                                                   int H, const bf16 *gain_a, const bf16 *gain_b, int split_row,
-                                                   float eps, bf16 *xn, bf16 *hidden_out) {
-    extern __shared__ float row[];
-    __shared__ float red[8];
+__global__ void __launch_bounds__(1024) norm_kernel(float *x, const float *part, int S, size_t split_stride, int ldp,
+                                                    int H, const bf16 *gain_a, const bf16 *gain_b, int split_row,
+                                                    float eps, bf16 *xn, bf16 *hidden_out) {
+    extern __shared__ float4 row4[];
+    __shared__ float red[32];
     const int r = blockIdx.x;
-    float *xr = x + (size_t)r * H;
+    const int H4 = H >> 2;
+    float4 *xr = reinterpret_cast<float4 *>(x + (size_t)r * H);
     float ss = 0.f;
-    for (int c = threadIdx.x; c < H; c += blockDim.x) {
-        float v = xr[c];
-        for (int s = 0; s < S; ++s) v += part[s * split_stride + (size_t)r * ldp + c];
-        row[c] = v;
-        ss += v * v;
+    for (int c = threadIdx.x; c < H4; c += blockDim.x) {
+        float4 v = xr[c];
+        for (int s = 0; s < S; ++s) {
+            const float4 p = __ldcg(reinterpret_cast<const float4 *>(part + s * split_stride + (size_t)r * ldp) + c);
+            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+        }
+        row4[c] = v;
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         if (S > 0) xr[c] = v;
-        if (hidden_out) hidden_out[(size_t)r * H + c] = __float2bfloat16(v);
+        if (hidden_out) {
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+            uint2 o;
+            o.x = *reinterpret_cast<uint32_t *>(&lo);
+            o.y = *reinterpret_cast<uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(hidden_out + (size_t)r * H)[c] = o;
+        }
     }
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
+    const int nw = (blockDim.x + 31) >> 5;
+    for (int w = 0; w < nw; ++w) tot += red[w];
     const float inv = rsqrtf(tot / (float)H + eps);
     const bf16 *g = (r >= split_row) ? gain_b : gain_a;
     if (xn)
-        for (int c = threadIdx.x; c < H; c += blockDim.x)
-            xn[(size_t)r * H + c] = __float2bfloat16(row[c] * inv * __bfloat162float(g[c]));
+        for (int c = threadIdx.x; c < H4; c += blockDim.x) {
+            const float4 v = row4[c];
+            const uint2 gg = reinterpret_cast<const uint2 *>(g)[c];
+            const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x);
+            const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
+            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv * __low2float(g01), v.y * inv * __high2float(g01));
+            __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv * __low2float(g23), v.w * inv * __high2float(g23));
+            uint2 o;
+            o.x = *reinterpret_cast<uint32_t *>(&lo);
+            o.y = *reinterpret_cast<uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(xn + (size_t)r * H)[c] = o;
+        }
 }
 
 void launch_norm(float *x, const float *part, int S, size_t part_split_stride, int ldp, int R, int H,
                  const bf16 *gain_a, const bf16 *gain_b, int split_row, float eps, bf16 *xn, bf16 *hidden_out,
                  cudaStream_t st) {
-    norm_kernel<<<R, 256, H * sizeof(float), st>>>(x, part, S, part_split_stride, ldp, H, gain_a,
-                                                   gain_b ? gain_b : gain_a, split_row, eps, xn, hidden_out);
+    int threads = ((H / 4) + 31) / 32 * 32;
+    threads = threads > 1024 ? 1024 : threads;
+    norm_kernel<<<R, threads, H * sizeof(float), st>>>(x, part, S, part_split_stride, ldp, H, gain_a,
+                                                       gain_b ? gain_b : gain_a, split_row, eps, xn, hidden_out);
 }
 
 // ------------------------------------------------------------------------------------------
 // QKV split-K reduction + rotary (pairs (i, i + d/2)) + paged K/V write
 // ------------------------------------------------------------------------------------------
 __global__ void rope_kv_kernel(RopeKv p) {
-    const int r = blockIdx.x;
+    // grid (R, Hq + 2 Hkv): one block per (row, head); heads are ordered q..., k..., v...
+    const int r = blockIdx.x, h = blockIdx.y;
     const int half = p.d >> 1;
+    const bool is_q = h < p.Hq, is_k = !is_q && h < p.Hq + p.Hkv;
+    if (is_q && r >= p.Rq) return;
     const int slot_pos = p.meta.kvslot[r];
-    const int s = p.meta.seq[r];
-    const float *cs = p.meta.rope_cos + (size_t)r * half;
-    const float *sn = p.meta.rope_sin + (size_t)r * half;
-    const int n_rot = (p.Hq + p.Hkv) * half;       // rotated pairs (q heads then k heads)
-    const int n_v = p.Hkv * p.d;
-    bf16 *krow = nullptr, *vrow = nullptr;
-    if (slot_pos >= 0) {
+    bf16 *dst = nullptr;
+    if (is_q) {
+        dst = p.q + ((size_t)r * p.Hq + h) * p.d;
+    } else {
+        if (slot_pos < 0) return;
+        const int s = p.meta.seq[r];
         const int pg = slot_pos / kPage;
         bool ok = pg < p.geom.max_pages_per_seq;
         int page = ok ? p.page_table[(size_t)s * p.geom.max_pages_per_seq + pg] : 0;
         if (page < 0 || page >= p.geom.n_pages) ok = false;
-        if (ok) {
-            krow = p.pool_layer + p.geom.row(page, 0, 0, slot_pos % kPage);
-            vrow = p.pool_layer + p.geom.row(page, 1, 0, slot_pos % kPage);
-        } else if (threadIdx.x == 0) {
-            set_status(p.status, GLANCE_E_BOUNDS);
+        if (!ok) {
+            if (threadIdx.x == 0) set_status(p.status, GLANCE_E_BOUNDS);
+            return;
         }
+        const int kvh = is_k ? h - p.Hq : h - p.Hq - p.Hkv;
+        dst = p.pool_layer + p.geom.row(page, is_k ? 0 : 1, kvh, slot_pos % kPage);
     }
-    const size_t head_stride = (size_t)kPage * p.d;    // distance between kv heads of one (page, kv)
-    for (int e = threadIdx.x; e < n_rot + n_v; e += blockDim.x) {
-        if (e < n_rot) {
-            const int h = e / half, i = e % half;
-            if (h < p.Hq && r >= p.Rq) continue;
-            const int col = h * p.d + i;
+    const int col0 = h * p.d;
+    const float *y = p.part + (size_t)r * p.ldy + col0;
+    if (is_q || is_k) {
+        const float *cs = p.meta.rope_cos + (size_t)r * half;
+        const float *sn = p.meta.rope_sin + (size_t)r * half;
+        for (int i = threadIdx.x; i < half; i += blockDim.x) {
             float a = 0.f, b = 0.f;
             for (int sp = 0; sp < p.S; ++sp) {
-                const float *y = p.part + sp * p.split_stride + (size_t)r * p.ldy;
-                a += y[col];
-                b += y[col + half];
+                a += __ldcg(y + sp * p.split_stride + i);
+                b += __ldcg(y + sp * p.split_stride + i + half);
             }
             const float c = cs[i], sv = sn[i];
-            const float ra = a * c - b * sv, rb = b * c + a * sv;
-            if (h < p.Hq) {
-                bf16 *q = p.q + (size_t)r * p.Hq * p.d + col;
-                q[0] = __float2bfloat16(ra);
-                q[half] = __float2bfloat16(rb);
-            } else if (krow) {
-                bf16 *k = krow + (size_t)(h - p.Hq) * head_stride + i;
-                k[0] = __float2bfloat16(ra);
-                k[half] = __float2bfloat16(rb);
-            }
-        } else if (vrow) {
-            const int ev = e - n_rot;
-            const int h = ev / p.d, i = ev % p.d;
-            const int col = (p.Hq + p.Hkv) * p.d + ev;
+            dst[i] = __float2bfloat16(a * c - b * sv);
+            dst[i + half] = __float2bfloat16(b * c + a * sv);
+        }
+    } else {
+        for (int i = threadIdx.x; i < p.d; i += blockDim.x) {
             float a = 0.f;
-            for (int sp = 0; sp < p.S; ++sp) a += p.part[sp * p.split_stride + (size_t)r * p.ldy + col];
-            vrow[(size_t)h * head_stride + i] = __float2bfloat16(a);
+            for (int sp = 0; sp < p.S; ++sp) a += __ldcg(y + sp * p.split_stride + i);
+            dst[i] = __float2bfloat16(a);
         }
     }
 }
 
-void launch_rope_kv(const RopeKv &p, cudaStream_t st) { rope_kv_kernel<<<p.R, 256, 0, st>>>(p); }
-
-// ------------------------------------------------------------------------------------------
-// SwiGLU: act = silu(gate) * up
-// ------------------------------------------------------------------------------------------
-__global__ void swiglu_kernel(const float *part, int ldp, int F, bf16 *act) {
-    const int r = blockIdx.y;
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= F) return;
-    const float g = part[(size_t)r * ldp + c], u = part[(size_t)r * ldp + F + c];
-    act[(size_t)r * F + c] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
-}
-
-void launch_swiglu(const float *part, int ldp, int R, int F, bf16 *act, cudaStream_t st) {
-    dim3 grid((F + 255) / 256, R);
-    swiglu_kernel<<<grid, 256, 0, st>>>(part, ldp, F, act);
+void launch_rope_kv(const RopeKv &p, cudaStream_t st) {
+    dim3 grid(p.R, p.Hq + 2 * p.Hkv);
+    rope_kv_kernel<<<grid, 64, 0, st>>>(p);
 }
 
 // ------------------------------------------------------------------------------------------
-// argmax over the vocabulary (value desc, id asc) on fp32 logits
+// block-wide max of packed (value desc, id asc) keys
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long *sh) {
     v = warp_max_u64(v);
@@ -252,69 +253,108 @@ __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v
     return r;
 }
 
-__global__ void __launch_bounds__(512) argmax_kernel(const float *logits, int V, int32_t *out) {
-    __shared__ unsigned long long sh[16];
-    const float *row = logits + (size_t)blockIdx.x * V;
-    unsigned long long best = 0;
-    for (int c = threadIdx.x; c < V; c += blockDim.x) {
-        unsigned long long k = pack_val_id(row[c], c);
-        best = k > best ? k : best;
+// ------------------------------------------------------------------------------------------
+// per-offset top-k and log-softmax (Assumption 1: marginals q_j over the full vocabulary), two stages.
+// Stage 1: every warp owns 1024 consecutive vocabulary entries held in registers and emits its k best
+// packed (value, id) keys plus its max and sum of exponentials.  Stage 2: one block per (sequence,
+// offset) merges the warps' candidates with k rounds of a block-wide max and combines the partial
+// log-sum-exp terms in a fixed order.  Keys are unique, so the result does not depend on timing.
+// ------------------------------------------------------------------------------------------
+constexpr int kTopkWarpSpan = 1024;
+
+__global__ void __launch_bounds__(128) topk_stage1_kernel(const float *logits, int B, int V, int k, int n_warps,
+                                                          unsigned long long *cand, float *ml) {
+    const int L = B - 1;
+    const int row = blockIdx.y;                         // (s, j-1)
+    const int s = row / L, j = row % L + 1;
+    const int gw = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (gw >= n_warps) return;
+    const float *src = logits + ((size_t)s * B + j) * V;
+    const int base = gw * kTopkWarpSpan;
+    unsigned long long key[32];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const int c = base + i * 32 + lane;
+        const float v = c < V ? src[c] : -INFINITY;
+        key[i] = c < V ? pack_val_id(v, c) : 0ull;
+        m = fmaxf(m, v);
     }
-    best = block_max_u64(best, sh);
-    if (threadIdx.x == 0) out[blockIdx.x] = unpack_id(best);
+    m = warp_max(m);
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const int c = base + i * 32 + lane;
+        if (c < V) sum += expf(unpack_val(key[i]) - m);
+    }
+    sum = warp_sum(sum);
+    if (lane == 0) {
+        ml[((size_t)row * n_warps + gw) * 2] = m;
+        ml[((size_t)row * n_warps + gw) * 2 + 1] = sum;
+    }
+    unsigned long long prev = ~0ull;
+    for (int t = 0; t < k; ++t) {
+        unsigned long long best = 0ull;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (key[i] < prev && key[i] > best) best = key[i];
+        best = warp_max_u64(best);
+        if (lane == 0) cand[((size_t)row * n_warps + gw) * k + t] = best;
+        prev = best;
+    }
 }
 
-void launch_argmax(const float *logits, int R, int V, int32_t *out, cudaStream_t st) {
-    argmax_kernel<<<R, 512, 0, st>>>(logits, V, out);
-}
-
-// ------------------------------------------------------------------------------------------
-// per-offset top-k and log-softmax (Assumption 1: marginals q_j over the full vocabulary)
-// ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(512) topk_kernel(const float *logits, int B, int V, int k, int32_t *ids, float *lp) {
+__global__ void __launch_bounds__(256) topk_stage2_kernel(int k, int n_warps, const unsigned long long *cand,
+                                                          const float *ml, int32_t *ids, float *lp) {
     __shared__ unsigned long long sh[16];
     __shared__ float shf[16];
-    const int L = B - 1;
-    const int s = blockIdx.x / L, j = blockIdx.x % L + 1;
-    const float *row = logits + ((size_t)s * B + j) * V;
-    // max
-    float m = -INFINITY;
-    for (int c = threadIdx.x; c < V; c += blockDim.x) m = fmaxf(m, row[c]);
-    m = warp_max(m);
-    if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = m;
+    const int row = blockIdx.x;
+    const float *rml = ml + (size_t)row * n_warps * 2;
+    float M = -INFINITY;
+    for (int w = threadIdx.x; w < n_warps; w += blockDim.x) M = fmaxf(M, rml[2 * w]);
+    M = warp_max(M);
+    if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = M;
     __syncthreads();
-    m = shf[0];
-    for (int w = 1; w < (blockDim.x >> 5); ++w) m = fmaxf(m, shf[w]);
+    M = shf[0];
+    for (int w = 1; w < 8; ++w) M = fmaxf(M, shf[w]);
     __syncthreads();
-    // sum exp
+    // fixed-order sum: thread t adds warps t, t+256, ...; partial sums are then added in warp/lane order
     float sum = 0.f;
-    for (int c = threadIdx.x; c < V; c += blockDim.x) sum += expf(row[c] - m);
+    for (int w = threadIdx.x; w < n_warps; w += blockDim.x) sum += rml[2 * w + 1] * expf(rml[2 * w] - M);
     sum = warp_sum(sum);
     if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = sum;
     __syncthreads();
     sum = 0.f;
-    for (int w = 0; w < (blockDim.x >> 5); ++w) sum += shf[w];
-    const float lse = m + logf(sum);
-    // k rounds of "largest key strictly below the previous winner"
+    for (int w = 0; w < 8; ++w) sum += shf[w];
+    const float lse = M + logf(sum);
+    const unsigned long long *rc = cand + (size_t)row * n_warps * k;
+    const int n = n_warps * k;
     unsigned long long prev = ~0ull;
     for (int t = 0; t < k; ++t) {
-        unsigned long long best = 0;
-        for (int c = threadIdx.x; c < V; c += blockDim.x) {
-            unsigned long long key = pack_val_id(row[c], c);
+        unsigned long long best = 0ull;
+        for (int c = threadIdx.x; c < n; c += blockDim.x) {
+            const unsigned long long key = rc[c];
             if (key < prev && key > best) best = key;
         }
         best = block_max_u64(best, sh);
         if (threadIdx.x == 0) {
-            ids[((size_t)s * L + (j - 1)) * k + t] = unpack_id(best);
-            lp[((size_t)s * L + (j - 1)) * k + t] = unpack_val(best) - lse;
+            ids[(size_t)row * k + t] = unpack_id(best);
+            lp[(size_t)row * k + t] = unpack_val(best) - lse;
         }
         prev = best;
     }
 }
 
-void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *ids, float *lp, cudaStream_t st) {
+int topk_warps(int V) { return (V + kTopkWarpSpan - 1) / kTopkWarpSpan; }
+
+void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *ids, float *lp,
+                 unsigned long long *cand, float *ml, cudaStream_t st) {
     if (B < 2) return;
-    topk_kernel<<<batch * (B - 1), 512, 0, st>>>(logits, B, V, k, ids, lp);
+    const int rows = batch * (B - 1), nw = topk_warps(V);
+    dim3 g1((nw + 3) / 4, rows);
+    topk_stage1_kernel<<<g1, 128, 0, st>>>(logits, B, V, k, nw, cand, ml);
+    topk_stage2_kernel<<<rows, 256, 0, st>>>(k, nw, cand, ml, ids, lp);
 }
 
 __global__ void prefill_advance_kernel(int32_t *seq_len, int32_t *root, int32_t *feat_count, const int32_t *argmax,

@@ -33,24 +33,68 @@ def make_engine(cfg, batch=1, max_len=None):
 
 # ------------------------------------------------------------------ GEMM alone
 
-@pytest.mark.parametrize("Nout,K,R,S", [(256, 256, 8, 1), (512, 256, 64, 2), (1408, 256, 16, 1), (1000, 704, 37, 3),
-                                        (4608, 3584, 64, 5), (3584, 18944, 64, 6), (640, 1024, 128, 4), (130, 64, 1, 1)])
-def test_gemm_matches_matmul(tiny_run, Nout, K, R, S):
-    eng = tiny_run.eng
+@pytest.fixture(scope="module")
+def gemm_eng(harness):
+    return make_engine(synth.CONFIGS["tiny"].replace(tree_N=128, vocab=256), batch=2)
+
+
+TC_SHAPES = [(256, 256, 8, 1), (512, 256, 64, 2), (1408, 256, 16, 1), (1000, 704, 37, 3), (4608, 3584, 64, 4),
+             (3584, 18944, 64, 5), (640, 1024, 128, 4), (130, 64, 1, 1), (384, 512, 200, 2), (37888, 3584, 64, 1)]
+
+
+@pytest.mark.parametrize("Nout,K,R,S", TC_SHAPES)
+def test_gemm_tc_planes(gemm_eng, Nout, K, R, S):
+    """Weight-streaming GEMM, fp32 split-K planes, against an fp64 matmul of the same bf16 inputs."""
+    eng = gemm_eng
     g = torch.Generator(device="cuda").manual_seed(Nout + K + R)
     W = (torch.randn(Nout, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
     X = torch.randn(R, K, generator=g, device="cuda").to(torch.bfloat16)
     Y = torch.full((S, R, Nout), float("nan"), device="cuda")
-    eng.glance_debug_gemm(W, X, Y, S)
-    eng.check_device_status()
-    ref = X.double().cpu() @ W.double().cpu().T
-    got = Y.double().sum(0).cpu()
-    scale = float(ref.abs().max())
-    assert float((got - ref).abs().max()) <= 1e-4 * scale + 1e-5
-    # run-to-run bit reproducibility
+    eng.glance_debug_gemm(0, W, X, Y=Y, S=S)
+    assert eng.glance_poll_status() == 0
+    ref = X.double() @ W.double().T
+    got = Y.double().sum(0)
+    assert float((got - ref).abs().max()) <= 1e-4 * float(ref.abs().max()) + 1e-5
     Y2 = torch.zeros_like(Y)
-    eng.glance_debug_gemm(W, X, Y2, S)
+    eng.glance_debug_gemm(0, W, X, Y=Y2, S=S)
     assert torch.equal(Y, Y2)
+
+
+@pytest.mark.parametrize("F,K,R", [(704, 256, 8), (2816, 1024, 32), (18944, 3584, 64), (320, 128, 130)])
+def test_gemm_tc_swiglu(gemm_eng, F, K, R):
+    eng = gemm_eng
+    g = torch.Generator(device="cuda").manual_seed(F + K + R)
+    W = (torch.randn(2 * F, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    X = torch.randn(R, K, generator=g, device="cuda").to(torch.bfloat16)
+    act = torch.full((R, F), float("nan"), dtype=torch.bfloat16, device="cuda")
+    eng.glance_debug_gemm(1, W, X, act=act)
+    assert eng.glance_poll_status() == 0
+    gu = X.double() @ W.double().T
+    ref = torch.nn.functional.silu(gu[:, :F]) * gu[:, F:]
+    assert float((act.double() - ref).abs().max()) <= 1e-2 * float(ref.abs().max())
+
+
+@pytest.mark.parametrize("V,K,R", [(1024, 256, 8), (32000, 1024, 32), (152064, 3584, 64), (1000, 128, 129)])
+def test_gemm_tc_argmax(gemm_eng, V, K, R):
+    eng = gemm_eng
+    g = torch.Generator(device="cuda").manual_seed(V + K + R)
+    W = (torch.randn(V, K, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    X = torch.randn(R, K, generator=g, device="cuda").to(torch.bfloat16)
+    W[7] = W[V - 3]                                       # an exact tie between two ids: the lower one must win
+    X[0] = W[7] * 4
+    am = torch.full((R,), -1, dtype=torch.int32, device="cuda")
+    Y = torch.full((R, V), float("nan"), device="cuda")
+    for rep in range(2):                                  # second call checks that keys and counter were re-armed
+        eng.glance_debug_gemm(2, W, X, Y=Y, argmax=am)
+        assert eng.glance_poll_status() == 0
+        ref = X.double() @ W.double().T
+        assert float((Y.double() - ref).abs().max()) <= 1e-4 * float(ref.abs().max()) + 1e-5
+        # the arg-max is taken on the kernel's own fp32 accumulators, ties to the lowest id
+        assert np.array_equal(am.cpu().numpy(), O.argmax_lowest(Y.cpu()))
+        assert int(am[0]) == 7
+    am2 = torch.full((R,), -1, dtype=torch.int32, device="cuda")
+    eng.glance_debug_gemm(2, W, X, argmax=am2)          # without the debug logits
+    assert torch.equal(am, am2)
 
 
 # ------------------------------------------------------------------ attention alone
