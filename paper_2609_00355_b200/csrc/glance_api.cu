@@ -67,8 +67,10 @@ Dims make_dims(const glance_config &c) {
     d.S_d = choose_split(c.hidden, c.ffn);
     const int G = c.n_q_heads / c.n_kv_heads;
     d.q_tiles_max = attention_q_tiles(std::max(c.tree_N, c.block_B), G);
-    int ctas = attention_q_tiles(c.tree_N, G) * c.n_kv_heads * c.max_batch;
-    d.S_att = std::max(1, std::min(8, 148 / ctas));
+    // attention split partials: the largest (q tiles x key splits) over every row count a pass can have
+    d.S_att = 0;
+    for (int T = 1; T <= std::max(c.tree_N, c.block_B); ++T)
+        d.S_att = std::max(d.S_att, attention_q_tiles(T, G) * attention_splits(T, G, c.n_kv_heads, c.max_batch));
     d.W = (c.tree_N + 63) / 64;
     return d;
 }
@@ -92,9 +94,9 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.attn = (bf16 *)take(R * d.qd * 2);
     w.act = (bf16 *)take(R * (size_t)c.ffn * 2);
     w.logits = (float *)take((size_t)d.Rlog * c.vocab * 4);
-    const size_t att_rows = (size_t)c.max_batch * c.n_kv_heads * d.q_tiles_max * 64;
-    w.att_o = (float *)take(att_rows * d.S_att * c.head_dim * 4);
-    w.att_ml = (float *)take(att_rows * d.S_att * 2 * 4);
+    const size_t att_rows = (size_t)c.max_batch * c.n_kv_heads * 64 * d.S_att;   // d.S_att = max q tiles x splits
+    w.att_o = (float *)take(att_rows * c.head_dim * 4);
+    w.att_ml = (float *)take(att_rows * 2 * 4);
     w.att_ctr = (int32_t *)take((size_t)c.max_batch * c.n_kv_heads * d.q_tiles_max * 4);
     w.walk_ctr = (int32_t *)take((size_t)c.max_batch * 4);
     w.row_seq = (int32_t *)take(R * 4);
@@ -267,7 +269,8 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     AttnParams ap;
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
-    ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn; ap.S = d.S_att; ap.part_o = ws.att_o;
+    ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn;
+    ap.S = attention_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch); ap.part_o = ws.att_o;
     ap.part_ml = ws.att_ml; ap.counters = ws.att_ctr; ap.status = ws.status;
     LAUNCH(ctx, KIND_ATTN, launch_attention(ap, st));
     const int R = ps.Rq;
@@ -575,7 +578,8 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     ap.batch = seqs->batch; ap.T = T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = (const bf16 *)q; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
-    ap.out = (bf16 *)out; ap.S = ctx->dims.S_att; ap.part_o = ctx->ws.att_o; ap.part_ml = ctx->ws.att_ml;
+    ap.out = (bf16 *)out; ap.S = attention_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch);
+    ap.part_o = ctx->ws.att_o; ap.part_ml = ctx->ws.att_ml;
     ap.counters = ctx->ws.att_ctr; ap.status = ctx->ws.status;
     LAUNCH(ctx, KIND_ATTN, launch_attention(ap, ctx->stream));
     return finish(ctx);

@@ -116,5 +116,6 @@ struct AttnParams {
 };
 void launch_attention(const AttnParams &p, cudaStream_t st);
 int attention_q_tiles(int T, int G);
+int attention_splits(int T, int G, int Hkv, int batch);   // key splits so that one wave of CTAs covers the SMs
 
 }  // namespace glance
