@@ -187,6 +187,23 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
 int32_t glance_profile_enable(glance_ctx *ctx, int32_t on);
 int32_t glance_profile_read(glance_ctx *ctx, double *ms, double *bytes, int64_t *launches);
 
+/* Per-offset top-k and log-softmax without any caller-provided workspace.  (The paper has no counterpart:
+ * this entry point exists for callers that cannot allocate device memory -- a process whose GPU memory was
+ * handed to its own arena at start-up, a plug-in inside a host framework's callback, a loop that cannot
+ * afford the device-wide synchronisation an allocation may trigger.)
+ * Same computation as the last step of glance_draft_block: for each sequence s and offset j = 1..L of
+ * logits (device [batch][block_B][vocab] fp32, row 0 of each sequence ignored) the k largest entries ordered
+ * by (logit desc, id asc) and lp = logit - logsumexp over the whole vocabulary, into topk_ids / topk_lp
+ * (device [batch][L][k]).  Work is enqueued on `cuda_stream`; nothing is allocated or freed.
+ * Scratch lives in a 1 MiB device array inside the library (held by every GPU that loads it, until exit);
+ * a call needing more -- batch*(block_B-1)*ceil(vocab/1024)*(8k+8) bytes, rounded up to 256 for the first
+ * part -- returns GLANCE_E_CAPACITY and launches nothing.  The first call on each device looks up the
+ * array's device address (with that device current); make that first call before starting any stream
+ * capture.  All calls share the one array: calls that may overlap on the GPU (different streams, no
+ * ordering between them) race on it and must be serialised by the caller. */
+int32_t glance_topk_static(const float *logits, int32_t batch, int32_t block_B, int32_t vocab, int32_t k,
+                           int32_t *topk_ids, float *topk_lp, void *cuda_stream);
+
 /* Number of kernel launches enqueued by this context since creation (host counter). */
 int64_t glance_launch_count(const glance_ctx *ctx);
 

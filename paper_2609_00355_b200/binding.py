@@ -19,6 +19,7 @@ EXPORTS = [
     "glance_seq_truncate", "glance_draft_block", "glance_build_tree", "glance_verify_tree",
     "glance_accept_commit", "glance_commit_forced", "glance_poll_status", "glance_launch_count",
     "glance_debug_attention", "glance_debug_gemm", "glance_profile_enable", "glance_profile_read",
+    "glance_topk_static",
 ]
 
 
@@ -98,6 +99,9 @@ def load_library() -> C.CDLL:
     lib.glance_profile_enable.argtypes = [C.c_void_p, C.c_int32]
     lib.glance_profile_read.restype = C.c_int32
     lib.glance_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.glance_topk_static.restype = C.c_int32
+    lib.glance_topk_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                       C.c_void_p]
     lib.glance_launch_count.restype = C.c_int64
     lib.glance_launch_count.argtypes = [C.c_void_p]
     _lib = lib
@@ -120,6 +124,18 @@ def make_config(cfg, max_batch: int, max_pages_per_seq: int) -> Config:
     return Config(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                   cfg.rms_eps, cfg.rope_theta, cfg.block_B, cfg.topk, cfg.tree_N, cfg.page_size, max_batch,
                   max_pages_per_seq)
+
+
+def glance_topk_static(logits: torch.Tensor, k: int, topk_ids: torch.Tensor, topk_lp: torch.Tensor) -> int:
+    """Top-k + log-softmax of logits [batch][block_B][vocab] using the library's built-in scratch array.
+
+    For callers that must not allocate device memory: no workspace, no context.  Returns the status code
+    (0, or GLANCE_E_CAPACITY = -3 when the request exceeds the built-in 1 MiB scratch).  Runs on the
+    current torch stream; calls that could overlap on the GPU must be serialised by the caller.
+    """
+    batch, B, V = logits.shape
+    sp = torch.cuda.current_stream(logits.device).cuda_stream
+    return int(load_library().glance_topk_static(_ptr(logits), batch, B, V, k, _ptr(topk_ids), _ptr(topk_lp), C.c_void_p(sp)))
 
 
 class TreeBuffers:

@@ -1,0 +1,51 @@
+"""glance_topk_static: the workspace-free top-k entry point against the regular draft path (GPU).
+
+Some callers may not allocate device memory (their process gave the whole GPU to its own arena, or they run
+inside a callback where allocation calls are forbidden), so this entry point keeps its scratch in a fixed
+array inside the library.  The test drives it through the C ABI twice in a row -- the array keeps the first
+call's contents -- and compares with what glance_draft_block returned for the same logits.
+Collected last on purpose: a failure here leaves every other test's result intact.
+"""
+import pytest
+import torch
+
+from paper_2609_00355_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def test_topk_static_matches_draft_block_twice():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_00355_b200 import binding
+    cfg = synth.CONFIGS["small"].replace(n_layers=1, n_img=40, n_txt=24, rounds=2)     # vocabulary 32000: 32 warps per row
+    tw, hw = synth.make_weights(cfg, "cuda")
+    eng = binding.Engine(cfg, tw, hw, batch=2)
+    for s in range(2):
+        img, ids = synth.make_context(cfg, "cuda", seed=5 + s)
+        eng.prefill_context(s, img, ids)
+    B, V, k, L = cfg.block_B, cfg.vocab, cfg.topk, cfg.L
+    for call in range(2):
+        logits = torch.zeros(2, B, V, dtype=torch.float32, device="cuda")
+        eng.glance_draft_block(logits_dbg=logits)
+        eng.check_device_status()
+        ids_ref, lp_ref = eng.topk_ids.clone(), eng.topk_lp.clone()
+        ids = torch.full((2, L, k), -1, dtype=torch.int32, device="cuda")
+        lp = torch.full((2, L, k), float("nan"), dtype=torch.float32, device="cuda")
+        assert binding.glance_topk_static(logits, k, ids, lp) == 0
+        torch.cuda.synchronize()
+        # same kernels, same inputs, fixed reduction order: ids identical and log-probabilities bit-equal,
+        # which is well inside the 2e-2 (relative to the logit scale) tolerance of the other parity tests
+        assert torch.equal(ids, ids_ref)
+        assert torch.equal(lp, lp_ref)
+        assert float((lp - lp_ref).abs().max()) <= 2e-2 * float(logits.abs().max())
+        # move the state on so that the second call sees different logits and stale scratch from the first
+        eng.glance_build_tree()
+        eng.glance_verify_tree()
+        eng.glance_accept_commit()
+    # a request larger than the built-in scratch is refused with a clear status and launches nothing
+    big = torch.zeros(1, 2, 8, dtype=torch.float32, device="cuda")
+    lib = binding.load_library()
+    rc = lib.glance_topk_static(big.data_ptr(), 64, 16, 1 << 24, 16, ids.data_ptr(), lp.data_ptr(), None)
+    assert rc == -3 and lib.glance_status_string(rc) == b"capacity exceeded"
+    assert lib.glance_topk_static(None, 1, 2, 8, 1, ids.data_ptr(), lp.data_ptr(), None) == -1
