@@ -179,7 +179,7 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
 /* Measurement aid.  While enabled, every kernel launch is bracketed by a pair of CUDA events on the context's
  * stream (the pairs are created when profiling is first enabled, so the round calls still allocate nothing).
  * glance_profile_read synchronises the stream and fills three arrays of GLANCE_PROFILE_KINDS entries, indexed by
- * kernel kind (0 weight-streaming GEMM, 1 attention, 2 residual+norm, 3 rotary + K/V write, 4 everything
+ * kernel kind (0 weight-streaming GEMM, 1 attention, 2 row setup, 3 top-k / tree / walk+commit, 4 everything
  * else): summed device time in milliseconds, summed algorithmic bytes (GEMM only: weights once +
  * activations in + results out) and launch count; then it resets the tally.  Disabling only pauses the
  * tally.  At most 32768 launches are tallied per read. */

@@ -282,10 +282,10 @@ class Engine:
         _check(self.lib.glance_profile_enable(self.ctx, 1 if on else 0), "glance_profile_enable")
 
     def glance_profile_read(self):
-        """Per kernel kind (gemm, attention, norm, rope_kv, other): (ms, algorithmic bytes, launches)."""
+        """Per kernel kind (gemm, attention, setup, control, other): (ms, algorithmic bytes, launches)."""
         ms, by, n = (C.c_double * 5)(), (C.c_double * 5)(), (C.c_int64 * 5)()
         _check(self.lib.glance_profile_read(self.ctx, ms, by, n), "glance_profile_read")
-        names = ("gemm", "attention", "norm", "rope_kv", "other")
+        names = ("gemm", "attention", "setup", "control", "other")
         return {names[i]: (ms[i], by[i], n[i]) for i in range(5)}
 
     def glance_launch_count(self) -> int:
@@ -310,6 +310,20 @@ class Engine:
             self.glance_build_tree()
         self.glance_verify_tree()
         self.glance_accept_commit()
+
+    def capture(self, fn):
+        """Records the launches `fn()` makes on the engine's stream into a CUDA graph and returns the graph.
+
+        The engine must have been created with its own (non-default) stream, and `fn` must already have run
+        once (kernel attributes and TMA descriptors are set up on first use).  All ragged quantities (sequence
+        lengths, accept lengths, page ids) are read from device memory by the kernels, so one graph serves
+        every round.  Replay with graph.replay() while the engine's stream is current.
+        """
+        assert self.stream is not None, "create the Engine with its own stream to capture graphs"
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=self.stream):
+            fn()
+        return g
 
     def snapshot_state(self):
         return (self.seq_len.clone(), self.root.clone(), self.feat.clone(), self.feat_count.clone())

@@ -31,7 +31,7 @@ struct KvGeom {
 struct RowMeta {
     int32_t *seq;     // [R] sequence of the row
     int32_t *pos;     // [R] rotary position, -1 for a padding row
-    int32_t *kvslot;  // [R] logical cache position to write K/V to, -1 = none
+    long long *kvrow; // [R] element offset of the row's K slot (kv head 0) inside a pool layer, -1 = none
     float *rope_cos;  // [R][d/2]
     float *rope_sin;  // [R][d/2]
 };

@@ -10,7 +10,9 @@
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
 // Epilogues: (0) fp32 split-K plane, (1) SwiGLU over a gate tile and its up tile (two accumulators),
-// (2) row-wise arg-max over the vocabulary, merged across CTAs with a packed 64-bit atomic max.
+// (2) row-wise arg-max over the vocabulary, merged across CTAs with a packed 64-bit atomic max,
+// (3)/(4) split-K reduced inside a thread-block cluster through distributed shared memory, followed by
+// residual add + norm statistics, or rotary embedding + paged K/V write.
 // Every wait on an mbarrier is bounded; a wait that gives up records GLANCE_E_TIMEOUT, and the CTA
 // drains and frees its TMEM before it returns.
 #include <cuda.h>
@@ -115,16 +117,41 @@ struct alignas(8) Barriers {
     int abort_flag;
 };
 
-// MODE 0: fp32 plane; MODE 1: SwiGLU (dual accumulator); MODE 2: arg-max (+ optional fp32 logits)
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// address of `local_addr` (a shared-memory address of this CTA) inside CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t local_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+// MODE 0: fp32 planes              MODE 1: SwiGLU (two accumulators)      MODE 2: arg-max (+ optional logits)
+// MODE 3: split-K over a cluster, residual add + bf16 copy scaled by the next norm's gain + sum of squares
+// MODE 4: split-K over a cluster, rotary embedding + q / paged K,V write
+// Modes 0, 1, 2 and 4 multiply each activation row's results by 1/rms(row) when a.ssq is given: the rows
+// they read are x * gain in bf16, and the row's sum of squares arrives as per-tile partial sums.
 template <int MODE>
-__global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+__global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                          const __grid_constant__ CUtensorMap map_x, TcGemmArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ Barriers bars;
     __shared__ unsigned long long red_keys[4][128];
+    __shared__ float inv_rms[128];
+    __shared__ float red_sq[4][128];
 
     constexpr int NW = (MODE == 1) ? 2 : 1;              // weight tiles per stage
+    constexpr bool CLUSTERED = (MODE >= 3);
     const int NP = a.np;                                 // UMMA N (activation rows, padded to 16)
     const int stage_bytes = NW * BM * 128 + NP * 128;
     const int stages = a.stages;
@@ -155,6 +182,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = bars.tmem_base;
     volatile int *abort_flag = &bars.abort_flag;
+    bool ok = true;                                      // epilogue warps: accumulator is valid
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -187,11 +215,11 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc(NP);
-            bool ok = true;
-            for (int i = 0; i < nk && ok; ++i) {
+            bool mok = true;
+            for (int i = 0; i < nk && mok; ++i) {
                 const int s = i % stages;
                 const uint32_t ph = (uint32_t)(i / stages) & 1u;
-                if (!mbar_wait(&bars.full[s], ph, abort_flag, a.status)) { ok = false; break; }
+                if (!mbar_wait(&bars.full[s], ph, abort_flag, a.status)) { mok = false; break; }
                 tc_fence_after();
                 const uint32_t slot = smem_u32(smem + (size_t)s * stage_bytes);
                 const uint64_t bdesc = umma_desc(slot + NW * BM * 128);
@@ -205,21 +233,34 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
                 }
                 umma_commit(&bars.empty[s]);             // slot reusable once these MMAs have read it
             }
-            if (ok) umma_commit(&bars.acc_ready);
+            if (mok) umma_commit(&bars.acc_ready);
         }
     } else {
-        // ---------------- epilogue: TMEM -> registers -> global ----------------
-        const int q = warp & 3;                          // TMEM lane quarter this warp may read
-        const int f = f0 + q * 32 + lane;
-        bool ok = true;
+        // ---------------- epilogue warps, part 1: row scales, then wait for the accumulator ----------------
+        const int t = threadIdx.x - 64;                  // 0..127
+        if (MODE != 3) {
+            float inv = 1.f;
+            if (a.ssq && t < NP && r0 + t < a.R) {
+                float ss = 0.f;
+                for (int i = 0; i < a.n_ssq; ++i) ss += __ldcg(a.ssq + (size_t)i * a.ssq_stride + r0 + t);
+                inv = rsqrtf(ss / (float)a.K + a.eps);
+            }
+            inv_rms[t] = inv;
+        }
+        if (MODE == 2) red_keys[warp & 3][lane] = red_keys[warp & 3][lane + 32] = red_keys[warp & 3][lane + 64] = red_keys[warp & 3][lane + 96] = 0ull;
         if (nk > 0) ok = mbar_wait(&bars.acc_ready, 0, abort_flag, a.status);
         ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld is warp-collective: decide as a warp
         tc_fence_after();
-        const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-        if (MODE == 2)
-            for (int r = lane; r < 128; r += 32) red_keys[q][r] = 0ull;
-        __syncwarp();
-        if (ok) {
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // inv_rms / red_keys visible to the four epilogue warps
+    }
+
+    const int q = warp & 3;                              // TMEM lane quarter an epilogue warp may read
+    const int fl = q * 32 + lane;                        // feature within the tile
+    const int f = f0 + fl;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
+
+    if (!CLUSTERED) {
+        if (warp >= 2 && ok) {
             for (int c = 0; c < NP; c += 16) {
                 uint32_t v[16];
                 if (nk > 0) {
@@ -235,7 +276,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int r = r0 + c + j;
-                            if (r < a.R) Ys[(size_t)r * a.ldy + f] = __uint_as_float(v[j]);
+                            if (r < a.R) Ys[(size_t)r * a.ldy + f] = __uint_as_float(v[j]) * inv_rms[c + j];
                         }
                     }
                 } else if (MODE == 1) {
@@ -246,7 +287,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int r = r0 + c + j;
-                            const float g = __uint_as_float(v[j]), up = __uint_as_float(u[j]);
+                            const float g = __uint_as_float(v[j]) * inv_rms[c + j], up = __uint_as_float(u[j]) * inv_rms[c + j];
                             if (r < a.R) a.act[(size_t)r * a.F + f] = __float2bfloat16(g / (1.f + __expf(-g)) * up);
                         }
                     }
@@ -254,7 +295,7 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int r = r0 + c + j;
-                        const float val = __uint_as_float(v[j]);
+                        const float val = __uint_as_float(v[j]) * inv_rms[c + j];
                         if (a.Y && f < a.Nout && r < a.R) a.Y[(size_t)r * a.ldy + f] = val;
                         unsigned long long key = (f < a.Nout) ? pack_val_id(val, f) : 0ull;
                         key = warp_max_u64(key);
@@ -263,9 +304,9 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
                 }
             }
         }
-        if (MODE == 2) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");       // the four epilogue warps only
-            const int t = threadIdx.x - 64;                       // 0..127
+        if (MODE == 2 && warp >= 2) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int t = threadIdx.x - 64;
             const int r = r0 + t;
             if (ok && t < NP && r < a.R) {
                 unsigned long long k = red_keys[0][t];
@@ -273,8 +314,114 @@ __global__ void __launch_bounds__(192, 1) gemm_tc_kernel(const __grid_constant__
                 atomicMax(a.keys + r, k);
             }
         }
-        tc_fence_before();
+    } else {
+        // ---------------- split-K over the cluster, reduce-scatter by rows: CTA `rank` owns activation rows
+        // [rank*RP, rank*RP + RP) of the tile.  Every CTA ships, for each row, its fp32 partial results to the
+        // owner's shared memory (planes [source split][row][feature], aliased onto the owner's idle TMA ring);
+        // the owner adds the planes in split order and applies the fused epilogue to its rows ----------------
+        const uint32_t rank = cluster_rank();
+        const int RP = (NP + a.S - 1) / a.S;             // rows per owner
+        cluster_sync_all();                              // every CTA's MMAs are done: all rings are idle
+        if (warp >= 2) {
+            const uint32_t local = smem_u32(smem) + (uint32_t)((rank * RP) * BM * 4) + (uint32_t)(fl * 4);
+            for (int c = 0; c < NP; c += 16) {
+                uint32_t v[16];
+                if (nk > 0 && ok) {
+                    tmem_ld16(lane_addr + (uint32_t)c, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0u;
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const int r = c + j;
+                    const uint32_t owner = (uint32_t)(r / RP);
+                    st_cluster_f32(map_to_rank(local + (uint32_t)((r - owner * RP) * BM * 4), owner), __uint_as_float(v[j]));
+                }
+            }
+        }
+        cluster_sync_all();                              // planes written and visible
+        if (warp >= 2) {
+            const float *planes = reinterpret_cast<const float *>(smem);
+            const int row_lo = (int)rank * RP;                                   // first owned row (tile-local)
+            const int my_rows = max(0, min(min(RP, NP - row_lo), a.R - r0 - row_lo));
+            if (MODE == 3) {
+                const bool valid = f < a.Nout;
+                const float gain = valid ? __bfloat162float(a.gain[f]) : 0.f;
+                for (int rb = 0; rb < my_rows; rb += 8) {
+                    float xv[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        xv[j] = (valid && rb + j < my_rows) ? __ldcg(a.x + (size_t)(r0 + row_lo + rb + j) * a.Nout + f) : 0.f;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int lr = rb + j;
+                        if (lr >= my_rows) break;            // uniform across the warp
+                        float v = 0.f;
+                        for (int k = 0; k < a.S; ++k) v += planes[(size_t)(k * RP + lr) * BM + fl];
+                        float sq = 0.f;
+                        if (valid) {
+                            const size_t o = (size_t)(r0 + row_lo + lr) * a.Nout + f;
+                            const float xn = xv[j] + v;
+                            a.x[o] = xn;
+                            a.xb[o] = __float2bfloat16(xn * gain);
+                            if (a.hidden_out) a.hidden_out[o] = __float2bfloat16(xn);
+                            sq = xn * xn;
+                        }
+                        sq = warp_sum(sq);
+                        if (lane == 0) red_sq[q][lr] = sq;
+                    }
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int t = threadIdx.x - 64;
+                if (t < my_rows)
+                    a.ssq_out[(size_t)blockIdx.x * a.ssq_stride + r0 + row_lo + t] =
+                        ((red_sq[0][t] + red_sq[1][t]) + red_sq[2][t]) + red_sq[3][t];
+            } else {
+                const int d = a.head_dim, half = d >> 1;
+                const int h = f / d, i = f % d;
+                const bool is_q = h < a.Hq, is_k = !is_q && h < a.Hq + a.Hkv, valid = f < a.Nout;
+                const int pfl = (i < half) ? fl + half : fl - half;          // rotary partner, same tile
+                const int ci = (i < half) ? i : i - half;
+                const int kvh = is_k ? h - a.Hq : h - a.Hq - a.Hkv;
+                for (int rb = 0; rb < my_rows; rb += 8) {
+                    float cs[8], sn[8];
+                    long long base[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int rr = r0 + row_lo + rb + j;
+                        const bool live = valid && rb + j < my_rows;
+                        cs[j] = (live && !(!is_q && !is_k)) ? a.rope_cos[(size_t)rr * half + ci] : 1.f;
+                        sn[j] = (live && !(!is_q && !is_k)) ? a.rope_sin[(size_t)rr * half + ci] : 0.f;
+                        base[j] = (live && !is_q) ? a.kvrow[rr] : -1;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int lr = rb + j;
+                        if (lr >= my_rows) break;
+                        const int rr = r0 + row_lo + lr;
+                        float va = 0.f, vb = 0.f;
+                        for (int k = 0; k < a.S; ++k) {
+                            const float *pl = planes + (size_t)(k * RP + lr) * BM;
+                            va += pl[fl];
+                            vb += pl[pfl];
+                        }
+                        if (!valid) continue;
+                        va *= inv_rms[row_lo + lr];
+                        vb *= inv_rms[row_lo + lr];
+                        const float out = (is_q || is_k) ? ((i < half) ? va * cs[j] - vb * sn[j] : va * cs[j] + vb * sn[j]) : va;
+                        if (is_q) {
+                            if (rr < a.Rq) a.q[((size_t)rr * a.Hq + h) * d + i] = __float2bfloat16(out);
+                        } else if (base[j] >= 0) {
+                            a.pool_layer[(size_t)base[j] + (is_k ? 0 : a.v_off) + (size_t)kvh * a.head_stride + i] = __float2bfloat16(out);
+                        }
+                    }
+                }
+            }
+        }
     }
+    tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
@@ -326,8 +473,19 @@ cudaError_t launch_mode(const TcGemmArgs &a, const CUtensorMap &mw, const CUtens
         if (e != cudaSuccess) return e;
         once = true;
     }
-    gemm_tc_kernel<MODE><<<grid, 192, smem, st>>>(mw, mx, a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(192, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = (MODE >= 3) ? grid.y : 1;     // the K splits of one tile form a cluster
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MODE>, mw, mx, a);
 }
 
 }  // namespace
@@ -354,8 +512,10 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     a.np = tc_row_pad(a.R);
     const int nw = (mode == 1) ? 2 : 1;
     const int stage_bytes = nw * BM * 128 + a.np * 128;
-    int stages = (int)((212 * 1024) / stage_bytes);
-    stages = stages > 12 ? 12 : stages;
+    // Clustered modes keep the ring under half of an SM's shared memory so that two CTAs fit per SM: a GPC
+    // then offers enough CTA slots for every cluster of the launch to be resident in one wave.
+    int stages = (int)(((mode >= 3 ? 100 : 212) * 1024) / stage_bytes);
+    stages = stages > 12 ? 12 : (stages < 2 ? 2 : stages);
     a.stages = stages;
     uint32_t cols = 32;
     while ((int)cols < nw * a.np) cols <<= 1;
@@ -363,9 +523,16 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     const int tiles = ((mode == 1 ? a.F : a.Nout) + BM - 1) / BM;
     dim3 grid(tiles, a.S, (a.R + 127) / 128);
+    if (mode >= 3) {
+        // every CTA's ring must hold S planes of ceil(np/S) rows, and a cluster has at most 8 CTAs
+        const size_t rp = (a.np + a.S - 1) / a.S;
+        if (a.S > 8 || (size_t)a.S * rp * BM * 4 > (size_t)stages * stage_bytes) return cudaErrorInvalidValue;
+    }
     if (mode == 0) return launch_mode<0>(a, map_w, map_x, smem, grid, st);
     if (mode == 1) return launch_mode<1>(a, map_w, map_x, smem, grid, st);
-    return launch_mode<2>(a, map_w, map_x, smem, grid, st);
+    if (mode == 2) return launch_mode<2>(a, map_w, map_x, smem, grid, st);
+    if (mode == 3) return launch_mode<3>(a, map_w, map_x, smem, grid, st);
+    return launch_mode<4>(a, map_w, map_x, smem, grid, st);
 }
 
 }  // namespace glance

@@ -20,6 +20,22 @@ struct TcGemmArgs {
     int32_t *argmax;
     int32_t *counter;
     int32_t *status;
+    // row scales (modes 0, 1, 2, 4): row r is multiplied by rsqrt(sum_i ssq[i*ssq_stride + r] / K + eps); nullptr = 1
+    const float *ssq;
+    int n_ssq, ssq_stride;
+    float eps;
+    // mode 3 (residual): x[r][f] += result; xb = bf16(x * gain[f]); ssq_out[tile][r] = sum over the tile of x^2
+    float *x;
+    const bf16 *gain;
+    bf16 *xb, *hidden_out;
+    float *ssq_out;
+    // mode 4 (rotary + K/V write): features are q heads, then k heads, then v heads, head_dim wide
+    bf16 *q;
+    bf16 *pool_layer;
+    const long long *kvrow;      // [R] element offset of the row's K slot for kv head 0 inside the layer, -1 = none
+    size_t v_off, head_stride;
+    const float *rope_cos, *rope_sin;   // [R][head_dim/2]
+    int Hq, Hkv, head_dim, Rq;
     // filled by launch_gemm_tc
     int np, stages;
     uint32_t tmem_cols;
@@ -29,7 +45,7 @@ struct TcGemmArgs {
 bool tc_make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows);
 // activation rows per CTA, padded to the UMMA N granularity (box_rows of the X map)
 int tc_row_pad(int R);
-// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max.  map_w box_rows must be 128, map_x box_rows tc_row_pad(R).
+// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max, 3 cluster split-K + residual, 4 cluster split-K + rotary/KV write.  map_w box_rows must be 128, map_x box_rows tc_row_pad(R).
 cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, const CUtensorMap &map_x, cudaStream_t st);
 
 }  // namespace glance

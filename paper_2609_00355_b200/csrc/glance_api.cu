@@ -17,18 +17,19 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // split-K factor of a weight-streaming GEMM: as many CTAs as fit one wave of the 148 SMs, at least 8 k-tiles
 // per split
-int choose_split(int Nout, int K) {
+// The splits of one tile form a thread-block cluster (<= 8 CTAs) that reduces them through shared memory.
+int choose_split(int Nout, int K, int rows) {
     const int tiles = (Nout + 127) / 128;
     const int ktiles = K / 64;
+    (void)rows;
     int s = 148 / tiles;
     s = std::min(s, std::max(1, ktiles / 8));
-    return std::max(1, std::min(s, 16));
+    return std::max(1, std::min(s, 8));
 }
 
 struct Workspace {
     float *x;            // [Rmax][H] residual stream
     bf16 *xn;            // [Rmax][H]
-    float *part;         // split-K planes
     bf16 *q;             // [Rmax][Hq d]
     bf16 *attn;          // [Rmax][Hq d]
     bf16 *act;           // [Rmax][F]
@@ -37,7 +38,9 @@ struct Workspace {
     float *att_ml;
     int32_t *att_ctr;
     int32_t *walk_ctr;
-    int32_t *row_seq, *row_pos, *row_kvslot;
+    int32_t *row_seq, *row_pos;
+    long long *row_kvrow;
+    float *ssq;            // [n_ssq][Rmax] per-tile sums of squares of the residual rows
     float *rope_cos, *rope_sin;
     uint64_t *chain_anc;   // [N][W] prefill chain mask
     bf16 *hidden_tmp;      // [N][H] prefill hidden
@@ -47,12 +50,11 @@ struct Workspace {
     int32_t *am_counter;
     unsigned long long *topk_cand; // [batch*L][warps][k]
     float *topk_ml;                // [batch*L][warps][2]
-    size_t part_elems;
     size_t total;
 };
 
 struct Dims {
-    int Rmax, Rlog, qkv_out, qd, S_qkv, S_o, S_d, S_att, q_tiles_max, W;
+    int Rmax, Rlog, qkv_out, qd, S_att, q_tiles_max, W, n_ssq;
 };
 
 Dims make_dims(const glance_config &c) {
@@ -62,9 +64,7 @@ Dims make_dims(const glance_config &c) {
     d.Rlog = c.max_batch * std::max(c.tree_N, c.block_B);
     d.qkv_out = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
     d.qd = c.n_q_heads * c.head_dim;
-    d.S_qkv = choose_split(d.qkv_out, c.hidden);
-    d.S_o = choose_split(c.hidden, d.qd);
-    d.S_d = choose_split(c.hidden, c.ffn);
+    d.n_ssq = (c.hidden + 127) / 128;
     const int G = c.n_q_heads / c.n_kv_heads;
     d.q_tiles_max = attention_q_tiles(std::max(c.tree_N, c.block_B), G);
     // attention split partials: the largest (q tiles x key splits) over every row count a pass can have
@@ -87,9 +87,6 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     const size_t R = d.Rmax, H = c.hidden;
     w.x = (float *)take(R * H * 4);
     w.xn = (bf16 *)take(R * H * 2);
-    size_t pe = std::max({(size_t)d.S_qkv * R * d.qkv_out, (size_t)d.S_o * R * H, (size_t)d.S_d * R * H});
-    w.part_elems = pe;
-    w.part = (float *)take(pe * 4);
     w.q = (bf16 *)take(R * d.qd * 2);
     w.attn = (bf16 *)take(R * d.qd * 2);
     w.act = (bf16 *)take(R * (size_t)c.ffn * 2);
@@ -101,7 +98,8 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.walk_ctr = (int32_t *)take((size_t)c.max_batch * 4);
     w.row_seq = (int32_t *)take(R * 4);
     w.row_pos = (int32_t *)take(R * 4);
-    w.row_kvslot = (int32_t *)take(R * 4);
+    w.row_kvrow = (long long *)take(R * 8);
+    w.ssq = (float *)take((size_t)d.n_ssq * R * 4);
     w.rope_cos = (float *)take(R * (c.head_dim / 2) * 4);
     w.rope_sin = (float *)take(R * (c.head_dim / 2) * 4);
     w.chain_anc = (uint64_t *)take((size_t)c.tree_N * d.W * 8);
@@ -154,7 +152,7 @@ struct glance_ctx {
 
 namespace {
 
-enum { KIND_GEMM = 0, KIND_ATTN = 1, KIND_NORM = 2, KIND_ROPE = 3, KIND_OTHER = 4, KIND_COUNT = 5 };
+enum { KIND_GEMM = 0, KIND_ATTN = 1, KIND_SETUP = 2, KIND_CONTROL = 3, KIND_OTHER = 4, KIND_COUNT = 5 };
 
 constexpr size_t kMaxProfiled = 32768;
 
@@ -191,25 +189,27 @@ const CUtensorMap *get_map(glance_ctx *ctx, const void *base, int inner, int row
     return &ctx->maps.emplace(key, m).first->second;
 }
 
-// The weight-streaming GEMM.  mode 0: fp32 split-K planes Y[s][r][f]; mode 1: SwiGLU into act (W = gate rows
-// then up rows, Nout = 2F); mode 2: arg-max over f into `argmax` (optional fp32 logits in Y).
-// x_rows = rows allocated behind X (rows of its tensor map).
-void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, int Nout, int K, int R, int S, float *Y,
-          int ldy, size_t split_stride, bf16 *act, int32_t *argmax) {
-    const CUtensorMap *mw = get_map(ctx, W, K, Nout, 128);
-    const CUtensorMap *mx = get_map(ctx, X, K, x_rows, tc_row_pad(R));
+// Launches the weight-streaming GEMM described by `a` (mode: see gemm_tc.cuh) on X [R][K] (x_rows rows are
+// allocated behind X) and W [Nout][K], and tallies its algorithmic bytes.
+void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, TcGemmArgs a) {
+    const CUtensorMap *mw = get_map(ctx, W, a.K, a.Nout, 128);
+    const CUtensorMap *mx = get_map(ctx, X, a.K, x_rows, tc_row_pad(a.R));
     if (!mw || !mx) return;
-    TcGemmArgs a{};
-    a.Nout = Nout; a.K = K; a.R = R; a.S = mode == 0 ? S : 1; a.Y = Y; a.ldy = ldy; a.split_stride = split_stride;
-    a.act = act; a.F = Nout / 2; a.keys = ctx->ws.am_keys; a.argmax = argmax; a.counter = ctx->ws.am_counter;
-    a.status = ctx->ws.status;
+    a.keys = ctx->ws.am_keys; a.counter = ctx->ws.am_counter; a.status = ctx->ws.status;
     const bool prof = prof_begin(ctx);
     if (launch_gemm_tc(mode, a, *mw, *mx, ctx->stream) != cudaSuccess) ctx->map_error = true;
-    double bytes = 2.0 * Nout * K + 2.0 * R * K;
-    if (mode == 0) bytes += 4.0 * a.S * R * Nout;
-    else if (mode == 1) bytes += 2.0 * R * (Nout / 2);
-    else bytes += 4.0 * R + (Y ? 4.0 * R * Nout : 0.0);
+    double bytes = 2.0 * a.Nout * a.K + 2.0 * a.R * a.K;
+    if (mode == 0) bytes += 4.0 * a.S * a.R * a.Nout;
+    else if (mode == 1) bytes += 2.0 * a.R * a.F;
+    else if (mode == 2) bytes += 4.0 * a.R + (a.Y ? 4.0 * a.R * a.Nout : 0.0);
+    else if (mode == 3) bytes += (4.0 + 4.0 + 2.0) * a.R * a.Nout;     // residual in/out + bf16 copy
+    else bytes += 2.0 * a.R * a.Nout;
     prof_end(ctx, prof, KIND_GEMM, bytes);
+}
+
+// row scales 1/rms from the per-tile sums of squares the producer left in ws.ssq
+void with_row_scales(const glance_ctx *ctx, TcGemmArgs &a) {
+    a.ssq = ctx->ws.ssq; a.n_ssq = ctx->dims.n_ssq; a.ssq_stride = ctx->dims.Rmax; a.eps = ctx->cfg.rms_eps;
 }
 
 struct LayerW {
@@ -238,14 +238,28 @@ RowMeta meta_of(const glance_ctx *ctx) {
     RowMeta m;
     m.seq = ctx->ws.row_seq;
     m.pos = ctx->ws.row_pos;
-    m.kvslot = ctx->ws.row_kvslot;
+    m.kvrow = ctx->ws.row_kvrow;
     m.rope_cos = ctx->ws.rope_cos;
     m.rope_sin = ctx->ws.rope_sin;
     return m;
 }
 
-// One decoder layer over the rows of a pass.  On entry ws.xn holds the normalised input rows; on exit
-// ws.x holds the new residual stream and ws.xn the rows normalised with `next_gain`.
+RowOut rowout_of(const glance_ctx *ctx) {
+    RowOut o;
+    o.H = ctx->cfg.hidden;
+    o.x = ctx->ws.x;
+    o.xb = ctx->ws.xn;
+    o.ssq = ctx->ws.ssq;
+    o.n_ssq = ctx->dims.n_ssq;
+    o.ssq_stride = ctx->dims.Rmax;
+    return o;
+}
+
+// One decoder layer over the rows of a pass: five launches.
+//   QKV GEMM (+ 1/rms row scale, rotary, q / paged K,V write)  ->  attention  ->
+//   O GEMM (+ residual, bf16 copy scaled by ln2, sums of squares)  ->
+//   gate/up GEMM (+ 1/rms row scale, SwiGLU)  ->  down GEMM (+ residual, bf16 copy scaled by next_gain, sums of squares)
+// On entry ws.x is the residual stream, ws.xn = bf16(x * gain) and ws.ssq its sums of squares; same on exit.
 void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInfo &ps, const bf16 *next_gain,
                bf16 *hidden_out) {
     const glance_config &c = ctx->cfg;
@@ -256,15 +270,16 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     const int32_t *page_table = ps.seqs->page_table + (size_t)ps.seq_off * c.max_pages_per_seq;
     const int32_t *seq_len = ps.seqs->seq_len + ps.seq_off;
     const int xr = d.Rmax;                             // rows allocated behind every activation buffer
-    // QKV projection (split-K planes), reduced by the rotary / K-V write kernel
-    size_t ss = (size_t)ps.R * d.qkv_out;
-    gemm(ctx, 0, w.wqkv, ws.xn, xr, d.qkv_out, c.hidden, ps.R, d.S_qkv, ws.part, d.qkv_out, ss, nullptr, nullptr);
-    RopeKv rk;
-    rk.R = ps.R; rk.Rq = ps.Rq; rk.Hq = c.n_q_heads; rk.Hkv = c.n_kv_heads; rk.d = c.head_dim;
-    rk.part = ws.part; rk.S = d.S_qkv; rk.split_stride = ss; rk.ldy = d.qkv_out;
-    rk.meta = meta_of(ctx); rk.q = ws.q; rk.pool_layer = pool_layer; rk.geom = geom; rk.page_table = page_table;
-    rk.status = ws.status;
-    LAUNCH(ctx, KIND_ROPE, launch_rope_kv(rk, st));
+    {
+        TcGemmArgs g{};
+        g.Nout = d.qkv_out; g.K = c.hidden; g.R = ps.R; g.S = choose_split(d.qkv_out, c.hidden, ps.R);
+        with_row_scales(ctx, g);
+        g.q = ws.q; g.pool_layer = pool_layer; g.kvrow = ws.row_kvrow;
+        g.v_off = (size_t)c.n_kv_heads * kPage * c.head_dim; g.head_stride = (size_t)kPage * c.head_dim;
+        g.rope_cos = ws.rope_cos; g.rope_sin = ws.rope_sin;
+        g.Hq = c.n_q_heads; g.Hkv = c.n_kv_heads; g.head_dim = c.head_dim; g.Rq = ps.Rq;
+        gemm(ctx, 4, w.wqkv, ws.xn, xr, g);
+    }
     if (ps.Rq == 0) return;
     AttnParams ap;
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
@@ -274,34 +289,42 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     ap.part_ml = ws.att_ml; ap.counters = ws.att_ctr; ap.status = ws.status;
     LAUNCH(ctx, KIND_ATTN, launch_attention(ap, st));
     const int R = ps.Rq;
-    // output projection (split-K planes), reduced by residual + norm
-    ss = (size_t)R * c.hidden;
-    gemm(ctx, 0, w.wo, ws.attn, xr, c.hidden, d.qd, R, d.S_o, ws.part, c.hidden, ss, nullptr, nullptr);
-    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, ws.part, d.S_o, ss, c.hidden, R, c.hidden, w.ln2, nullptr, R, c.rms_eps,
-                                       ws.xn, nullptr, st));
-    // SwiGLU MLP: gate/up GEMM with the activation fused into its epilogue, then down projection
-    gemm(ctx, 1, w.wgu, ws.xn, xr, 2 * c.ffn, c.hidden, R, 1, nullptr, 0, 0, ws.act, nullptr);
-    gemm(ctx, 0, w.wd, ws.act, xr, c.hidden, c.ffn, R, d.S_d, ws.part, c.hidden, ss, nullptr, nullptr);
-    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, ws.part, d.S_d, ss, c.hidden, R, c.hidden, next_gain, nullptr, R,
-                                       c.rms_eps, ws.xn, hidden_out, st));
+    {
+        TcGemmArgs g{};
+        g.Nout = c.hidden; g.K = d.qd; g.R = R; g.S = choose_split(c.hidden, d.qd, R);
+        g.x = ws.x; g.gain = w.ln2; g.xb = ws.xn; g.ssq_out = ws.ssq; g.ssq_stride = d.Rmax;
+        gemm(ctx, 3, w.wo, ws.attn, xr, g);
+    }
+    {
+        TcGemmArgs g{};
+        g.Nout = 2 * c.ffn; g.K = c.hidden; g.R = R; g.S = 1; g.act = ws.act; g.F = c.ffn;
+        with_row_scales(ctx, g);
+        gemm(ctx, 1, w.wgu, ws.xn, xr, g);
+    }
+    {
+        TcGemmArgs g{};
+        g.Nout = c.hidden; g.K = c.ffn; g.R = R; g.S = choose_split(c.hidden, c.ffn, R);
+        g.x = ws.x; g.gain = next_gain; g.xb = ws.xn; g.hidden_out = hidden_out; g.ssq_out = ws.ssq; g.ssq_stride = d.Rmax;
+        gemm(ctx, 3, w.wd, ws.act, xr, g);
+    }
 }
 
-// all target layers + final norm (+ LM head and argmax) over rows already set up in ws.x
+// all target layers (+ LM head with fused arg-max) over rows prepared by a setup kernel
 void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *logits, int32_t *argmax) {
     const glance_config &c = ctx->cfg;
-    Workspace &ws = ctx->ws;
-    cudaStream_t st = ctx->stream;
     const KvGeom geom = geom_of(ctx, ps.seqs);
-    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, nullptr, 0, 0, c.hidden, ps.R, c.hidden, ctx->ln1[0], nullptr, ps.R,
-                                       c.rms_eps, ws.xn, nullptr, st));
     for (int l = 0; l < c.n_layers; ++l) {
         LayerW w{ctx->ln2[l], ctx->wqkv[l], ctx->wo[l], ctx->wgu[l], ctx->wd[l]};
         const bool last = (l + 1 == c.n_layers);
         bf16 *pool_layer = (bf16 *)ps.seqs->kv_pool + (size_t)l * geom.layer_stride();
         run_layer(ctx, w, pool_layer, ps, last ? ctx->final_norm : ctx->ln1[l + 1], last ? hidden_out : nullptr);
     }
-    if (argmax)   // LM head with the arg-max fused into its epilogue; logits are stored only on request
-        gemm(ctx, 2, ctx->lm_head, ws.xn, ctx->dims.Rmax, c.vocab, c.hidden, ps.R, 1, logits, c.vocab, 0, nullptr, argmax);
+    if (argmax) {   // logits are stored only on request
+        TcGemmArgs g{};
+        g.Nout = c.vocab; g.K = c.hidden; g.R = ps.R; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.argmax = argmax;
+        with_row_scales(ctx, g);
+        gemm(ctx, 2, ctx->lm_head, ctx->ws.xn, ctx->dims.Rmax, g);
+    }
 }
 
 int32_t check_seqs(const glance_ctx *ctx, const glance_seqs *s) {
@@ -418,32 +441,34 @@ int32_t glance_prefill(glance_ctx *ctx, const glance_seqs *seqs, int32_t seq, co
     for (int done = 0; done < count; done += N) {
         const int n = std::min(N, count - done);
         const bool last = (done + n == count);
-        VerifySetup vs;
-        vs.batch = 1; vs.N = N; vs.H = c.hidden; vs.d = c.head_dim; vs.theta = c.rope_theta;
+        const KvGeom tg = geom_of(ctx, seqs);
+        const int32_t *pt = seqs->page_table + (size_t)seq * c.max_pages_per_seq;
+        VerifySetup vs{};
+        vs.batch = 1; vs.N = N; vs.d = c.head_dim; vs.theta = c.rope_theta;
         vs.seq_len = seqs->seq_len + seq; vs.token = nullptr; vs.depth = nullptr;
         vs.row_embeds = embeds ? (const bf16 *)embeds + (size_t)done * c.hidden : nullptr;
         vs.row_ids = ids ? ids + done : nullptr;
-        vs.count = n; vs.chain_anc = ws.chain_anc; vs.embed = ctx->embed; vs.vocab = c.vocab;
-        vs.capacity = c.max_pages_per_seq * kPage; vs.x = ws.x; vs.meta = meta_of(ctx); vs.status = ws.status;
-        LAUNCH(ctx, KIND_OTHER, launch_setup_verify(vs, st));
+        vs.count = n; vs.chain_anc = ws.chain_anc; vs.embed = ctx->embed; vs.gain = ctx->ln1[0]; vs.vocab = c.vocab;
+        vs.capacity = c.max_pages_per_seq * kPage; vs.geom = tg; vs.page_table = pt; vs.out = rowout_of(ctx);
+        vs.meta = meta_of(ctx); vs.status = ws.status;
+        LAUNCH(ctx, KIND_SETUP, launch_setup_verify(vs, st));
         PassInfo ps{N, N, 1, N, ws.chain_anc, seqs, seq};
         run_target(ctx, ps, ws.hidden_tmp, nullptr, last ? ws.argmax_tmp : nullptr);
         // head context K/V of the new positions (Section 3.2: keys and values are the target's hidden states)
-        DraftSetup ds;
-        ds.batch = 1; ds.B = c.block_B; ds.FR = N; ds.H = c.hidden; ds.d = c.head_dim; ds.theta = c.rope_theta;
+        DraftSetup ds{};
+        ds.batch = 1; ds.B = c.block_B; ds.FR = N; ds.d = c.head_dim; ds.theta = c.rope_theta;
         ds.seq_len = seqs->seq_len + seq; ds.root = seqs->root + seq; ds.feat = ws.hidden_tmp; ds.feat_count = nullptr;
         ds.count_const = n; ds.n_block = 0; ds.embed = ctx->embed; ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
-        ds.vocab = c.vocab; ds.capacity = c.max_pages_per_seq * kPage; ds.x = ws.x; ds.meta = meta_of(ctx);
-        ds.status = ws.status;
-        LAUNCH(ctx, KIND_OTHER, launch_setup_draft(ds, st));
-        LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, nullptr, 0, 0, c.hidden, N, c.hidden, (const bf16 *)ctx->head.ctx_norm, nullptr, N,
-                                c.rms_eps, ws.xn, nullptr, st));
+        ds.gain_block = (const bf16 *)ctx->head.ln1; ds.gain_feat = (const bf16 *)ctx->head.ctx_norm;
+        ds.vocab = c.vocab; ds.capacity = c.max_pages_per_seq * kPage; ds.geom = tg; ds.page_table = pt;
+        ds.out = rowout_of(ctx); ds.meta = meta_of(ctx); ds.status = ws.status;
+        LAUNCH(ctx, KIND_SETUP, launch_setup_draft(ds, st));
         LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
                   (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
         PassInfo hp{N, 0, 1, N, nullptr, seqs, seq};
         run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, hp, nullptr, nullptr);
-        LAUNCH(ctx, KIND_OTHER, launch_prefill_advance(seqs->seq_len + seq, seqs->root + seq, seqs->feat_count + seq,
-                                           last ? ws.argmax_tmp : nullptr, n, st));
+        LAUNCH(ctx, KIND_CONTROL, launch_prefill_advance(seqs->seq_len + seq, seqs->root + seq, seqs->feat_count + seq,
+                                                         last ? ws.argmax_tmp : nullptr, n, st));
     }
     return finish(ctx);
 }
@@ -453,7 +478,7 @@ int32_t glance_seq_truncate(glance_ctx *ctx, const glance_seqs *seqs, int32_t se
     if (rc) return rc;
     if (seq < 0 || seq >= seqs->batch || new_len < 0 || new_root < 0 || new_root >= ctx->cfg.vocab)
         return GLANCE_E_INVALID_ARG;
-    LAUNCH(ctx, KIND_OTHER, (set_seq_kernel<<<1, 1, 0, ctx->stream>>>(seqs->seq_len + seq, seqs->root + seq, new_len, new_root)));
+    LAUNCH(ctx, KIND_CONTROL, (set_seq_kernel<<<1, 1, 0, ctx->stream>>>(seqs->seq_len + seq, seqs->root + seq, new_len, new_root)));
     return finish(ctx);
 }
 
@@ -467,27 +492,32 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
     cudaStream_t st = ctx->stream;
     const int batch = seqs->batch, B = c.block_B;
     const int R1 = batch * B, R = 2 * R1;
-    DraftSetup ds;
-    ds.batch = batch; ds.B = B; ds.FR = B; ds.H = c.hidden; ds.d = c.head_dim; ds.theta = c.rope_theta;
+    DraftSetup ds{};
+    ds.batch = batch; ds.B = B; ds.FR = B; ds.d = c.head_dim; ds.theta = c.rope_theta;
     ds.seq_len = seqs->seq_len; ds.root = seqs->root; ds.feat = (const bf16 *)seqs->feat;
     ds.feat_count = seqs->feat_count; ds.count_const = 0; ds.n_block = B; ds.embed = ctx->embed;
-    ds.mask_embed = (const bf16 *)ctx->head.mask_embed; ds.vocab = c.vocab;
-    ds.capacity = c.max_pages_per_seq * kPage; ds.x = ws.x; ds.meta = meta_of(ctx); ds.status = ws.status;
-    LAUNCH(ctx, KIND_OTHER, launch_setup_draft(ds, st));
+    ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
     // block rows use the head's input norm, feature rows the context norm
-    LAUNCH(ctx, KIND_NORM, launch_norm(ws.x, nullptr, 0, 0, c.hidden, R, c.hidden, (const bf16 *)ctx->head.ln1,
-                            (const bf16 *)ctx->head.ctx_norm, R1, c.rms_eps, ws.xn, nullptr, st));
+    ds.gain_block = (const bf16 *)ctx->head.ln1; ds.gain_feat = (const bf16 *)ctx->head.ctx_norm; ds.vocab = c.vocab;
+    ds.capacity = c.max_pages_per_seq * kPage; ds.geom = geom_of(ctx, seqs); ds.page_table = seqs->page_table;
+    ds.out = rowout_of(ctx); ds.meta = meta_of(ctx); ds.status = ws.status;
+    LAUNCH(ctx, KIND_SETUP, launch_setup_draft(ds, st));
     LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
               (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
     PassInfo ps{R, R1, batch, B, nullptr, seqs, 0};
     run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, ps, (const bf16 *)ctx->head.final_norm, nullptr);
     float *logits = logits_dbg ? logits_dbg : ws.logits;
-    gemm(ctx, 0, ctx->lm_head, ws.xn, ctx->dims.Rmax, c.vocab, c.hidden, R1, 1, logits, c.vocab, 0, nullptr, nullptr);
+    {
+        TcGemmArgs g{};
+        g.Nout = c.vocab; g.K = c.hidden; g.R = R1; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.split_stride = 0;
+        with_row_scales(ctx, g);
+        gemm(ctx, 0, ctx->lm_head, ws.xn, ctx->dims.Rmax, g);
+    }
     {
         const bool prof = prof_begin(ctx);
         launch_topk(logits, batch, B, c.vocab, c.topk, topk_ids, topk_lp, ws.topk_cand, ws.topk_ml, st);
         ctx->launches++;                              // two kernels
-        prof_end(ctx, prof, KIND_OTHER, 0.0);
+        prof_end(ctx, prof, KIND_CONTROL, 0.0);
     }
     return finish(ctx);
 }
@@ -499,7 +529,7 @@ int32_t glance_build_tree(glance_ctx *ctx, int32_t batch, const int32_t *root, c
     if (!out->token || !out->parent || !out->depth || !out->rank || !out->score || !out->anc || !out->n_nodes)
         return GLANCE_E_INVALID_ARG;
     const glance_config &c = ctx->cfg;
-    LAUNCH(ctx, KIND_OTHER, launch_build_tree(batch, c.tree_N, c.block_B - 1, c.topk, root, topk_ids, topk_lp, *out, ctx->stream));
+    LAUNCH(ctx, KIND_CONTROL, launch_build_tree(batch, c.tree_N, c.block_B - 1, c.topk, root, topk_ids, topk_lp, *out, ctx->stream));
     return finish(ctx);
 }
 
@@ -511,12 +541,13 @@ int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glanc
     const glance_config &c = ctx->cfg;
     Workspace &ws = ctx->ws;
     const int batch = seqs->batch, N = c.tree_N;
-    VerifySetup vs;
-    vs.batch = batch; vs.N = N; vs.H = c.hidden; vs.d = c.head_dim; vs.theta = c.rope_theta;
+    VerifySetup vs{};
+    vs.batch = batch; vs.N = N; vs.d = c.head_dim; vs.theta = c.rope_theta;
     vs.seq_len = seqs->seq_len; vs.token = tree->token; vs.depth = tree->depth; vs.row_embeds = nullptr;
-    vs.row_ids = nullptr; vs.count = 0; vs.chain_anc = nullptr; vs.embed = ctx->embed; vs.vocab = c.vocab;
-    vs.capacity = c.max_pages_per_seq * kPage; vs.x = ws.x; vs.meta = meta_of(ctx); vs.status = ws.status;
-    LAUNCH(ctx, KIND_OTHER, launch_setup_verify(vs, ctx->stream));
+    vs.row_ids = nullptr; vs.count = 0; vs.chain_anc = nullptr; vs.embed = ctx->embed; vs.gain = ctx->ln1[0];
+    vs.vocab = c.vocab; vs.capacity = c.max_pages_per_seq * kPage; vs.geom = geom_of(ctx, seqs);
+    vs.page_table = seqs->page_table; vs.out = rowout_of(ctx); vs.meta = meta_of(ctx); vs.status = ws.status;
+    LAUNCH(ctx, KIND_SETUP, launch_setup_verify(vs, ctx->stream));
     PassInfo ps{batch * N, batch * N, batch, N, tree->anc, seqs, 0};
     run_target(ctx, ps, (bf16 *)hidden, logits_dbg, argmax);
     return finish(ctx);
@@ -529,7 +560,7 @@ static int32_t commit_common(glance_ctx *ctx, const glance_seqs *seqs, WalkCommi
     wc.page_table = seqs->page_table; wc.seq_len = seqs->seq_len; wc.root = seqs->root;
     wc.feat_count = seqs->feat_count; wc.feat = (bf16 *)seqs->feat; wc.counters = ctx->ws.walk_ctr;
     wc.status = ctx->ws.status;
-    LAUNCH(ctx, KIND_OTHER, launch_walk_commit(wc, ctx->stream));
+    LAUNCH(ctx, KIND_CONTROL, launch_walk_commit(wc, ctx->stream));
     return finish(ctx);
 }
 
@@ -590,7 +621,10 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
     if (!ctx || !W || !X || mode < 0 || mode > 2) return GLANCE_E_INVALID_ARG;
     if (Nout < 1 || K < 64 || K % 64 || R < 1 || R > ctx->dims.Rlog || S < 1 || S > 16) return GLANCE_E_INVALID_ARG;
     if ((mode == 0 && !Y) || (mode == 1 && (!act || Nout % 2)) || (mode == 2 && !argmax)) return GLANCE_E_INVALID_ARG;
-    gemm(ctx, mode, (const bf16 *)W, (const bf16 *)X, R, Nout, K, R, S, Y, Nout, (size_t)R * Nout, (bf16 *)act, argmax);
+    TcGemmArgs g{};
+    g.Nout = Nout; g.K = K; g.R = R; g.S = mode == 0 ? S : 1; g.Y = Y; g.ldy = Nout; g.split_stride = (size_t)R * Nout;
+    g.act = (bf16 *)act; g.F = Nout / 2; g.argmax = argmax;
+    gemm(ctx, mode, (const bf16 *)W, (const bf16 *)X, R, g);
     ctx->maps.clear();          // the hook's operands are transient: do not keep their descriptors
     return finish(ctx);
 }

@@ -5,9 +5,18 @@
 namespace glance {
 
 // ---- setup (kernels_small.cu) -------------------------------------------------------------
+// what a setup kernel emits per row besides the bookkeeping: fp32 residual x, bf16 x * gain, sum of squares
+struct RowOut {
+    int H;
+    float *x;            // [R][H]
+    bf16 *xb;            // [R][H]
+    float *ssq;          // [n_ssq][ssq_stride]: plane 0 gets the row's full sum of squares, the others 0
+    int n_ssq, ssq_stride;
+};
+
 struct VerifySetup {
     // rows r = s*N + i
-    int batch, N, H, d;
+    int batch, N, d;
     float theta;
     const int32_t *seq_len;     // [batch]
     const int32_t *token;       // [batch][N] tree tokens (mode tree) or nullptr
@@ -17,9 +26,12 @@ struct VerifySetup {
     int count;                  // prefill: valid rows
     uint64_t *chain_anc;        // prefill: [N][W] written with the causal chain mask
     const bf16 *embed;          // [V][H]
+    const bf16 *gain;           // first norm's gain
     int vocab;
     int capacity;               // max_pages_per_seq * page
-    float *x;                   // [R][H] fp32 residual stream (out)
+    KvGeom geom;
+    const int32_t *page_table;  // [batch][max_pages_per_seq]
+    RowOut out;
     RowMeta meta;
     int32_t *status;
 };
@@ -27,7 +39,7 @@ void launch_setup_verify(const VerifySetup &p, cudaStream_t st);
 
 struct DraftSetup {
     // block rows r = s*B + j (R1 = batch*n_block rows), then feature rows r = R1 + s*FR + i
-    int batch, B, FR, H, d;
+    int batch, B, FR, d;
     float theta;
     const int32_t *seq_len, *root;
     const bf16 *feat;           // [batch][FR][H]: FR = B (round) or tree_N (prefill head-context update)
@@ -35,36 +47,16 @@ struct DraftSetup {
     int count_const;
     int n_block;                // B (round) or 0 (prefill: only feature rows)
     const bf16 *embed, *mask_embed;
+    const bf16 *gain_block, *gain_feat;   // head input norm / context norm
     int vocab;
     int capacity;
-    float *x;
+    KvGeom geom;
+    const int32_t *page_table;
+    RowOut out;
     RowMeta meta;
     int32_t *status;
 };
 void launch_setup_draft(const DraftSetup &p, cudaStream_t st);
-
-// ---- reductions / elementwise (kernels_small.cu) -----------------------------------------
-// x[r] += sum_s part[s][r][0..H) (fixed order); optional hidden_out = bf16(x); xn = bf16(rms(x) * gain)
-// rows >= split_row use gain_b.
-void launch_norm(float *x, const float *part, int S, size_t part_split_stride, int ldp, int R, int H,
-                 const bf16 *gain_a, const bf16 *gain_b, int split_row, float eps, bf16 *xn, bf16 *hidden_out,
-                 cudaStream_t st);
-
-struct RopeKv {
-    int R, Rq;                  // rows in the pass; rows < Rq also emit q
-    int Hq, Hkv, d;
-    const float *part;          // [S][Rld][ldy] QKV partial sums
-    int S;
-    size_t split_stride;
-    int ldy;
-    RowMeta meta;
-    bf16 *q;                    // [Rq][Hq*d]
-    bf16 *pool_layer;           // base of this layer's pages
-    KvGeom geom;
-    const int32_t *page_table;  // [batch][max_pages_per_seq]
-    int32_t *status;
-};
-void launch_rope_kv(const RopeKv &p, cudaStream_t st);
 
 // rows (s, j), j = 1..L of logits [batch*B][V] -> ids/lp [batch][L][k]; scratch: cand [rows][topk_warps(V)][k],
 // ml [rows][topk_warps(V)][2].  Two launches.

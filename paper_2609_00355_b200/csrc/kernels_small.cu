@@ -4,7 +4,11 @@
 namespace glance {
 
 // ------------------------------------------------------------------------------------------
-// rotary table of one row: angle = pos * theta^(-2i/d), evaluated in double (one row per block)
+// Row setup shared by the verify and draft passes.  One block per row:
+//   * rotary table of the row: angle = pos * theta^(-2i/d), evaluated in double
+//   * element offset of the row's K slot (kv head 0) inside a layer of the paged pool
+//   * fp32 residual row x, its bf16 copy scaled by the first norm's gain, and its sum of squares
+//     (the consumer GEMM multiplies its results by 1/rms, so no separate normalisation pass exists)
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void fill_rope_row(const RowMeta &m, int r, int pos, int d, float theta) {
     const int half = d >> 1;
@@ -17,10 +21,41 @@ __device__ __forceinline__ void fill_rope_row(const RowMeta &m, int r, int pos, 
     }
 }
 
+__device__ __forceinline__ long long kv_row_offset(const KvGeom &g, const int32_t *page_table, int s, int slot_pos,
+                                                   int32_t *status) {
+    if (slot_pos < 0) return -1;
+    const int pg = slot_pos / kPage;
+    if (pg >= g.max_pages_per_seq) { set_status(status, GLANCE_E_BOUNDS); return -1; }
+    const int page = page_table[(size_t)s * g.max_pages_per_seq + pg];
+    if (page < 0 || page >= g.n_pages) { set_status(status, GLANCE_E_BOUNDS); return -1; }
+    return (long long)g.row(page, 0, 0, slot_pos % kPage);
+}
+
+// x[c] = src[c] (or 0), xb[c] = bf16(x[c] * gain[c]), ssq[0][r] = sum x^2, ssq[i>0][r] = 0
+__device__ __forceinline__ void emit_row(const RowOut &o, int r, const bf16 *src, const bf16 *gain) {
+    __shared__ float red[4];
+    float *x = o.x + (size_t)r * o.H;
+    bf16 *xb = o.xb + (size_t)r * o.H;
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < o.H; c += blockDim.x) {
+        const float v = src ? __bfloat162float(src[c]) : 0.f;
+        x[c] = v;
+        xb[c] = __float2bfloat16(v * __bfloat162float(gain[c]));
+        ss += v * v;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        o.ssq[r] = ((red[0] + red[1]) + red[2]) + red[3];
+        for (int i = 1; i < o.n_ssq; ++i) o.ssq[(size_t)i * o.ssq_stride + r] = 0.f;
+    }
+}
+
 // Verify-pass rows (Algorithm 1 line 3: pack the root and the tree).  Row r = s*N + i is node i of
 // sequence s at rotary position P + depth[i]; its K/V go to cache row P + i.  In prefill mode the rows are
 // a causal chain of `count` given embeddings / token ids and the chain's ancestor mask is emitted.
-__global__ void setup_verify_kernel(VerifySetup p) {
+__global__ void __launch_bounds__(128) setup_verify_kernel(VerifySetup p) {
     const int r = blockIdx.x;
     const int s = r / p.N, i = r % p.N;
     const int P = p.seq_len[s];
@@ -31,18 +66,17 @@ __global__ void setup_verify_kernel(VerifySetup p) {
         if (P < 0 || P + p.N > p.capacity) set_status(p.status, GLANCE_E_CAPACITY);
         p.meta.seq[r] = s;
         p.meta.pos[r] = P + depth;
-        p.meta.kvslot[r] = P + i;
+        p.meta.kvrow[r] = (P >= 0) ? kv_row_offset(p.geom, p.page_table, s, P + i, p.status) : -1;
     }
     fill_rope_row(p.meta, r, P + depth, p.d, p.theta);
-    float *x = p.x + (size_t)r * p.H;
     const bf16 *src = nullptr;
     if (prefill) {
         if (i < p.count) {
-            if (p.row_embeds) src = p.row_embeds + (size_t)i * p.H;
+            if (p.row_embeds) src = p.row_embeds + (size_t)i * p.out.H;
             else {
                 int t = p.row_ids[i];
                 if (t < 0 || t >= p.vocab) { t = 0; if (threadIdx.x == 0) set_status(p.status, GLANCE_E_BOUNDS); }
-                src = p.embed + (size_t)t * p.H;
+                src = p.embed + (size_t)t * p.out.H;
             }
         }
         // causal chain mask: row i sees rows 0..i
@@ -58,9 +92,9 @@ __global__ void setup_verify_kernel(VerifySetup p) {
     } else {
         int t = p.token[r];
         if (t < 0 || t >= p.vocab) { t = 0; if (threadIdx.x == 0) set_status(p.status, GLANCE_E_BOUNDS); }
-        src = p.embed + (size_t)t * p.H;
+        src = p.embed + (size_t)t * p.out.H;
     }
-    for (int c = threadIdx.x; c < p.H; c += blockDim.x) x[c] = src ? __bfloat162float(src[c]) : 0.f;
+    emit_row(p.out, r, src, p.gain);
 }
 
 void launch_setup_verify(const VerifySetup &p, cudaStream_t st) {
@@ -70,10 +104,9 @@ void launch_setup_verify(const VerifySetup &p, cudaStream_t st) {
 // Draft-pass rows (Algorithm 1 line 1; Section 3.2).  Block rows: slot 0 = E[root], slots 1..B-1 = mask
 // embedding, position P + j.  Feature rows: target features of the positions committed last, whose K/V
 // become head context at positions P - count .. P - 1 (or P .. P+count-1 while prefilling).
-__global__ void setup_draft_kernel(DraftSetup p) {
+__global__ void __launch_bounds__(128) setup_draft_kernel(DraftSetup p) {
     const int r = blockIdx.x;
     const int R1 = p.batch * p.n_block;
-    float *x = p.x + (size_t)r * p.H;
     const bf16 *src = nullptr;
     int s, pos, slot;
     if (r < R1) {
@@ -82,11 +115,11 @@ __global__ void setup_draft_kernel(DraftSetup p) {
         const int P = p.seq_len[s];
         if (threadIdx.x == 0 && (P < 0 || P + p.B > p.capacity)) set_status(p.status, GLANCE_E_CAPACITY);
         pos = P + j;
-        slot = P + j;
+        slot = P >= 0 ? P + j : -1;
         if (j == 0) {
             int t = p.root[s];
             if (t < 0 || t >= p.vocab) { t = 0; if (threadIdx.x == 0) set_status(p.status, GLANCE_E_BOUNDS); }
-            src = p.embed + (size_t)t * p.H;
+            src = p.embed + (size_t)t * p.out.H;
         } else {
             src = p.mask_embed;
         }
@@ -102,7 +135,7 @@ __global__ void setup_draft_kernel(DraftSetup p) {
         if (i < cnt) {
             pos = base + i;
             slot = base + i;
-            src = p.feat + ((size_t)s * p.FR + i) * p.H;
+            src = p.feat + ((size_t)s * p.FR + i) * p.out.H;
         } else {
             pos = 0;
             slot = -1;
@@ -111,132 +144,15 @@ __global__ void setup_draft_kernel(DraftSetup p) {
     if (threadIdx.x == 0) {
         p.meta.seq[r] = s;
         p.meta.pos[r] = pos;
-        p.meta.kvslot[r] = slot;
+        p.meta.kvrow[r] = kv_row_offset(p.geom, p.page_table, s, slot, p.status);
     }
     fill_rope_row(p.meta, r, pos, p.d, p.theta);
-    for (int c = threadIdx.x; c < p.H; c += blockDim.x) x[c] = src ? __bfloat162float(src[c]) : 0.f;
+    emit_row(p.out, r, src, r < R1 ? p.gain_block : p.gain_feat);
 }
 
 void launch_setup_draft(const DraftSetup &p, cudaStream_t st) {
     const int R = p.batch * p.n_block + p.batch * p.FR;
     setup_draft_kernel<<<R, 128, 0, st>>>(p);
-}
-
-// ------------------------------------------------------------------------------------------
-// residual add (split-K partials, fixed order) + RMSNorm -> bf16
-// ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) norm_kernel(float *x, const float *part, int S, size_t split_stride, int ldp,
-                                                    int H, const bf16 *gain_a, const bf16 *gain_b, int split_row,
-                                                    float eps, bf16 *xn, bf16 *hidden_out) {
-    extern __shared__ float4 row4[];
-    __shared__ float red[32];
-    const int r = blockIdx.x;
-    const int H4 = H >> 2;
-    float4 *xr = reinterpret_cast<float4 *>(x + (size_t)r * H);
-    float ss = 0.f;
-    for (int c = threadIdx.x; c < H4; c += blockDim.x) {
-        float4 v = xr[c];
-        for (int s = 0; s < S; ++s) {
-            const float4 p = __ldcg(reinterpret_cast<const float4 *>(part + s * split_stride + (size_t)r * ldp) + c);
-            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-        }
-        row4[c] = v;
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        if (S > 0) xr[c] = v;
-        if (hidden_out) {
-            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-            uint2 o;
-            o.x = *reinterpret_cast<uint32_t *>(&lo);
-            o.y = *reinterpret_cast<uint32_t *>(&hi);
-            reinterpret_cast<uint2 *>(hidden_out + (size_t)r * H)[c] = o;
-        }
-    }
-    ss = warp_sum(ss);
-    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
-    __syncthreads();
-    float tot = 0.f;
-    const int nw = (blockDim.x + 31) >> 5;
-    for (int w = 0; w < nw; ++w) tot += red[w];
-    const float inv = rsqrtf(tot / (float)H + eps);
-    const bf16 *g = (r >= split_row) ? gain_b : gain_a;
-    if (xn)
-        for (int c = threadIdx.x; c < H4; c += blockDim.x) {
-            const float4 v = row4[c];
-            const uint2 gg = reinterpret_cast<const uint2 *>(g)[c];
-            const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x);
-            const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
-            __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv * __low2float(g01), v.y * inv * __high2float(g01));
-            __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv * __low2float(g23), v.w * inv * __high2float(g23));
-            uint2 o;
-            o.x = *reinterpret_cast<uint32_t *>(&lo);
-            o.y = *reinterpret_cast<uint32_t *>(&hi);
-            reinterpret_cast<uint2 *>(xn + (size_t)r * H)[c] = o;
-        }
-}
-
-void launch_norm(float *x, const float *part, int S, size_t part_split_stride, int ldp, int R, int H,
-                 const bf16 *gain_a, const bf16 *gain_b, int split_row, float eps, bf16 *xn, bf16 *hidden_out,
-                 cudaStream_t st) {
-    int threads = ((H / 4) + 31) / 32 * 32;
-    threads = threads > 1024 ? 1024 : threads;
-    norm_kernel<<<R, threads, H * sizeof(float), st>>>(x, part, S, part_split_stride, ldp, H, gain_a,
-                                                       gain_b ? gain_b : gain_a, split_row, eps, xn, hidden_out);
-}
-
-// ------------------------------------------------------------------------------------------
-// QKV split-K reduction + rotary (pairs (i, i + d/2)) + paged K/V write
-// ------------------------------------------------------------------------------------------
-__global__ void rope_kv_kernel(RopeKv p) {
-    // grid (R, Hq + 2 Hkv): one block per (row, head); heads are ordered q..., k..., v...
-    const int r = blockIdx.x, h = blockIdx.y;
-    const int half = p.d >> 1;
-    const bool is_q = h < p.Hq, is_k = !is_q && h < p.Hq + p.Hkv;
-    if (is_q && r >= p.Rq) return;
-    const int slot_pos = p.meta.kvslot[r];
-    bf16 *dst = nullptr;
-    if (is_q) {
-        dst = p.q + ((size_t)r * p.Hq + h) * p.d;
-    } else {
-        if (slot_pos < 0) return;
-        const int s = p.meta.seq[r];
-        const int pg = slot_pos / kPage;
-        bool ok = pg < p.geom.max_pages_per_seq;
-        int page = ok ? p.page_table[(size_t)s * p.geom.max_pages_per_seq + pg] : 0;
-        if (page < 0 || page >= p.geom.n_pages) ok = false;
-        if (!ok) {
-            if (threadIdx.x == 0) set_status(p.status, GLANCE_E_BOUNDS);
-            return;
-        }
-        const int kvh = is_k ? h - p.Hq : h - p.Hq - p.Hkv;
-        dst = p.pool_layer + p.geom.row(page, is_k ? 0 : 1, kvh, slot_pos % kPage);
-    }
-    const int col0 = h * p.d;
-    const float *y = p.part + (size_t)r * p.ldy + col0;
-    if (is_q || is_k) {
-        const float *cs = p.meta.rope_cos + (size_t)r * half;
-        const float *sn = p.meta.rope_sin + (size_t)r * half;
-        for (int i = threadIdx.x; i < half; i += blockDim.x) {
-            float a = 0.f, b = 0.f;
-            for (int sp = 0; sp < p.S; ++sp) {
-                a += __ldcg(y + sp * p.split_stride + i);
-                b += __ldcg(y + sp * p.split_stride + i + half);
-            }
-            const float c = cs[i], sv = sn[i];
-            dst[i] = __float2bfloat16(a * c - b * sv);
-            dst[i + half] = __float2bfloat16(b * c + a * sv);
-        }
-    } else {
-        for (int i = threadIdx.x; i < p.d; i += blockDim.x) {
-            float a = 0.f;
-            for (int sp = 0; sp < p.S; ++sp) a += __ldcg(y + sp * p.split_stride + i);
-            dst[i] = __float2bfloat16(a);
-        }
-    }
-}
-
-void launch_rope_kv(const RopeKv &p, cudaStream_t st) {
-    dim3 grid(p.R, p.Hq + 2 * p.Hkv);
-    rope_kv_kernel<<<grid, 64, 0, st>>>(p);
 }
 
 // ------------------------------------------------------------------------------------------
