@@ -176,6 +176,12 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
 int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const void *X, float *Y, void *act,
                              int32_t *argmax, int32_t Nout, int32_t K, int32_t R, int32_t S);
 
+/* Test hook: phase timestamps of the GEMM kernel.  While a buffer (device, slots x 16 uint64) is set, the
+ * n-th GEMM launch after this call makes its first CTA write nanosecond timestamps (entry, set-up done,
+ * predecessor finished, first tile landed, accumulator ready, cluster barrier 1, tile shipped, cluster
+ * barrier 2, epilogue done, exit) into slot n % slots.  buffer = NULL, slots = 0 switches it off. */
+int32_t glance_debug_trace(glance_ctx *ctx, uint64_t *buffer, int32_t slots);
+
 /* Measurement aid.  While enabled, every kernel launch is bracketed by a pair of CUDA events on the context's
  * stream (the pairs are created when profiling is first enabled, so the round calls still allocate nothing).
  * glance_profile_read synchronises the stream and fills three arrays of GLANCE_PROFILE_KINDS entries, indexed by

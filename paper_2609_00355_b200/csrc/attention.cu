@@ -84,6 +84,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_kernel(AttnParams p) {
     __shared__ int sh_pages[PAGE_CACHE];
     __shared__ int sh_last;
 
+    // programmatic dependent launch: let the next kernel begin its prologue now; this kernel reads data of
+    // its predecessors, so it waits for them before touching global memory
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int G = p.Hq / p.Hkv;
     const int PR = p.T * G;
     const int qt = blockIdx.x, kvh = blockIdx.y;
@@ -392,6 +396,20 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_kernel(AttnParams p) {
     if (tid == 0) *ctr = 0;
 }
 
+void launch_pdl(void (*kernel)(AttnParams), dim3 grid, size_t smem, cudaStream_t st, const AttnParams &p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(NTHREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 }  // namespace
 
 int attention_q_tiles(int T, int G) { return (T * G + QT - 1) / QT; }
@@ -411,14 +429,14 @@ void launch_attention(const AttnParams &p, cudaStream_t st) {
             cudaFuncSetAttribute(attn_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<128>::TOTAL);
             once = true;
         }
-        attn_kernel<128><<<grid, NTHREADS, Smem<128>::TOTAL, st>>>(p);
+        launch_pdl(attn_kernel<128>, grid, Smem<128>::TOTAL, st, p);
     } else {
         static bool once = false;
         if (!once) {
             cudaFuncSetAttribute(attn_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<64>::TOTAL);
             once = true;
         }
-        attn_kernel<64><<<grid, NTHREADS, Smem<64>::TOTAL, st>>>(p);
+        launch_pdl(attn_kernel<64>, grid, Smem<64>::TOTAL, st, p);
     }
 }
 

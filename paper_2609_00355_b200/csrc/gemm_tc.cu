@@ -9,7 +9,7 @@
 // epilogue warps (one TMEM lane = one output feature).
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
-// Epilogues: (0) fp32 split-K plane, (1) SwiGLU over a gate tile and its up tile (two accumulators),
+// Epilogues: (0) fp32 split-K plane, (1) SwiGLU over 64 gate rows and their 64 up rows stacked into one tile,
 // (2) row-wise arg-max over the vocabulary, merged across CTAs with a packed 64-bit atomic max,
 // (3)/(4) split-K reduced inside a thread-block cluster through distributed shared memory, followed by
 // residual add + norm statistics, or rotary embedding + paged K/V write.
@@ -117,6 +117,11 @@ struct alignas(8) Barriers {
     int abort_flag;
 };
 
+// Programmatic dependent launch: the next kernel of the stream may start its prologue (and prefetch weights)
+// while this one is still running; a kernel touches data written by its predecessors only after pdl_wait().
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void cluster_sync_all() {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
@@ -135,28 +140,27 @@ __device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 
-// MODE 0: fp32 planes              MODE 1: SwiGLU (two accumulators)      MODE 2: arg-max (+ optional logits)
+// MODE 0: fp32 planes              MODE 1: SwiGLU (64 gate + 64 up rows per tile)   MODE 2: arg-max (+ optional logits)
 // MODE 3: split-K over a cluster, residual add + bf16 copy scaled by the next norm's gain + sum of squares
 // MODE 4: split-K over a cluster, rotary embedding + q / paged K,V write
 // Modes 0, 1, 2 and 4 multiply each activation row's results by 1/rms(row) when a.ssq is given: the rows
 // they read are x * gain in bf16, and the row's sum of squares arrives as per-tile partial sums.
 template <int MODE>
-__global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+__global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                          const __grid_constant__ CUtensorMap map_x, TcGemmArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     __shared__ Barriers bars;
-    __shared__ unsigned long long red_keys[4][128];
     __shared__ float inv_rms[128];
-    __shared__ float red_sq[4][128];
 
-    constexpr int NW = (MODE == 1) ? 2 : 1;              // weight tiles per stage
+    // MODE 1 stacks 64 gate rows and the matching 64 up rows into one 128-row weight tile (two TMA boxes)
+    constexpr int FT = (MODE == 1) ? 64 : BM;            // output features per CTA
     constexpr bool CLUSTERED = (MODE >= 3);
     const int NP = a.np;                                 // UMMA N (activation rows, padded to 16)
-    const int stage_bytes = NW * BM * 128 + NP * 128;
+    const int stage_bytes = BM * 128 + NP * 128;
     const int stages = a.stages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int f0 = blockIdx.x * BM;
+    const int f0 = blockIdx.x * FT;
     const int split = blockIdx.y;
     const int r0 = blockIdx.z * 128;
     const int ktiles = a.K / BK;
@@ -164,6 +168,10 @@ __global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const
     const int nk = kt1 - kt0;
     const uint32_t tmem_cols = a.tmem_cols;
 
+    // optional phase timestamps of CTA (0,0,0) (test hook; a.trace is nullptr in normal use)
+    unsigned long long *trace = (a.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? a.trace : nullptr;
+    if (trace && threadIdx.x == 0) trace[0] = global_ns();
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(&bars.full[s], 1);
@@ -183,23 +191,41 @@ __global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const
     const uint32_t tmem_base = bars.tmem_base;
     volatile int *abort_flag = &bars.abort_flag;
     bool ok = true;                                      // epilogue warps: accumulator is valid
+    if (trace && threadIdx.x == 0) trace[1] = global_ns();
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
-            int issued = 0;
-            for (int i = 0; i < nk; ++i) {
+            auto load_w = [&](int i, unsigned char *slot, uint64_t *bar) {
+                const int k0 = (kt0 + i) * BK;
+                if (MODE == 1) {
+                    tma_load_2d(slot, &map_w, bar, k0, f0);                       // gate rows
+                    tma_load_2d(slot + 64 * 128, &map_w, bar, k0, a.F + f0);     // up rows
+                } else {
+                    tma_load_2d(slot, &map_w, bar, k0, f0);
+                }
+            };
+            // weights do not depend on earlier kernels: fill the ring with them before waiting on the predecessor
+            const int pre = min(nk, stages);
+            for (int i = 0; i < pre; ++i) {
+                mbar_expect_tx(&bars.full[i], (uint32_t)stage_bytes);
+                load_w(i, smem + (size_t)i * stage_bytes, &bars.full[i]);
+            }
+            pdl_wait();
+            if (trace) trace[2] = global_ns();
+            for (int i = 0; i < pre; ++i)
+                tma_load_2d(smem + (size_t)i * stage_bytes + BM * 128, &map_x, &bars.full[i], (kt0 + i) * BK, r0);
+            int issued = pre;
+            for (int i = pre; i < nk; ++i) {
                 const int s = i % stages;
                 const uint32_t ph = (uint32_t)(i / stages) & 1u;
                 if (!mbar_wait(&bars.empty[s], ph ^ 1u, abort_flag, a.status)) break;
                 unsigned char *slot = smem + (size_t)s * stage_bytes;
                 mbar_expect_tx(&bars.full[s], (uint32_t)stage_bytes);
-                const int k0 = (kt0 + i) * BK;
-                tma_load_2d(slot, &map_w, &bars.full[s], k0, f0);
-                if (NW == 2) tma_load_2d(slot + BM * 128, &map_w, &bars.full[s], k0, a.F + f0);
-                tma_load_2d(slot + NW * BM * 128, &map_x, &bars.full[s], k0, r0);
+                load_w(i, slot, &bars.full[s]);
+                tma_load_2d(slot + BM * 128, &map_x, &bars.full[s], (kt0 + i) * BK, r0);
                 issued = i + 1;
             }
             if (*abort_flag) {
@@ -220,17 +246,14 @@ __global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const
                 const int s = i % stages;
                 const uint32_t ph = (uint32_t)(i / stages) & 1u;
                 if (!mbar_wait(&bars.full[s], ph, abort_flag, a.status)) { mok = false; break; }
+                if (trace && i == 0) trace[3] = global_ns();
                 tc_fence_after();
                 const uint32_t slot = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint64_t bdesc = umma_desc(slot + NW * BM * 128);
+                const uint64_t bdesc = umma_desc(slot + BM * 128);
+                const uint64_t adesc = umma_desc(slot);
 #pragma unroll
-                for (int w = 0; w < NW; ++w) {
-                    const uint64_t adesc = umma_desc(slot + w * BM * 128);
-#pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        umma_f16(tmem_base + (uint32_t)(w * NP), adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc,
-                                 (i > 0 || k > 0) ? 1u : 0u);
-                }
+                for (int k = 0; k < BK / 16; ++k)
+                    umma_f16(tmem_base, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (i > 0 || k > 0) ? 1u : 0u);
                 umma_commit(&bars.empty[s]);             // slot reusable once these MMAs have read it
             }
             if (mok) umma_commit(&bars.acc_ready);
@@ -238,6 +261,7 @@ __global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const
     } else {
         // ---------------- epilogue warps, part 1: row scales, then wait for the accumulator ----------------
         const int t = threadIdx.x - 64;                  // 0..127
+        pdl_wait();                                      // everything below reads or writes data other kernels own
         if (MODE != 3) {
             float inv = 1.f;
             if (a.ssq && t < NP && r0 + t < a.R) {
@@ -247,182 +271,207 @@ __global__ void __launch_bounds__(192, (MODE >= 3) ? 2 : 1) gemm_tc_kernel(const
             }
             inv_rms[t] = inv;
         }
-        if (MODE == 2) red_keys[warp & 3][lane] = red_keys[warp & 3][lane + 32] = red_keys[warp & 3][lane + 64] = red_keys[warp & 3][lane + 96] = 0ull;
         if (nk > 0) ok = mbar_wait(&bars.acc_ready, 0, abort_flag, a.status);
         ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld is warp-collective: decide as a warp
         tc_fence_after();
         asm volatile("bar.sync 1, 128;" ::: "memory");   // inv_rms / red_keys visible to the four epilogue warps
+        if (trace && threadIdx.x == 64) trace[4] = global_ns();
     }
 
+    // ---------------- epilogue, part 2 ----------------
+    // (a) every epilogue thread owns one TMEM lane (= one output feature of the tile) and moves its NP fp32
+    //     results into a shared-memory tile laid out [row][feature] on top of the idle TMA ring -- its own
+    //     ring, or, with split-K over a cluster, the ring of the CTA that owns the row;
+    // (b) after a barrier the tile is processed one activation row per warp, four consecutive features per
+    //     thread, so that every shared and global access is a 16-byte (fp32) or 8-byte (bf16) vector.
     const int q = warp & 3;                              // TMEM lane quarter an epilogue warp may read
-    const int fl = q * 32 + lane;                        // feature within the tile
-    const int f = f0 + fl;
+    const int fl = q * 32 + lane;                        // feature within the tile (stage a)
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
-
-    if (!CLUSTERED) {
-        if (warp >= 2 && ok) {
-            for (int c = 0; c < NP; c += 16) {
-                uint32_t v[16];
-                if (nk > 0) {
-                    tmem_ld16(lane_addr + (uint32_t)c, v);
-                    tmem_ld_wait();
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0u;
-                }
-                if (MODE == 0) {
-                    float *Ys = a.Y + (size_t)split * a.split_stride;
-                    if (f < a.Nout) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int r = r0 + c + j;
-                            if (r < a.R) Ys[(size_t)r * a.ldy + f] = __uint_as_float(v[j]) * inv_rms[c + j];
-                        }
-                    }
-                } else if (MODE == 1) {
-                    uint32_t u[16];
-                    tmem_ld16(lane_addr + (uint32_t)(NP + c), u);
-                    tmem_ld_wait();
-                    if (f < a.F) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int r = r0 + c + j;
-                            const float g = __uint_as_float(v[j]) * inv_rms[c + j], up = __uint_as_float(u[j]) * inv_rms[c + j];
-                            if (r < a.R) a.act[(size_t)r * a.F + f] = __float2bfloat16(g / (1.f + __expf(-g)) * up);
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int r = r0 + c + j;
-                        const float val = __uint_as_float(v[j]) * inv_rms[c + j];
-                        if (a.Y && f < a.Nout && r < a.R) a.Y[(size_t)r * a.ldy + f] = val;
-                        unsigned long long key = (f < a.Nout) ? pack_val_id(val, f) : 0ull;
-                        key = warp_max_u64(key);
-                        if (lane == 0) red_keys[q][c + j] = key;
-                    }
-                }
-            }
-        }
-        if (MODE == 2 && warp >= 2) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            const int t = threadIdx.x - 64;
-            const int r = r0 + t;
-            if (ok && t < NP && r < a.R) {
-                unsigned long long k = red_keys[0][t];
-                for (int w = 1; w < 4; ++w) k = red_keys[w][t] > k ? red_keys[w][t] : k;
-                atomicMax(a.keys + r, k);
-            }
-        }
-    } else {
-        // ---------------- split-K over the cluster, reduce-scatter by rows: CTA `rank` owns activation rows
-        // [rank*RP, rank*RP + RP) of the tile.  Every CTA ships, for each row, its fp32 partial results to the
-        // owner's shared memory (planes [source split][row][feature], aliased onto the owner's idle TMA ring);
-        // the owner adds the planes in split order and applies the fused epilogue to its rows ----------------
-        const uint32_t rank = cluster_rank();
-        const int RP = (NP + a.S - 1) / a.S;             // rows per owner
+    const uint32_t rank = CLUSTERED ? cluster_rank() : 0u;
+    const int RP = CLUSTERED ? (NP + a.S - 1) / a.S : NP; // rows per owner CTA
+    if (CLUSTERED) {
         cluster_sync_all();                              // every CTA's MMAs are done: all rings are idle
-        if (warp >= 2) {
-            const uint32_t local = smem_u32(smem) + (uint32_t)((rank * RP) * BM * 4) + (uint32_t)(fl * 4);
-            for (int c = 0; c < NP; c += 16) {
-                uint32_t v[16];
-                if (nk > 0 && ok) {
-                    tmem_ld16(lane_addr + (uint32_t)c, v);
-                    tmem_ld_wait();
-                } else {
+        if (trace && threadIdx.x == 64) trace[5] = global_ns();
+    }
+    if (warp >= 2) {
+        const uint32_t local = smem_u32(smem) + (uint32_t)((rank * RP) * BM * 4) + (uint32_t)(fl * 4);
+        for (int c = 0; c < NP; c += 16) {
+            uint32_t v[16];
+            if (nk > 0 && ok) {
+                tmem_ld16(lane_addr + (uint32_t)c, v);
+                tmem_ld_wait();
+            } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0u;
-                }
+                for (int j = 0; j < 16; ++j) v[j] = 0u;
+            }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int r = c + j;
+            for (int j = 0; j < 16; ++j) {
+                const int r = c + j;
+                if (CLUSTERED) {
                     const uint32_t owner = (uint32_t)(r / RP);
                     st_cluster_f32(map_to_rank(local + (uint32_t)((r - owner * RP) * BM * 4), owner), __uint_as_float(v[j]));
-                }
-            }
-        }
-        cluster_sync_all();                              // planes written and visible
-        if (warp >= 2) {
-            const float *planes = reinterpret_cast<const float *>(smem);
-            const int row_lo = (int)rank * RP;                                   // first owned row (tile-local)
-            const int my_rows = max(0, min(min(RP, NP - row_lo), a.R - r0 - row_lo));
-            if (MODE == 3) {
-                const bool valid = f < a.Nout;
-                const float gain = valid ? __bfloat162float(a.gain[f]) : 0.f;
-                for (int rb = 0; rb < my_rows; rb += 8) {
-                    float xv[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        xv[j] = (valid && rb + j < my_rows) ? __ldcg(a.x + (size_t)(r0 + row_lo + rb + j) * a.Nout + f) : 0.f;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int lr = rb + j;
-                        if (lr >= my_rows) break;            // uniform across the warp
-                        float v = 0.f;
-                        for (int k = 0; k < a.S; ++k) v += planes[(size_t)(k * RP + lr) * BM + fl];
-                        float sq = 0.f;
-                        if (valid) {
-                            const size_t o = (size_t)(r0 + row_lo + lr) * a.Nout + f;
-                            const float xn = xv[j] + v;
-                            a.x[o] = xn;
-                            a.xb[o] = __float2bfloat16(xn * gain);
-                            if (a.hidden_out) a.hidden_out[o] = __float2bfloat16(xn);
-                            sq = xn * xn;
-                        }
-                        sq = warp_sum(sq);
-                        if (lane == 0) red_sq[q][lr] = sq;
-                    }
-                }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int t = threadIdx.x - 64;
-                if (t < my_rows)
-                    a.ssq_out[(size_t)blockIdx.x * a.ssq_stride + r0 + row_lo + t] =
-                        ((red_sq[0][t] + red_sq[1][t]) + red_sq[2][t]) + red_sq[3][t];
-            } else {
-                const int d = a.head_dim, half = d >> 1;
-                const int h = f / d, i = f % d;
-                const bool is_q = h < a.Hq, is_k = !is_q && h < a.Hq + a.Hkv, valid = f < a.Nout;
-                const int pfl = (i < half) ? fl + half : fl - half;          // rotary partner, same tile
-                const int ci = (i < half) ? i : i - half;
-                const int kvh = is_k ? h - a.Hq : h - a.Hq - a.Hkv;
-                for (int rb = 0; rb < my_rows; rb += 8) {
-                    float cs[8], sn[8];
-                    long long base[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int rr = r0 + row_lo + rb + j;
-                        const bool live = valid && rb + j < my_rows;
-                        cs[j] = (live && !(!is_q && !is_k)) ? a.rope_cos[(size_t)rr * half + ci] : 1.f;
-                        sn[j] = (live && !(!is_q && !is_k)) ? a.rope_sin[(size_t)rr * half + ci] : 0.f;
-                        base[j] = (live && !is_q) ? a.kvrow[rr] : -1;
-                    }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int lr = rb + j;
-                        if (lr >= my_rows) break;
-                        const int rr = r0 + row_lo + lr;
-                        float va = 0.f, vb = 0.f;
-                        for (int k = 0; k < a.S; ++k) {
-                            const float *pl = planes + (size_t)(k * RP + lr) * BM;
-                            va += pl[fl];
-                            vb += pl[pfl];
-                        }
-                        if (!valid) continue;
-                        va *= inv_rms[row_lo + lr];
-                        vb *= inv_rms[row_lo + lr];
-                        const float out = (is_q || is_k) ? ((i < half) ? va * cs[j] - vb * sn[j] : va * cs[j] + vb * sn[j]) : va;
-                        if (is_q) {
-                            if (rr < a.Rq) a.q[((size_t)rr * a.Hq + h) * d + i] = __float2bfloat16(out);
-                        } else if (base[j] >= 0) {
-                            a.pool_layer[(size_t)base[j] + (is_k ? 0 : a.v_off) + (size_t)kvh * a.head_stride + i] = __float2bfloat16(out);
-                        }
-                    }
+                } else {
+                    reinterpret_cast<float *>(smem)[r * BM + fl] = __uint_as_float(v[j]);
                 }
             }
         }
     }
+    if (CLUSTERED) {
+        if (trace && threadIdx.x == 64) trace[6] = global_ns();
+        cluster_sync_all();                              // planes written and visible
+        if (trace && threadIdx.x == 64) trace[7] = global_ns();
+    } else if (warp >= 2) {
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+    }
+    if (warp >= 2 && ok) {
+        const float *tile = reinterpret_cast<const float *>(smem);
+        const int ew = warp - 2;                         // epilogue warp 0..3
+        const int row_lo = (int)rank * RP;               // first owned row (tile-local)
+        const int my_rows = max(0, min(min(RP, NP - row_lo), a.R - r0 - row_lo));
+        const int fo = 4 * lane;                         // first of this thread's four features (tile-local)
+        if (MODE == 0 || MODE == 2) {
+            const bool vec = (a.ldy & 3) == 0;
+            for (int r = ew; r < my_rows; r += 4) {
+                const int rr = r0 + r;
+                float4 v = *reinterpret_cast<const float4 *>(tile + r * BM + fo);
+                const float sc = inv_rms[r];
+                v.x *= sc; v.y *= sc; v.z *= sc; v.w *= sc;
+                const int f = f0 + fo;
+                if (MODE == 0 || a.Y) {
+                    float *dst = a.Y + (MODE == 0 ? (size_t)split * a.split_stride : 0) + (size_t)rr * a.ldy + f;
+                    if (vec && f + 3 < a.Nout) *reinterpret_cast<float4 *>(dst) = v;
+                    else {
+                        if (f < a.Nout) dst[0] = v.x;
+                        if (f + 1 < a.Nout) dst[1] = v.y;
+                        if (f + 2 < a.Nout) dst[2] = v.z;
+                        if (f + 3 < a.Nout) dst[3] = v.w;
+                    }
+                }
+                if (MODE == 2) {
+                    unsigned long long key = 0ull, k2;
+                    if (f < a.Nout) key = pack_val_id(v.x, f);
+                    if (f + 1 < a.Nout) { k2 = pack_val_id(v.y, f + 1); key = k2 > key ? k2 : key; }
+                    if (f + 2 < a.Nout) { k2 = pack_val_id(v.z, f + 2); key = k2 > key ? k2 : key; }
+                    if (f + 3 < a.Nout) { k2 = pack_val_id(v.w, f + 3); key = k2 > key ? k2 : key; }
+                    key = warp_max_u64(key);
+                    if (lane == 0) atomicMax(a.keys + rr, key);
+                }
+            }
+        } else if (MODE == 1) {
+            // tile features 0..63 are gate rows, 64..127 the matching up rows; item = (row, 4 gate features)
+            const int t = threadIdx.x - 64;
+            for (int item = t; item < my_rows * 16; item += 128) {
+                const int r = item >> 4, fg = (item & 15) * 4;
+                const float4 g = *reinterpret_cast<const float4 *>(tile + r * BM + fg);
+                const float4 u = *reinterpret_cast<const float4 *>(tile + r * BM + 64 + fg);
+                const float sc = inv_rms[r];
+                const int f = f0 + fg;
+                if (f < a.F) {          // F is a multiple of 4
+                    const float g0 = g.x * sc, g1 = g.y * sc, g2 = g.z * sc, g3 = g.w * sc;
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * (u.x * sc), g1 / (1.f + __expf(-g1)) * (u.y * sc));
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(g2 / (1.f + __expf(-g2)) * (u.z * sc), g3 / (1.f + __expf(-g3)) * (u.w * sc));
+                    uint2 o;
+                    o.x = *reinterpret_cast<uint32_t *>(&lo);
+                    o.y = *reinterpret_cast<uint32_t *>(&hi);
+                    *reinterpret_cast<uint2 *>(a.act + (size_t)(r0 + r) * a.F + f) = o;
+                }
+            }
+        } else if (MODE == 3) {
+            const int f = f0 + fo;
+            const bool valid = f < a.Nout;               // Nout is a multiple of 4
+            float4 gain = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (valid) {
+                const uint2 gg = *reinterpret_cast<const uint2 *>(a.gain + f);
+                const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x);
+                const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
+                gain = make_float4(__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23));
+            }
+            for (int lr = ew; lr < my_rows; lr += 4) {
+                const size_t o = (size_t)(r0 + row_lo + lr) * a.Nout + f;
+                float4 xv = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (valid) xv = __ldcg(reinterpret_cast<const float4 *>(a.x + o));
+                float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int k = 0; k < a.S; ++k) {          // split order: bit-reproducible
+                    const float4 p = *reinterpret_cast<const float4 *>(tile + (size_t)(k * RP + lr) * BM + fo);
+                    v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+                }
+                float sq = 0.f;
+                if (valid) {
+                    xv.x += v.x; xv.y += v.y; xv.z += v.z; xv.w += v.w;
+                    *reinterpret_cast<float4 *>(a.x + o) = xv;
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(xv.x * gain.x, xv.y * gain.y);
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(xv.z * gain.z, xv.w * gain.w);
+                    uint2 ob;
+                    ob.x = *reinterpret_cast<uint32_t *>(&lo);
+                    ob.y = *reinterpret_cast<uint32_t *>(&hi);
+                    *reinterpret_cast<uint2 *>(a.xb + o) = ob;
+                    if (a.hidden_out) {
+                        lo = __floats2bfloat162_rn(xv.x, xv.y);
+                        hi = __floats2bfloat162_rn(xv.z, xv.w);
+                        ob.x = *reinterpret_cast<uint32_t *>(&lo);
+                        ob.y = *reinterpret_cast<uint32_t *>(&hi);
+                        *reinterpret_cast<uint2 *>(a.hidden_out + o) = ob;
+                    }
+                    sq = ((xv.x * xv.x + xv.y * xv.y) + xv.z * xv.z) + xv.w * xv.w;
+                }
+                sq = warp_sum(sq);                       // one warp spans the tile's 128 features
+                if (lane == 0) a.ssq_out[(size_t)blockIdx.x * a.ssq_stride + r0 + row_lo + lr] = sq;
+            }
+        } else {
+            // MODE 4: q heads, then k heads, then v heads; rotary pairs (i, i + d/2) lie in the same tile
+            const int d = a.head_dim, half = d >> 1;
+            const int f = f0 + fo;
+            const bool valid = f < a.Nout;
+            const int h = f / d, i = f % d;              // the four features share head and half
+            const bool is_q = h < a.Hq, is_k = !is_q && h < a.Hq + a.Hkv;
+            const int pfo = (i < half) ? fo + half : fo - half;
+            const int ci = (i < half) ? i : i - half;
+            const int kvh = is_k ? h - a.Hq : h - a.Hq - a.Hkv;
+            for (int lr = ew; lr < my_rows; lr += 4) {
+                const int rr = r0 + row_lo + lr;
+                float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
+                for (int k = 0; k < a.S; ++k) {
+                    const float *pl = tile + (size_t)(k * RP + lr) * BM;
+                    const float4 pa = *reinterpret_cast<const float4 *>(pl + fo);
+                    const float4 pb = *reinterpret_cast<const float4 *>(pl + pfo);
+                    va.x += pa.x; va.y += pa.y; va.z += pa.z; va.w += pa.w;
+                    vb.x += pb.x; vb.y += pb.y; vb.z += pb.z; vb.w += pb.w;
+                }
+                if (!valid) continue;
+                const float sc = inv_rms[row_lo + lr];
+                va.x *= sc; va.y *= sc; va.z *= sc; va.w *= sc;
+                vb.x *= sc; vb.y *= sc; vb.z *= sc; vb.w *= sc;
+                float4 out = va;
+                if (is_q || is_k) {
+                    const float4 cs = *reinterpret_cast<const float4 *>(a.rope_cos + (size_t)rr * half + ci);
+                    const float4 sn = *reinterpret_cast<const float4 *>(a.rope_sin + (size_t)rr * half + ci);
+                    if (i < half) {
+                        out.x = va.x * cs.x - vb.x * sn.x; out.y = va.y * cs.y - vb.y * sn.y;
+                        out.z = va.z * cs.z - vb.z * sn.z; out.w = va.w * cs.w - vb.w * sn.w;
+                    } else {
+                        out.x = va.x * cs.x + vb.x * sn.x; out.y = va.y * cs.y + vb.y * sn.y;
+                        out.z = va.z * cs.z + vb.z * sn.z; out.w = va.w * cs.w + vb.w * sn.w;
+                    }
+                }
+                __nv_bfloat162 lo = __floats2bfloat162_rn(out.x, out.y), hi = __floats2bfloat162_rn(out.z, out.w);
+                uint2 ob;
+                ob.x = *reinterpret_cast<uint32_t *>(&lo);
+                ob.y = *reinterpret_cast<uint32_t *>(&hi);
+                if (is_q) {
+                    if (rr < a.Rq) *reinterpret_cast<uint2 *>(a.q + ((size_t)rr * a.Hq + h) * d + i) = ob;
+                } else {
+                    const long long base = a.kvrow[rr];
+                    if (base >= 0)
+                        *reinterpret_cast<uint2 *>(a.pool_layer + (size_t)base + (is_k ? 0 : a.v_off) + (size_t)kvh * a.head_stride + i) = ob;
+                }
+            }
+        }
+    }
+
+    if (trace && threadIdx.x == 64) trace[8] = global_ns();
     tc_fence_before();
     __syncthreads();
+    if (trace && threadIdx.x == 0) trace[9] = global_ns();
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
@@ -478,13 +527,15 @@ cudaError_t launch_mode(const TcGemmArgs &a, const CUtensorMap &mw, const CUtens
     cfg.blockDim = dim3(192, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
     attr[0].val.clusterDim.y = (MODE >= 3) ? grid.y : 1;     // the K splits of one tile form a cluster
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<MODE>, mw, mx, a);
 }
 
@@ -510,18 +561,18 @@ int tc_row_pad(int R) {
 
 cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, const CUtensorMap &map_x, cudaStream_t st) {
     a.np = tc_row_pad(a.R);
-    const int nw = (mode == 1) ? 2 : 1;
-    const int stage_bytes = nw * BM * 128 + a.np * 128;
-    // Clustered modes keep the ring under half of an SM's shared memory so that two CTAs fit per SM: a GPC
-    // then offers enough CTA slots for every cluster of the launch to be resident in one wave.
-    int stages = (int)(((mode >= 3 ? 100 : 212) * 1024) / stage_bytes);
+    const int stage_bytes = BM * 128 + a.np * 128;
+    // The ring stays under half of an SM's shared memory so that two CTAs fit per SM: a GPC then offers enough
+    // CTA slots for every cluster of a launch to be resident in one wave, and one CTA's prologue and epilogue
+    // overlap the other's streaming.
+    int stages = (int)((100 * 1024) / stage_bytes);
     stages = stages > 12 ? 12 : (stages < 2 ? 2 : stages);
     a.stages = stages;
     uint32_t cols = 32;
-    while ((int)cols < nw * a.np) cols <<= 1;
+    while ((int)cols < a.np) cols <<= 1;
     a.tmem_cols = cols;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
-    const int tiles = ((mode == 1 ? a.F : a.Nout) + BM - 1) / BM;
+    const int tiles = mode == 1 ? (a.F + 63) / 64 : (a.Nout + BM - 1) / BM;
     dim3 grid(tiles, a.S, (a.R + 127) / 128);
     if (mode >= 3) {
         // every CTA's ring must hold S planes of ceil(np/S) rows, and a cluster has at most 8 CTAs

@@ -36,6 +36,7 @@ struct TcGemmArgs {
     size_t v_off, head_stride;
     const float *rope_cos, *rope_sin;   // [R][head_dim/2]
     int Hq, Hkv, head_dim, Rq;
+    unsigned long long *trace;   // test hook: 16 phase timestamps (ns) of CTA (0,0,0), or nullptr
     // filled by launch_gemm_tc
     int np, stages;
     uint32_t tmem_cols;
@@ -45,7 +46,8 @@ struct TcGemmArgs {
 bool tc_make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows);
 // activation rows per CTA, padded to the UMMA N granularity (box_rows of the X map)
 int tc_row_pad(int R);
-// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max, 3 cluster split-K + residual, 4 cluster split-K + rotary/KV write.  map_w box_rows must be 128, map_x box_rows tc_row_pad(R).
+// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max, 3 cluster split-K + residual, 4 cluster split-K + rotary/KV write.
+// map_w box_rows must be 128 (64 in mode 1), map_x box_rows tc_row_pad(R).
 cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, const CUtensorMap &map_x, cudaStream_t st);
 
 }  // namespace glance

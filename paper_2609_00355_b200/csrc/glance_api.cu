@@ -148,6 +148,9 @@ struct glance_ctx {
     // TMA descriptors, keyed by (base, inner extent, rows, box rows); built on first use by a host-only call
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;
     bool map_error = false;
+    // test hook: phase timestamps of successive GEMM launches, 16 words each, ring of trace_slots launches
+    unsigned long long *trace = nullptr;
+    int trace_slots = 0, trace_next = 0;
 };
 
 namespace {
@@ -192,10 +195,14 @@ const CUtensorMap *get_map(glance_ctx *ctx, const void *base, int inner, int row
 // Launches the weight-streaming GEMM described by `a` (mode: see gemm_tc.cuh) on X [R][K] (x_rows rows are
 // allocated behind X) and W [Nout][K], and tallies its algorithmic bytes.
 void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, TcGemmArgs a) {
-    const CUtensorMap *mw = get_map(ctx, W, a.K, a.Nout, 128);
+    const CUtensorMap *mw = get_map(ctx, W, a.K, a.Nout, mode == 1 ? 64 : 128);
     const CUtensorMap *mx = get_map(ctx, X, a.K, x_rows, tc_row_pad(a.R));
     if (!mw || !mx) return;
     a.keys = ctx->ws.am_keys; a.counter = ctx->ws.am_counter; a.status = ctx->ws.status;
+    if (ctx->trace && ctx->trace_slots > 0) {
+        a.trace = ctx->trace + (size_t)(ctx->trace_next % ctx->trace_slots) * 16;
+        ctx->trace_next++;
+    }
     const bool prof = prof_begin(ctx);
     if (launch_gemm_tc(mode, a, *mw, *mx, ctx->stream) != cudaSuccess) ctx->map_error = true;
     double bytes = 2.0 * a.Nout * a.K + 2.0 * a.R * a.K;
@@ -627,6 +634,14 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
     gemm(ctx, mode, (const bf16 *)W, (const bf16 *)X, R, g);
     ctx->maps.clear();          // the hook's operands are transient: do not keep their descriptors
     return finish(ctx);
+}
+
+int32_t glance_debug_trace(glance_ctx *ctx, uint64_t *buffer, int32_t slots) {
+    if (!ctx || slots < 0 || (buffer == nullptr) != (slots == 0)) return GLANCE_E_INVALID_ARG;
+    ctx->trace = (unsigned long long *)buffer;
+    ctx->trace_slots = slots;
+    ctx->trace_next = 0;
+    return GLANCE_OK;
 }
 
 int32_t glance_profile_enable(glance_ctx *ctx, int32_t on) {
