@@ -31,6 +31,11 @@ import torch
 
 from paper_2609_00355_b200 import synth
 
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, averaged over the 118 GEMM launches of a round,
+# from the ncu capture summarised in profiles/gemm_tc_and_attn_7b_2layers_ncu_full.md (2-layer case scaled to
+# 29 layers' worth of launches + the two LM-head passes; traffic grows in proportion to the layer count)
+TRAFFIC_PER_LAUNCH = {"7b": 136.8e6}
+
 METRIC = "committed_tokens_per_s"
 UNIT = "tokens/s"
 
@@ -439,13 +444,15 @@ def main():
                       "frac_of_measured_peak": round_bytes / (ms_per_step * 1e-3) / 1e9 / peak},
         "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections, MLP, LM head)",
                      "achieved": gemm_gbs, "peak": peak, "unit": "GB/s", "frac": gemm_gbs / peak,
-                     "traffic": None, "peak_source": peak_src, "launches_timed": gemm_launches,
+                     "traffic": TRAFFIC_PER_LAUNCH.get(cfg.name), "peak_source": peak_src, "launches_timed": gemm_launches,
                      "avg_launch_us": 1e3 * gemm_ms / max(gemm_launches, 1),
                      "algorithmic_bytes_per_launch": gemm_bytes / max(gemm_launches, 1),
                      "share_of_profiled_round_time": gemm_ms / prof_ms if prof_ms > 0 else None},
         "kernel_time_share": {k: (v[0] / prof_ms if prof_ms > 0 else None) for k, v in prof.items()},
         "kernel_avg_us": {k: (1e3 * v[0] / v[2] if v[2] else None) for k, v in prof.items()},
         "e2e": {"value": e2e_committed / e2e_s if e2e_s > 0 else None, "unit": UNIT,
+                "ms_per_step": 1e3 * e2e_s / args.steps if e2e_s > 0 else None,
+                "tau": e2e_committed / (args.steps * cfg.batch * world) if e2e_s > 0 else None,
                 "h2d_bytes_per_step": int(bench.ids_host.numel() * 4 + bench.lp_host.numel() * 4),
                 "d2h_bytes_per_step": int(bench.res_host.numel() * 4)},
         "gpu_launches": int(launches_per_round * args.steps),
@@ -454,6 +461,7 @@ def main():
     }
     if not args.no_cpu_baseline and world == 1:
         sample = OracleSample(cfg, bench.tw, bench.hw)
+        sample.round_seconds()                                   # first call pages the fp32 copies in
         t_round, desc, threads = sample.round_seconds(), sample.desc, sample.threads
         tau = line["tau"]
         line["cpu_baseline"] = {"value": tau / t_round, "unit": UNIT, "cores": threads, "kind": "oracle",
