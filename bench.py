@@ -272,6 +272,17 @@ class OracleSample:
         return t_draft + tb + per_layer * (cfg.n_layers - self.lb)
 
 
+def combine_replica_stats(total_ms, committed, e2e_s, e2e_committed, dist, device):
+    """Replicas share nothing on the data path: the job's time is the slowest replica's, its tokens the sum."""
+    stats = torch.tensor([total_ms, float(committed), e2e_s, float(e2e_committed)], dtype=torch.float64, device=device)
+    if dist is None:
+        return total_ms, float(committed), e2e_s, float(e2e_committed)
+    mx, sm = stats.clone(), stats.clone()
+    dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+    dist.all_reduce(sm, op=dist.ReduceOp.SUM)
+    return float(mx[0]), float(sm[1]), float(mx[2]), float(sm[3])
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -415,14 +426,7 @@ def main():
     eng.check_device_status()
 
     total_ms = sum(round_ms)
-    stats = torch.tensor([total_ms, float(committed), e2e_s, float(e2e_committed)], dtype=torch.float64, device=dev)
-    if dist is not None:
-        mx = stats.clone()
-        dist.all_reduce(mx, op=dist.ReduceOp.MAX)
-        sm = stats.clone()
-        dist.all_reduce(sm, op=dist.ReduceOp.SUM)
-        total_ms, e2e_s = float(mx[0]), float(mx[2])
-        committed, e2e_committed = float(sm[1]), float(sm[3])
+    total_ms, committed, e2e_s, e2e_committed = combine_replica_stats(total_ms, committed, e2e_s, e2e_committed, dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()

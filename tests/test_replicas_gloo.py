@@ -1,0 +1,45 @@
+"""The multi-GPU path is "replicas only": no data-path collective, only the barrier and the reduction of the
+timing statistics.  That host logic is exercised here with two gloo ranks on CPU."""
+import os
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    # replica `rank` took (10 + rank) ms and committed 100 * (rank + 1) tokens
+    res = bench.combine_replica_stats(10.0 + rank, 100 * (rank + 1), 0.02 * (rank + 1), 50 + rank, dist, "cpu")
+    dist.barrier()
+    out.put((rank, res))
+    dist.destroy_process_group()
+
+
+def test_replica_statistics_max_time_sum_tokens():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = dict(out.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank in (0, 1):
+        total_ms, committed, e2e_s, e2e_committed = results[rank]
+        assert total_ms == 11.0 and committed == 300.0           # slowest replica's time, all replicas' tokens
+        assert abs(e2e_s - 0.04) < 1e-12 and e2e_committed == 101.0
+
+
+def test_single_replica_passthrough():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.combine_replica_stats(5.0, 7, 0.1, 3, None, "cpu") == (5.0, 7.0, 0.1, 3.0)
