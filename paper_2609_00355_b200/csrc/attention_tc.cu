@@ -1,0 +1,501 @@
+// Split-KV paged attention on the 5th-generation tensor cores (tcgen05 + TMEM) for the packed tree rows
+// (Definition 1: ancestor-masked target pass) and the draft block (Section 3.2).
+//
+// One CTA = (128 packed query rows of one kv head, one key split).  The G query heads that share a kv
+// head are packed into the row dimension (packed row = node * G + g), so each K/V page is fetched once
+// per CTA for all of them.  Per 64-key tile (= one KV page, TMA-loaded with 128-byte swizzle):
+//     S[128 x 64]  = Q K^T          tcgen05.mma, A = Q (K-major), B = K page (K-major), accumulator in TMEM
+//     P            = 2^(S' - m)     softmax warps read S from TMEM (four threads per row), apply the scale and
+//                                   the ancestor mask, write bf16 P into shared memory
+//     O[128 x d]  += P V            tcgen05.mma, A = P (K-major), B = V page (MN-major), accumulator in TMEM
+// The running reference maximum m of a row is only raised when a tile exceeds it by more than 2^8 (the
+// accumulator is then rescaled in TMEM), so exponentials stay far inside fp32/bf16 range and O is almost
+// never touched between tiles.  Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
+// warps 2..17 = softmax / epilogue (a row's scores and outputs are split over four threads).  The key splits of a tile form a thread-block cluster and are merged
+// through distributed shared memory.  Every mbarrier wait is bounded; a wait that gives up records
+// GLANCE_E_TIMEOUT.
+#include "kernels.cuh"
+#include "tc_ptx.cuh"
+
+namespace glance {
+
+namespace {
+
+using namespace tc;
+
+constexpr int QT = 128;          // packed query rows per CTA (UMMA M)
+constexpr int KT = kPage;        // keys per tile (UMMA N of S, K of P V)
+constexpr int MAX_SPLITS = 8;     // the splits of a tile form one thread-block cluster
+constexpr float kRescaleThreshold = 8.f;   // log2 units
+constexpr int NSOFT = 512;       // softmax / epilogue threads (16 warps)
+constexpr int NTHREADS = 64 + NSOFT;
+
+template <int D>
+struct Smem {
+    static constexpr int SLABS = D / 64;                 // 64-element (128-byte) column slabs of a d-wide tile
+    static constexpr int Q_BYTES = SLABS * QT * 128;     // 32 KB at d = 128
+    static constexpr int KV_BYTES = SLABS * KT * 128;    // one K or V page: 16 KB at d = 128
+    static constexpr int P_BYTES = QT * 128;             // 128 rows x 64 keys bf16
+    static constexpr int TOTAL = Q_BYTES + 4 * KV_BYTES + P_BYTES + 1024;
+    static constexpr uint32_t TMEM_COLS = (64 + D) <= 128 ? 128 : 256;
+};
+
+struct alignas(8) AttnBars {
+    uint64_t q_ready, kv_full[2], kv_empty[2], s_full, p_full, o_done;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int D>
+__global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_constant__ CUtensorMap map_kv, AttnParams p) {
+    constexpr int SLABS = Smem<D>::SLABS;
+    constexpr int CH = D / 8;                            // 16-byte chunks per row
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    unsigned char *sQ = smem;
+    unsigned char *sK = sQ + Smem<D>::Q_BYTES;                       // 2 stages
+    unsigned char *sV = sK + 2 * Smem<D>::KV_BYTES;                  // 2 stages
+    unsigned char *sP = sV + 2 * Smem<D>::KV_BYTES;
+    __shared__ AttnBars bars;
+    __shared__ float red[2][4][QT];                       // cross-column-group exchange of row maxima / sums
+
+    unsigned long long *trace = (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? p.trace : nullptr;
+    if (trace && threadIdx.x == 0) trace[0] = global_ns();
+    pdl_launch_dependents();
+    const int G = p.Hq / p.Hkv;
+    const int PR = p.T * G;
+    const int qt = blockIdx.x, kvh = blockIdx.y;
+    const int s = blockIdx.z / p.S, split = blockIdx.z % p.S;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        mbar_init(&bars.q_ready, NSOFT);
+        mbar_init(&bars.kv_full[0], 1);
+        mbar_init(&bars.kv_full[1], 1);
+        mbar_init(&bars.kv_empty[0], 1);
+        mbar_init(&bars.kv_empty[1], 1);
+        mbar_init(&bars.s_full, 1);
+        mbar_init(&bars.p_full, NSOFT);
+        mbar_init(&bars.o_done, 1);
+        bars.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars.tmem_base)), "r"(Smem<D>::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_S = bars.tmem_base, tmem_O = bars.tmem_base + 64;
+    volatile int *abort_flag = &bars.abort_flag;
+    bool sm_ok = true;                                   // softmax warps: state carried into the split merge
+    float sm_m = -INFINITY, sm_l = 0.f;
+
+    if (trace && threadIdx.x == 0) trace[1] = global_ns();
+    pdl_wait();                                          // everything below reads data of earlier kernels
+    if (trace && threadIdx.x == 0) trace[2] = global_ns();
+    const int P = p.seq_len[s];
+    const int n_keys = P + p.T;
+    const int n_tiles = (n_keys + KT - 1) / KT;
+    const int t_begin = (int)((long long)split * n_tiles / p.S);
+    const int t_end = (int)((long long)(split + 1) * n_tiles / p.S);
+    const int nt = t_end - t_begin;
+    const int32_t *pt = p.page_table + (size_t)s * p.geom.max_pages_per_seq;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: one K page + one V page per tile ----------------
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kv) : "memory");
+            int issued = 0;
+            for (int i = 0; i < nt; ++i) {
+                const int st = i & 1;
+                if (!mbar_wait(&bars.kv_empty[st], (uint32_t)((i >> 1) & 1) ^ 1u, abort_flag, p.status)) break;
+                const int t = t_begin + i;
+                int page = (t < p.geom.max_pages_per_seq) ? pt[t] : -1;
+                if (page < 0 || page >= p.geom.n_pages) {
+                    page = 0;
+                    set_status(p.status, GLANCE_E_BOUNDS);
+                }
+                const int krow = ((page * 2 + 0) * p.geom.n_kv_heads + kvh) * KT;
+                const int vrow = ((page * 2 + 1) * p.geom.n_kv_heads + kvh) * KT;
+                mbar_expect_tx(&bars.kv_full[st], 2u * Smem<D>::KV_BYTES);
+#pragma unroll
+                for (int sl = 0; sl < SLABS; ++sl) {
+                    tma_load_2d(sK + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.kv_full[st], sl * 64, krow);
+                    tma_load_2d(sV + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.kv_full[st], sl * 64, vrow);
+                }
+                issued = i + 1;
+            }
+            if (*abort_flag) {
+                for (int i = max(0, issued - 2); i < issued; ++i) {
+                    const uint64_t t0 = global_ns();
+                    while (!mbar_try_wait(&bars.kv_full[i & 1], (uint32_t)(i >> 1) & 1u))
+                        if (global_ns() - t0 > kWaitLimitNs) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0 && nt > 0) {
+            const uint32_t idesc_s = umma_idesc(KT);              // M 128, N 64 keys
+            const uint32_t idesc_o = umma_idesc_bmn(D);           // M 128, N d, B = V is MN-major
+            bool ok = mbar_wait(&bars.q_ready, 0, abort_flag, p.status);
+            for (int i = 0; i < nt && ok; ++i) {
+                const int st = i & 1;
+                if (!mbar_wait(&bars.kv_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t kbase = smem_u32(sK + st * Smem<D>::KV_BYTES), vbase = smem_u32(sV + st * Smem<D>::KV_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const int sl = ks >> 2, kk = ks & 3;
+                    umma_f16(tmem_S, umma_desc(smem_u32(sQ) + sl * QT * 128) + (uint64_t)(kk * 2),
+                             umma_desc(kbase + sl * KT * 128) + (uint64_t)(kk * 2), idesc_s, ks > 0 ? 1u : 0u);
+                }
+                umma_commit(&bars.s_full);
+                if (!mbar_wait(&bars.p_full, (uint32_t)i & 1u, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int kk = 0; kk < KT / 16; ++kk)
+                    umma_f16(tmem_O, umma_desc(smem_u32(sP)) + (uint64_t)(kk * 2), umma_desc_mn(vbase + kk * 16 * 128, KT * 128),
+                             idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
+                umma_commit(&bars.kv_empty[st]);          // K and V pages free once these MMAs have read them
+                umma_commit(&bars.o_done);                // P free, O updated
+            }
+        }
+    } else {
+        // ---------------- softmax / epilogue warps ----------------
+        // 16 warps: warp (q, cg) serves the TMEM lane quarter q (32 query rows) and the column group cg;
+        // a row's 64 scores are split over four threads (16 keys each), its d output columns likewise.
+        const int q = warp & 3;                           // TMEM lane quarter this warp may access
+        const int cg = (warp - 2) >> 2;                   // column group 0..3
+        const int row = q * 32 + lane;
+        const int tsm = threadIdx.x - 64;                 // 0..511
+        int pr = qt * QT + row;
+        const bool row_valid = pr < PR;
+        if (!row_valid) pr = PR - 1;
+        const int node = pr / G, g = pr % G;
+        uint64_t anc0 = 0, anc1 = 0;
+        if (p.anc) {
+            const uint64_t *a = p.anc + ((size_t)s * p.T + node) * p.W;
+            anc0 = a[0];
+            anc1 = p.W > 1 ? a[1] : 0ull;
+        }
+        // Q tile -> shared memory in the K-major 128-byte-swizzled operand layout (async copies, all in flight)
+        for (int it = tsm; it < QT * CH; it += NSOFT) {
+            const int r = it / CH, c = it % CH;
+            int prr = qt * QT + r;
+            if (prr >= PR) prr = PR - 1;
+            const bf16 *src = p.q + ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c * 8;
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(sQ + (c >> 3) * QT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4))), "l"(src));
+        }
+        asm volatile("cp.async.commit_group;" ::);
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        fence_async_smem();
+        mbar_arrive(&bars.q_ready);
+        if (trace && threadIdx.x == 64) trace[3] = global_ns();
+
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;
+        constexpr int OC = D / 4;                         // output columns per thread
+        float m_ref = -INFINITY, l_run = 0.f;             // l_run: this thread's share of the row sum
+        bool ok = true;
+        for (int i = 0; i < nt; ++i) {
+            const int t = t_begin + i;
+            const int st = i & 1;
+            const int key0 = t * KT;
+            const int valid_keys = min(KT, n_keys - key0);
+            if (valid_keys < KT) {
+                // rows of the page beyond the last key may hold anything (NaN bits included): zero them in V
+                ok = ok && mbar_wait(&bars.kv_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status);
+                if (ok) {
+                    unsigned char *v = sV + st * Smem<D>::KV_BYTES;
+                    for (int it = tsm; it < (KT - valid_keys) * CH; it += NSOFT) {
+                        const int r = valid_keys + it / CH, c = it % CH;
+                        *reinterpret_cast<int4 *>(v + (c >> 3) * KT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = make_int4(0, 0, 0, 0);
+                    }
+                    fence_async_smem();
+                }
+            }
+            ok = ok && mbar_wait(&bars.s_full, (uint32_t)i & 1u, abort_flag, p.status);
+            ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are warp-collective
+            if (trace && threadIdx.x == 64 && i == 0) trace[4] = global_ns();
+            tc_fence_after();
+            float sc[16];
+            {
+                uint32_t v[16];
+                if (ok) {
+                    tmem_ld16(tmem_S + lane_addr + (uint32_t)(cg * 16), v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0u;
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) sc[j] = __uint_as_float(v[j]);
+            }
+            const bool need_mask = key0 + KT > P;
+            float mt = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                float v = sc[j] * sl2;
+                if (need_mask) {
+                    const int key = key0 + cg * 16 + j;
+                    bool vis = key < P;
+                    if (!vis && key < n_keys) {
+                        const int b = key - P;
+                        const uint64_t w = (b >> 6) ? anc1 : anc0;
+                        vis = p.anc ? ((w >> (b & 63)) & 1ull) : true;
+                    }
+                    v = vis ? v : -INFINITY;
+                }
+                sc[j] = v;
+                mt = fmaxf(mt, v);
+            }
+            // row maximum of the tile across the four column groups
+            red[i & 1][cg][row] = mt;
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (*abort_flag) break;                       // uniform across the 16 warps: read right after the barrier
+            mt = fmaxf(fmaxf(red[i & 1][0][row], red[i & 1][1][row]), fmaxf(red[i & 1][2][row], red[i & 1][3][row]));
+            if (i > 0) {
+                // P and O are in use by the previous tile's second MMA until o_done
+                ok = ok && mbar_wait(&bars.o_done, (uint32_t)(i - 1) & 1u, abort_flag, p.status);
+                ok = __all_sync(0xffffffffu, ok);
+                tc_fence_after();
+            }
+            float factor = 1.f;
+            if (m_ref == -INFINITY) {
+                m_ref = mt;                               // nothing accumulated for this row yet
+            } else if (mt > m_ref + kRescaleThreshold) {
+                factor = exp2f(m_ref - mt);
+                m_ref = mt;
+            }
+            if (__any_sync(0xffffffffu, factor != 1.f) && ok) {
+                l_run *= factor;
+#pragma unroll
+                for (int c = 0; c < OC; c += 16) {
+                    uint32_t v[16];
+                    tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * factor);
+                    tmem_st16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                }
+                tmem_st_wait();
+            }
+            // P = 2^(S' - m_ref), bf16: this thread's 16 keys = two 16-byte chunks of its row of the A operand
+            float rs = 0.f;
+            unsigned char *prow = sP + row * 128;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t w[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const float a = sc[c * 8 + 2 * j], b = sc[c * 8 + 2 * j + 1];
+                    const float pa = (a == -INFINITY) ? 0.f : exp2f(a - m_ref);
+                    const float pb = (b == -INFINITY) ? 0.f : exp2f(b - m_ref);
+                    rs += pa + pb;
+                    __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
+                    w[j] = *reinterpret_cast<uint32_t *>(&h2);
+                }
+                *reinterpret_cast<uint4 *>(prow + (((cg * 2 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            l_run += rs;
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(&bars.p_full);                    // always arrive: the MMA issuer counts 512 arrivals
+            if (trace && threadIdx.x == 64 && i == 0) trace[5] = global_ns();
+        }
+        if (trace && threadIdx.x == 64) trace[6] = global_ns();
+        if (ok && nt > 0) {
+            ok = mbar_wait(&bars.o_done, (uint32_t)(nt - 1) & 1u, abort_flag, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after();
+        }
+        // row sums across the four column groups (fixed order)
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        red[0][cg][row] = l_run;
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+        const float l_row = ((red[0][0][row] + red[0][1][row]) + red[0][2][row]) + red[0][3][row];
+        ok = ok && (*abort_flag == 0);
+        // ---------------- epilogue ----------------
+        if (p.S == 1 && ok) {
+            const float inv = 1.f / l_row;
+            bf16 *dst = p.out + ((size_t)(s * p.T + node) * p.Hq + kvh * G + g) * D + cg * OC;
+#pragma unroll
+            for (int c = 0; c < OC; c += 16) {
+                uint32_t v[16];
+                tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                tmem_ld_wait();
+                if (row_valid) {
+                    uint32_t w[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[2 * j]) * inv, __uint_as_float(v[2 * j + 1]) * inv);
+                        w[j] = *reinterpret_cast<uint32_t *>(&h2);
+                    }
+                    *reinterpret_cast<uint4 *>(dst + c) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4 *>(dst + c + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            }
+        }
+        tc_fence_before();
+        sm_ok = ok;
+        sm_m = m_ref;
+        sm_l = l_row;
+    }
+
+    if (p.S > 1) {
+        // ---------------- merge of the key splits inside the cluster (reduce-scatter by rows) ----------------
+        // The S CTAs of one (sequence, kv head, q tile) form a cluster.  CTA `rank` owns rows [rank*RPC, +RPC):
+        // every CTA ships, per row, its unnormalised O row and (m, l) to the owner's shared memory (on top of
+        // the idle Q/K/V buffers), the owner combines the S partial rows in split order.
+        constexpr int ROWF = D + 4;                       // floats per shipped row: O, m, l, padding
+        constexpr int OC = D / 4;
+        const int RPC = (QT + p.S - 1) / p.S;
+        const uint32_t rank = cluster_rank();
+        if (trace && threadIdx.x == 64) trace[7] = global_ns();
+        cluster_sync_all();                               // all MMAs of the cluster are done: buffers are idle
+        if (trace && threadIdx.x == 64) trace[8] = global_ns();
+        if (warp >= 2) {
+            const int q = warp & 3, cg = (warp - 2) >> 2;
+            const int row = q * 32 + lane;
+            const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+            const uint32_t owner = (uint32_t)(row / RPC);
+            const uint32_t dst = map_to_rank(smem_u32(smem) + (uint32_t)(((rank * RPC + (row - owner * RPC)) * ROWF) * 4), owner);
+            const bool live = nt > 0 && sm_ok;
+#pragma unroll
+            for (int c = 0; c < OC; c += 16) {
+                uint32_t v[16];
+                if (live) {
+                    tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = 0u;
+                }
+#pragma unroll
+                for (int j = 0; j < 16; j += 4)
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((cg * OC + c + j) * 4)), "r"(v[j]),
+                                 "r"(v[j + 1]), "r"(v[j + 2]), "r"(v[j + 3]) : "memory");
+            }
+            if (cg == 0) {
+                st_cluster_f32(dst + D * 4, live ? sm_m : -INFINITY);
+                st_cluster_f32(dst + D * 4 + 4, live ? sm_l : 0.f);
+            }
+        }
+        if (trace && threadIdx.x == 64) trace[9] = global_ns();
+        cluster_sync_all();                               // shipped rows are visible to their owners
+        if (trace && threadIdx.x == 64) trace[10] = global_ns();
+        if (warp >= 2) {
+            const int tsm = threadIdx.x - 64;
+            const float *rows = reinterpret_cast<const float *>(smem);
+            const int row_lo = (int)rank * RPC;
+            const int my_rows = max(0, min(min(RPC, QT - row_lo), PR - qt * QT - row_lo));
+            constexpr int SEG = D / 4;                    // 4-float segments per row
+            for (int item = tsm; item < my_rows * SEG; item += NSOFT) {
+                const int lr = item / SEG, c0 = (item % SEG) * 4;
+                float M = -INFINITY;
+                for (int sp = 0; sp < p.S; ++sp) M = fmaxf(M, rows[(size_t)(sp * RPC + lr) * ROWF + D]);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float den = 0.f;
+                for (int sp = 0; sp < p.S; ++sp) {        // split order: bit-reproducible
+                    const float *rp = rows + (size_t)(sp * RPC + lr) * ROWF;
+                    const float ms = rp[D];
+                    const float w = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
+                    den += w * rp[D + 1];
+                    const float4 v = *reinterpret_cast<const float4 *>(rp + c0);
+                    acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+                }
+                const float inv = 1.f / den;
+                const int prr = qt * QT + row_lo + lr;
+                bf16 *dst = p.out + ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c0;
+                __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+                uint2 o;
+                o.x = *reinterpret_cast<uint32_t *>(&lo);
+                o.y = *reinterpret_cast<uint32_t *>(&hi);
+                *reinterpret_cast<uint2 *>(dst) = o;
+            }
+        }
+    }
+    if (trace && threadIdx.x == 64) trace[11] = global_ns();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(bars.tmem_base), "r"(Smem<D>::TMEM_COLS) : "memory");
+    }
+}
+
+template <int D>
+cudaError_t launch_d(const AttnParams &p, const CUtensorMap &map_kv, dim3 grid, cudaStream_t st) {
+    static bool once = false;
+    if (!once) {
+        cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL);
+        if (e != cudaSuccess) return e;
+        once = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(NTHREADS, 1, 1);
+    cfg.dynamicSmemBytes = Smem<D>::TOTAL;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // the key splits of one tile form a cluster
+    attr[1].val.clusterDim.x = 1;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = p.S;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, attn_tc_kernel<D>, map_kv, p);
+}
+
+// largest number of co-resident clusters of `cs` CTAs of this kernel (queried once per cluster size)
+template <int D>
+int max_active_clusters(int cs) {
+    static int cache[MAX_SPLITS + 1] = {0};
+    if (cache[cs] == 0) {
+        cudaFuncSetAttribute(attn_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Smem<D>::TOTAL);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1, 1, cs);
+        cfg.blockDim = dim3(NTHREADS, 1, 1);
+        cfg.dynamicSmemBytes = Smem<D>::TOTAL;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 1;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = cs;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, attn_tc_kernel<D>, &cfg) != cudaSuccess || n < 1) n = 148 / cs - 4;
+        cache[cs] = n < 1 ? 1 : n;
+    }
+    return cache[cs];
+}
+
+}  // namespace
+
+int attention_tc_q_tiles(int T, int G) { return (T * G + QT - 1) / QT; }
+
+// Key splits per (sequence, kv head, q tile): the splits of a tile form a cluster, and all clusters of the
+// launch should be resident at once (a second wave would double the kernel's latency).
+int attention_tc_splits(int T, int G, int Hkv, int batch, int d) {
+    const int base = attention_tc_q_tiles(T, G) * Hkv * batch;
+    for (int s = MAX_SPLITS; s > 1; --s) {
+        const int fit = d == 128 ? max_active_clusters<128>(s) : max_active_clusters<64>(s);
+        if (base <= fit) return s;
+    }
+    return 1;
+}
+
+cudaError_t launch_attention_tc(const AttnParams &p, const CUtensorMap &map_kv, cudaStream_t st) {
+    const int G = p.Hq / p.Hkv;
+    dim3 grid(attention_tc_q_tiles(p.T, G), p.Hkv, p.batch * p.S);
+    if (p.d == 128) return launch_d<128>(p, map_kv, grid, st);
+    return launch_d<64>(p, map_kv, grid, st);
+}
+
+}  // namespace glance

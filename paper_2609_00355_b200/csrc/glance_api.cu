@@ -214,6 +214,20 @@ void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, T
     prof_end(ctx, prof, KIND_GEMM, bytes);
 }
 
+// tree / block attention on one pool layer (K/V pages are fetched by TMA through a per-layer descriptor)
+void attention(glance_ctx *ctx, AttnParams ap) {
+    ap.trace = nullptr;
+    if (ctx->trace && ctx->trace_slots > 0) {
+        ap.trace = ctx->trace + (size_t)(ctx->trace_next % ctx->trace_slots) * 16;
+        ctx->trace_next++;
+    }
+    const CUtensorMap *m = get_map(ctx, ap.pool_layer, ap.d, ap.geom.n_pages * 2 * ap.geom.n_kv_heads * kPage, kPage);
+    if (!m) return;
+    const bool prof = prof_begin(ctx);
+    if (launch_attention_tc(ap, *m, ctx->stream) != cudaSuccess) ctx->map_error = true;
+    prof_end(ctx, prof, KIND_ATTN, 0.0);
+}
+
 // row scales 1/rms from the per-tile sums of squares the producer left in ws.ssq
 void with_row_scales(const glance_ctx *ctx, TcGemmArgs &a) {
     a.ssq = ctx->ws.ssq; a.n_ssq = ctx->dims.n_ssq; a.ssq_stride = ctx->dims.Rmax; a.eps = ctx->cfg.rms_eps;
@@ -292,9 +306,9 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
     ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn;
-    ap.S = attention_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch); ap.part_o = ws.att_o;
+    ap.S = attention_tc_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch, c.head_dim); ap.part_o = ws.att_o;
     ap.part_ml = ws.att_ml; ap.counters = ws.att_ctr; ap.status = ws.status;
-    LAUNCH(ctx, KIND_ATTN, launch_attention(ap, st));
+    attention(ctx, ap);
     const int R = ps.Rq;
     {
         TcGemmArgs g{};
@@ -616,10 +630,10 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     ap.batch = seqs->batch; ap.T = T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = (const bf16 *)q; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
-    ap.out = (bf16 *)out; ap.S = attention_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch);
+    ap.out = (bf16 *)out; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
     ap.part_o = ctx->ws.att_o; ap.part_ml = ctx->ws.att_ml;
     ap.counters = ctx->ws.att_ctr; ap.status = ctx->ws.status;
-    LAUNCH(ctx, KIND_ATTN, launch_attention(ap, ctx->stream));
+    attention(ctx, ap);
     return finish(ctx);
 }
 

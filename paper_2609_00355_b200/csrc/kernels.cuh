@@ -1,5 +1,7 @@
 // Launch wrappers of the round's kernels (definitions in the .cu files beside this header).
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace glance {
@@ -105,8 +107,13 @@ struct AttnParams {
     float *part_ml;              // [batch][Hkv][PR][S][2]
     int32_t *counters;           // [batch][Hkv][q_tiles], zero between calls
     int32_t *status;
+    unsigned long long *trace;   // test hook: phase timestamps of the first CTA, or nullptr
 };
 void launch_attention(const AttnParams &p, cudaStream_t st);
+// tcgen05 version (attention_tc.cu): map_kv = 2-D map of the pool layer {d, n_pages*2*Hkv*64 rows}, box {64, 64}
+cudaError_t launch_attention_tc(const AttnParams &p, const CUtensorMap &map_kv, cudaStream_t st);
+int attention_tc_q_tiles(int T, int G);
+int attention_tc_splits(int T, int G, int Hkv, int batch, int d);
 int attention_q_tiles(int T, int G);
 int attention_splits(int T, int G, int Hkv, int batch);   // key splits so that one wave of CTAs covers the SMs
 
