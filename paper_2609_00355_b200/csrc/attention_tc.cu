@@ -37,11 +37,11 @@ struct Smem {
     static constexpr int KV_BYTES = SLABS * KT * 128;    // one K or V page: 16 KB at d = 128
     static constexpr int P_BYTES = QT * 128;             // 128 rows x 64 keys bf16
     static constexpr int TOTAL = Q_BYTES + 4 * KV_BYTES + P_BYTES + 1024;
-    static constexpr uint32_t TMEM_COLS = (64 + D) <= 128 ? 128 : 256;
+    static constexpr uint32_t TMEM_COLS = 256;           // two S buffers (2 x 64) + O (d)
 };
 
 struct alignas(8) AttnBars {
-    uint64_t q_ready, kv_full[2], kv_empty[2], s_full, p_full, o_done;
+    uint64_t q_ready, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full, o_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -70,11 +70,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 
     if (threadIdx.x == 0) {
         mbar_init(&bars.q_ready, NSOFT);
-        mbar_init(&bars.kv_full[0], 1);
-        mbar_init(&bars.kv_full[1], 1);
-        mbar_init(&bars.kv_empty[0], 1);
-        mbar_init(&bars.kv_empty[1], 1);
-        mbar_init(&bars.s_full, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bars.k_full[b], 1);
+            mbar_init(&bars.k_empty[b], 1);
+            mbar_init(&bars.v_full[b], 1);
+            mbar_init(&bars.v_empty[b], 1);
+            mbar_init(&bars.s_full[b], 1);
+        }
         mbar_init(&bars.p_full, NSOFT);
         mbar_init(&bars.o_done, 1);
         bars.abort_flag = 0;
@@ -87,14 +89,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_S = bars.tmem_base, tmem_O = bars.tmem_base + 64;
+    const uint32_t tmem_S = bars.tmem_base, tmem_O = bars.tmem_base + 128;   // S is double-buffered: columns 0-63, 64-127
     volatile int *abort_flag = &bars.abort_flag;
     bool sm_ok = true;                                   // softmax warps: state carried into the split merge
     float sm_m = -INFINITY, sm_l = 0.f;
 
     if (trace && threadIdx.x == 0) trace[1] = global_ns();
-    pdl_wait();                                          // everything below reads data of earlier kernels
-    if (trace && threadIdx.x == 0) trace[2] = global_ns();
+    // Sequence lengths and page tables only change in the commit kernel of the previous round, long finished:
+    // they may be read before the dependency wait.  Pages entirely below seq_len - block_B hold committed
+    // context that no kernel of this pass writes, so the producer prefetches them before the wait as well.
     const int P = p.seq_len[s];
     const int n_keys = P + p.T;
     const int n_tiles = (n_keys + KT - 1) / KT;
@@ -102,16 +105,27 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const int t_end = (int)((long long)(split + 1) * n_tiles / p.S);
     const int nt = t_end - t_begin;
     const int32_t *pt = p.page_table + (size_t)s * p.geom.max_pages_per_seq;
+    if (warp != 0) {
+        pdl_wait();                                      // q, the tree rows' K/V and the outputs belong to other kernels
+        if (trace && threadIdx.x == 64) trace[2] = global_ns();
+    }
 
     if (warp == 0) {
-        // ---------------- TMA producer: one K page + one V page per tile ----------------
+        // ---------------- TMA producer: K pages and V pages in separate two-slot rings ----------------
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kv) : "memory");
+            bool waited = false;
             int issued = 0;
             for (int i = 0; i < nt; ++i) {
                 const int st = i & 1;
-                if (!mbar_wait(&bars.kv_empty[st], (uint32_t)((i >> 1) & 1) ^ 1u, abort_flag, p.status)) break;
+                const uint32_t ph = (uint32_t)((i >> 1) & 1);
                 const int t = t_begin + i;
+                // rows written by this pass lie in [P - block_B, P + T): the head's refreshed context rows and
+                // the new tree / block rows
+                if (!waited && (i >= 2 || (t + 1) * KT > P - kMaxBlock)) {
+                    pdl_wait();
+                    waited = true;
+                }
                 int page = (t < p.geom.max_pages_per_seq) ? pt[t] : -1;
                 if (page < 0 || page >= p.geom.n_pages) {
                     page = 0;
@@ -119,47 +133,70 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 }
                 const int krow = ((page * 2 + 0) * p.geom.n_kv_heads + kvh) * KT;
                 const int vrow = ((page * 2 + 1) * p.geom.n_kv_heads + kvh) * KT;
-                mbar_expect_tx(&bars.kv_full[st], 2u * Smem<D>::KV_BYTES);
+                if (!mbar_wait(&bars.k_empty[st], ph ^ 1u, abort_flag, p.status)) break;
+                mbar_expect_tx(&bars.k_full[st], (uint32_t)Smem<D>::KV_BYTES);
 #pragma unroll
-                for (int sl = 0; sl < SLABS; ++sl) {
-                    tma_load_2d(sK + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.kv_full[st], sl * 64, krow);
-                    tma_load_2d(sV + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.kv_full[st], sl * 64, vrow);
-                }
+                for (int sl = 0; sl < SLABS; ++sl)
+                    tma_load_2d(sK + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.k_full[st], sl * 64, krow);
+                if (!mbar_wait(&bars.v_empty[st], ph ^ 1u, abort_flag, p.status)) { issued = -(i + 1); break; }
+                mbar_expect_tx(&bars.v_full[st], (uint32_t)Smem<D>::KV_BYTES);
+#pragma unroll
+                for (int sl = 0; sl < SLABS; ++sl)
+                    tma_load_2d(sV + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.v_full[st], sl * 64, vrow);
                 issued = i + 1;
             }
+            if (!waited) pdl_wait();
             if (*abort_flag) {
-                for (int i = max(0, issued - 2); i < issued; ++i) {
+                // copies already issued must land before the CTA may exit
+                const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
+                for (int i = max(0, nk - 2); i < nk; ++i) {
                     const uint64_t t0 = global_ns();
-                    while (!mbar_try_wait(&bars.kv_full[i & 1], (uint32_t)(i >> 1) & 1u))
+                    while (!mbar_try_wait(&bars.k_full[i & 1], (uint32_t)(i >> 1) & 1u))
+                        if (global_ns() - t0 > kWaitLimitNs) break;
+                }
+                for (int i = max(0, nv - 2); i < nv; ++i) {
+                    const uint64_t t0 = global_ns();
+                    while (!mbar_try_wait(&bars.v_full[i & 1], (uint32_t)(i >> 1) & 1u))
                         if (global_ns() - t0 > kWaitLimitNs) break;
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
+        // S = Q K^T of tile i+1 is issued before P V of tile i, into the other S buffer, so that the softmax
+        // warps find the next scores ready when they finish a tile.
         if (lane == 0 && nt > 0) {
             const uint32_t idesc_s = umma_idesc(KT);              // M 128, N 64 keys
             const uint32_t idesc_o = umma_idesc_bmn(D);           // M 128, N d, B = V is MN-major
-            bool ok = mbar_wait(&bars.q_ready, 0, abort_flag, p.status);
-            for (int i = 0; i < nt && ok; ++i) {
+            auto issue_s = [&](int i) -> bool {
                 const int st = i & 1;
-                if (!mbar_wait(&bars.kv_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+                if (!mbar_wait(&bars.k_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) return false;
                 tc_fence_after();
-                const uint32_t kbase = smem_u32(sK + st * Smem<D>::KV_BYTES), vbase = smem_u32(sV + st * Smem<D>::KV_BYTES);
+                const uint32_t kbase = smem_u32(sK + st * Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const int sl = ks >> 2, kk = ks & 3;
-                    umma_f16(tmem_S, umma_desc(smem_u32(sQ) + sl * QT * 128) + (uint64_t)(kk * 2),
+                    umma_f16(tmem_S + (uint32_t)(st * 64), umma_desc(smem_u32(sQ) + sl * QT * 128) + (uint64_t)(kk * 2),
                              umma_desc(kbase + sl * KT * 128) + (uint64_t)(kk * 2), idesc_s, ks > 0 ? 1u : 0u);
                 }
-                umma_commit(&bars.s_full);
+                umma_commit(&bars.k_empty[st]);           // K page free once these MMAs have read it
+                umma_commit(&bars.s_full[st]);
+                return true;
+            };
+            bool ok = mbar_wait(&bars.q_ready, 0, abort_flag, p.status);
+            ok = ok && issue_s(0);
+            for (int i = 0; i < nt && ok; ++i) {
+                const int st = i & 1;
+                if (i + 1 < nt && !issue_s(i + 1)) { ok = false; break; }
                 if (!mbar_wait(&bars.p_full, (uint32_t)i & 1u, abort_flag, p.status)) { ok = false; break; }
+                if (!mbar_wait(&bars.v_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
+                const uint32_t vbase = smem_u32(sV + st * Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < KT / 16; ++kk)
                     umma_f16(tmem_O, umma_desc(smem_u32(sP)) + (uint64_t)(kk * 2), umma_desc_mn(vbase + kk * 16 * 128, KT * 128),
                              idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(&bars.kv_empty[st]);          // K and V pages free once these MMAs have read them
+                umma_commit(&bars.v_empty[st]);           // V page free once these MMAs have read it
                 umma_commit(&bars.o_done);                // P free, O updated
             }
         }
@@ -207,7 +244,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             const int valid_keys = min(KT, n_keys - key0);
             if (valid_keys < KT) {
                 // rows of the page beyond the last key may hold anything (NaN bits included): zero them in V
-                ok = ok && mbar_wait(&bars.kv_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status);
+                ok = ok && mbar_wait(&bars.v_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status);
                 if (ok) {
                     unsigned char *v = sV + st * Smem<D>::KV_BYTES;
                     for (int it = tsm; it < (KT - valid_keys) * CH; it += NSOFT) {
@@ -217,7 +254,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     fence_async_smem();
                 }
             }
-            ok = ok && mbar_wait(&bars.s_full, (uint32_t)i & 1u, abort_flag, p.status);
+            ok = ok && mbar_wait(&bars.s_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status);
             ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are warp-collective
             if (trace && threadIdx.x == 64 && i == 0) trace[4] = global_ns();
             tc_fence_after();
@@ -225,7 +262,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             {
                 uint32_t v[16];
                 if (ok) {
-                    tmem_ld16(tmem_S + lane_addr + (uint32_t)(cg * 16), v);
+                    tmem_ld16(tmem_S + lane_addr + (uint32_t)(st * 64 + cg * 16), v);
                     tmem_ld_wait();
                 } else {
 #pragma unroll
