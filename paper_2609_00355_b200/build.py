@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libglance.so")
-SOURCES = ["glance_api.cu", "kernels_small.cu", "tree_walk.cu", "attention.cu", "attention_tc.cu", "gemm_tc.cu", "topk_static.cu"]
+SOURCES = ["glance_api.cu", "kernels_small.cu", "tree_walk.cu", "attention_tc.cu", "gemm_tc.cu", "topk_static.cu"]
 
 
 def _stale() -> bool:

@@ -8,7 +8,7 @@
 // tcgen05.mma issued from a single thread; the fp32 accumulator lives in TMEM and is read back by four
 // epilogue warps (one TMEM lane = one output feature).
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..5 = epilogue.
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..9 = epilogue.
 // Epilogues: (0) fp32 split-K plane, (1) SwiGLU over 64 gate rows and their 64 up rows stacked into one tile,
 // (2) row-wise arg-max over the vocabulary, merged across CTAs with a packed 64-bit atomic max,
 // (3)/(4) split-K reduced inside a thread-block cluster through distributed shared memory, followed by
@@ -26,6 +26,9 @@ namespace {
 
 using namespace tc;
 
+constexpr int NEPI = 8;                  // epilogue warps: two per TMEM lane quarter, splitting the columns
+constexpr int NTHR = 64 + 32 * NEPI;
+
 struct alignas(8) Barriers {
     uint64_t full[12];
     uint64_t empty[12];
@@ -40,7 +43,7 @@ struct alignas(8) Barriers {
 // Modes 0, 1, 2 and 4 multiply each activation row's results by 1/rms(row) when a.ssq is given: the rows
 // they read are x * gain in bf16, and the row's sum of squares arrives as per-tile partial sums.
 template <int MODE>
-__global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+__global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                          const __grid_constant__ CUtensorMap map_x, TcGemmArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -154,21 +157,21 @@ __global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__
         }
     } else {
         // ---------------- epilogue warps, part 1: row scales, then wait for the accumulator ----------------
-        const int t = threadIdx.x - 64;                  // 0..127
+        const int t = threadIdx.x - 64;                  // 0..255
         pdl_wait();                                      // everything below reads or writes data other kernels own
         if (MODE != 3) {
             float inv = 1.f;
-            if (a.ssq && t < NP && r0 + t < a.R) {
+            if (a.ssq && t < NP && r0 + t < a.R) {   // NP <= 128 < 256 epilogue threads
                 float ss = 0.f;
                 for (int i = 0; i < a.n_ssq; ++i) ss += __ldcg(a.ssq + (size_t)i * a.ssq_stride + r0 + t);
                 inv = rsqrtf(ss / (float)a.K + a.eps);
             }
-            inv_rms[t] = inv;
+            if (t < 128) inv_rms[t] = inv;
         }
         if (nk > 0) ok = mbar_wait(&bars.acc_ready, 0, abort_flag, a.status);
         ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld is warp-collective: decide as a warp
         tc_fence_after();
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // inv_rms / red_keys visible to the four epilogue warps
+        asm volatile("bar.sync 1, 256;" ::: "memory");   // inv_rms visible to all epilogue warps
         if (trace && threadIdx.x == 64) trace[4] = global_ns();
     }
 
@@ -189,7 +192,8 @@ __global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__
     }
     if (warp >= 2) {
         const uint32_t local = smem_u32(smem) + (uint32_t)((rank * RP) * BM * 4) + (uint32_t)(fl * 4);
-        for (int c = 0; c < NP; c += 16) {
+        const int chalf = (warp - 2) >> 2;               // the two warps of a lane quarter alternate 16-column chunks
+        for (int c = chalf * 16; c < NP; c += 32) {
             uint32_t v[16];
             if (nk > 0 && ok) {
                 tmem_ld16(lane_addr + (uint32_t)c, v);
@@ -215,17 +219,17 @@ __global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__
         cluster_sync_all();                              // planes written and visible
         if (trace && threadIdx.x == 64) trace[7] = global_ns();
     } else if (warp >= 2) {
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
     }
     if (warp >= 2 && ok) {
         const float *tile = reinterpret_cast<const float *>(smem);
-        const int ew = warp - 2;                         // epilogue warp 0..3
+        const int ew = warp - 2;                         // epilogue warp 0..7
         const int row_lo = (int)rank * RP;               // first owned row (tile-local)
         const int my_rows = max(0, min(min(RP, NP - row_lo), a.R - r0 - row_lo));
         const int fo = 4 * lane;                         // first of this thread's four features (tile-local)
         if (MODE == 0 || MODE == 2) {
             const bool vec = (a.ldy & 3) == 0;
-            for (int r = ew; r < my_rows; r += 4) {
+            for (int r = ew; r < my_rows; r += NEPI) {
                 const int rr = r0 + r;
                 float4 v = *reinterpret_cast<const float4 *>(tile + r * BM + fo);
                 const float sc = inv_rms[r];
@@ -254,7 +258,7 @@ __global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__
         } else if (MODE == 1) {
             // tile features 0..63 are gate rows, 64..127 the matching up rows; item = (row, 4 gate features)
             const int t = threadIdx.x - 64;
-            for (int item = t; item < my_rows * 16; item += 128) {
+            for (int item = t; item < my_rows * 16; item += 32 * NEPI) {
                 const int r = item >> 4, fg = (item & 15) * 4;
                 const float4 g = *reinterpret_cast<const float4 *>(tile + r * BM + fg);
                 const float4 u = *reinterpret_cast<const float4 *>(tile + r * BM + 64 + fg);
@@ -280,7 +284,7 @@ __global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__
                 const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
                 gain = make_float4(__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23));
             }
-            for (int lr = ew; lr < my_rows; lr += 4) {
+            for (int lr = ew; lr < my_rows; lr += NEPI) {
                 const size_t o = (size_t)(r0 + row_lo + lr) * a.Nout + f;
                 float4 xv = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (valid) xv = __ldcg(reinterpret_cast<const float4 *>(a.x + o));
@@ -321,7 +325,7 @@ __global__ void __launch_bounds__(192, 2) gemm_tc_kernel(const __grid_constant__
             const int pfo = (i < half) ? fo + half : fo - half;
             const int ci = (i < half) ? i : i - half;
             const int kvh = is_k ? h - a.Hq : h - a.Hq - a.Hkv;
-            for (int lr = ew; lr < my_rows; lr += 4) {
+            for (int lr = ew; lr < my_rows; lr += NEPI) {
                 const int rr = r0 + row_lo + lr;
                 float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
                 for (int k = 0; k < a.S; ++k) {
@@ -418,7 +422,7 @@ cudaError_t launch_mode(const TcGemmArgs &a, const CUtensorMap &mw, const CUtens
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
-    cfg.blockDim = dim3(192, 1, 1);
+    cfg.blockDim = dim3(NTHR, 1, 1);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];

@@ -34,9 +34,6 @@ struct Workspace {
     bf16 *attn;          // [Rmax][Hq d]
     bf16 *act;           // [Rmax][F]
     float *logits;       // [Rlog][V]
-    float *att_o;        // attention split partials
-    float *att_ml;
-    int32_t *att_ctr;
     int32_t *walk_ctr;
     int32_t *row_seq, *row_pos;
     long long *row_kvrow;
@@ -54,7 +51,7 @@ struct Workspace {
 };
 
 struct Dims {
-    int Rmax, Rlog, qkv_out, qd, S_att, q_tiles_max, W, n_ssq;
+    int Rmax, Rlog, qkv_out, qd, W, n_ssq;
 };
 
 Dims make_dims(const glance_config &c) {
@@ -65,12 +62,6 @@ Dims make_dims(const glance_config &c) {
     d.qkv_out = (c.n_q_heads + 2 * c.n_kv_heads) * c.head_dim;
     d.qd = c.n_q_heads * c.head_dim;
     d.n_ssq = (c.hidden + 127) / 128;
-    const int G = c.n_q_heads / c.n_kv_heads;
-    d.q_tiles_max = attention_q_tiles(std::max(c.tree_N, c.block_B), G);
-    // attention split partials: the largest (q tiles x key splits) over every row count a pass can have
-    d.S_att = 0;
-    for (int T = 1; T <= std::max(c.tree_N, c.block_B); ++T)
-        d.S_att = std::max(d.S_att, attention_q_tiles(T, G) * attention_splits(T, G, c.n_kv_heads, c.max_batch));
     d.W = (c.tree_N + 63) / 64;
     return d;
 }
@@ -91,10 +82,6 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.attn = (bf16 *)take(R * d.qd * 2);
     w.act = (bf16 *)take(R * (size_t)c.ffn * 2);
     w.logits = (float *)take((size_t)d.Rlog * c.vocab * 4);
-    const size_t att_rows = (size_t)c.max_batch * c.n_kv_heads * 64 * d.S_att;   // d.S_att = max q tiles x splits
-    w.att_o = (float *)take(att_rows * c.head_dim * 4);
-    w.att_ml = (float *)take(att_rows * 2 * 4);
-    w.att_ctr = (int32_t *)take((size_t)c.max_batch * c.n_kv_heads * d.q_tiles_max * 4);
     w.walk_ctr = (int32_t *)take((size_t)c.max_batch * 4);
     w.row_seq = (int32_t *)take(R * 4);
     w.row_pos = (int32_t *)take(R * 4);
@@ -306,8 +293,8 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
     ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn;
-    ap.S = attention_tc_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch, c.head_dim); ap.part_o = ws.att_o;
-    ap.part_ml = ws.att_ml; ap.counters = ws.att_ctr; ap.status = ws.status;
+    ap.S = attention_tc_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch, c.head_dim);
+    ap.status = ws.status;
     attention(ctx, ap);
     const int R = ps.Rq;
     {
@@ -429,9 +416,7 @@ int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, 
     ctx->head = *h;
     ctx->launches = 0;
     // counters and the status word start at zero
-    if (cudaMemsetAsync(ws.att_ctr, 0, (size_t)cfg->max_batch * cfg->n_kv_heads * d.q_tiles_max * 4, ctx->stream) !=
-            cudaSuccess ||
-        cudaMemsetAsync(ws.walk_ctr, 0, (size_t)cfg->max_batch * 4, ctx->stream) != cudaSuccess ||
+    if (cudaMemsetAsync(ws.walk_ctr, 0, (size_t)cfg->max_batch * 4, ctx->stream) != cudaSuccess ||
         cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess ||
         cudaMemsetAsync(ws.am_keys, 0, (size_t)d.Rlog * 8, ctx->stream) != cudaSuccess ||
         cudaMemsetAsync(ws.am_counter, 0, 256, ctx->stream) != cudaSuccess) {
@@ -631,8 +616,7 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     ap.q = (const bf16 *)q; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
     ap.out = (bf16 *)out; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
-    ap.part_o = ctx->ws.att_o; ap.part_ml = ctx->ws.att_ml;
-    ap.counters = ctx->ws.att_ctr; ap.status = ctx->ws.status;
+    ap.status = ctx->ws.status;
     attention(ctx, ap);
     return finish(ctx);
 }

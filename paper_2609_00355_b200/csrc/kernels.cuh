@@ -91,7 +91,7 @@ void launch_walk_commit(const WalkCommit &p, cudaStream_t st);
 void launch_prefill_advance(int32_t *seq_len, int32_t *root, int32_t *feat_count, const int32_t *argmax, int count,
                             cudaStream_t st);
 
-// ---- attention (attention.cu) -------------------------------------------------------------
+// ---- attention (attention_tc.cu) ----------------------------------------------------------
 struct AttnParams {
     int batch, T, Hq, Hkv, d;    // T = query rows per sequence = extra (uncommitted) keys per sequence
     const bf16 *q;               // [batch*T][Hq*d]
@@ -102,19 +102,13 @@ struct AttnParams {
     const uint64_t *anc;         // [batch][T][W] or nullptr (all T extra keys visible)
     int W;
     bf16 *out;                   // [batch*T][Hq*d]
-    int S;                       // key splits
-    float *part_o;               // [batch][Hkv][PR][S][d]
-    float *part_ml;              // [batch][Hkv][PR][S][2]
-    int32_t *counters;           // [batch][Hkv][q_tiles], zero between calls
+    int S;                       // key splits (= cluster size)
     int32_t *status;
     unsigned long long *trace;   // test hook: phase timestamps of the first CTA, or nullptr
 };
-void launch_attention(const AttnParams &p, cudaStream_t st);
-// tcgen05 version (attention_tc.cu): map_kv = 2-D map of the pool layer {d, n_pages*2*Hkv*64 rows}, box {64, 64}
+// map_kv = 2-D map of the pool layer {d, n_pages*2*Hkv*64 rows}, box {64, 64}
 cudaError_t launch_attention_tc(const AttnParams &p, const CUtensorMap &map_kv, cudaStream_t st);
 int attention_tc_q_tiles(int T, int G);
 int attention_tc_splits(int T, int G, int Hkv, int batch, int d);
-int attention_q_tiles(int T, int G);
-int attention_splits(int T, int G, int Hkv, int batch);   // key splits so that one wave of CTAs covers the SMs
 
 }  // namespace glance
