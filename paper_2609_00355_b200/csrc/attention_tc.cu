@@ -101,8 +101,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const int P = p.seq_len[s];
     const int n_keys = P + p.T;
     const int n_tiles = (n_keys + KT - 1) / KT;
-    const int t_begin = (int)((long long)split * n_tiles / p.S);
-    const int t_end = (int)((long long)(split + 1) * n_tiles / p.S);
+    // ceil-distribution: the extra tiles go to the first splits, because the last split already carries the
+    // costlier masked tiles and the partial page
+    const int t_begin = (int)(((long long)split * n_tiles + p.S - 1) / p.S);
+    const int t_end = (int)(((long long)(split + 1) * n_tiles + p.S - 1) / p.S);
     const int nt = t_end - t_begin;
     const int32_t *pt = p.page_table + (size_t)s * p.geom.max_pages_per_seq;
     if (warp != 0) {

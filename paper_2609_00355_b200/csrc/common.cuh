@@ -32,6 +32,7 @@ struct RowMeta {
     int32_t *seq;     // [R] sequence of the row
     int32_t *pos;     // [R] rotary position, -1 for a padding row
     long long *kvrow; // [R] element offset of the row's K slot (kv head 0) inside a pool layer, -1 = none
+    const double *inv_freq;  // [d/2] theta^(-2i/d), computed in double on the host
     float *rope_cos;  // [R][d/2]
     float *rope_sin;  // [R][d/2]
 };

@@ -1,6 +1,7 @@
 // C ABI of the GLANCE round library: context, workspace carving, and the stream-ordered sequence of
 // kernels behind each entry point declared in glance.h.
 #include <algorithm>
+#include <cmath>
 #include <map>
 #include <new>
 #include <tuple>
@@ -39,6 +40,7 @@ struct Workspace {
     long long *row_kvrow;
     float *ssq;            // [n_ssq][Rmax] per-tile sums of squares of the residual rows
     float *rope_cos, *rope_sin;
+    double *inv_freq;      // [d/2]
     uint64_t *chain_anc;   // [N][W] prefill chain mask
     bf16 *hidden_tmp;      // [N][H] prefill hidden
     int32_t *argmax_tmp;   // [N]
@@ -89,6 +91,7 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.ssq = (float *)take((size_t)d.n_ssq * R * 4);
     w.rope_cos = (float *)take(R * (c.head_dim / 2) * 4);
     w.rope_sin = (float *)take(R * (c.head_dim / 2) * 4);
+    w.inv_freq = (double *)take((size_t)(c.head_dim / 2) * 8);
     w.chain_anc = (uint64_t *)take((size_t)c.tree_N * d.W * 8);
     w.hidden_tmp = (bf16 *)take((size_t)c.tree_N * H * 2);
     w.argmax_tmp = (int32_t *)take((size_t)c.tree_N * 4);
@@ -135,6 +138,7 @@ struct glance_ctx {
     // TMA descriptors, keyed by (base, inner extent, rows, box rows); built on first use by a host-only call
     std::map<std::tuple<const void *, int, int, int>, CUtensorMap> maps;
     bool map_error = false;
+    std::vector<double> inv_freq_host;   // staged for the one-time upload at creation
     // test hook: phase timestamps of successive GEMM launches, 16 words each, ring of trace_slots launches
     unsigned long long *trace = nullptr;
     int trace_slots = 0, trace_next = 0;
@@ -247,6 +251,7 @@ RowMeta meta_of(const glance_ctx *ctx) {
     m.seq = ctx->ws.row_seq;
     m.pos = ctx->ws.row_pos;
     m.kvrow = ctx->ws.row_kvrow;
+    m.inv_freq = ctx->ws.inv_freq;
     m.rope_cos = ctx->ws.rope_cos;
     m.rope_sin = ctx->ws.rope_sin;
     return m;
@@ -415,6 +420,15 @@ int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, 
     }
     ctx->head = *h;
     ctx->launches = 0;
+    // rotary frequencies theta^(-2i/d) in double, uploaded once
+    ctx->inv_freq_host.resize(cfg->head_dim / 2);
+    for (int i = 0; i < cfg->head_dim / 2; ++i)
+        ctx->inv_freq_host[i] = std::pow((double)cfg->rope_theta, -(2.0 * i) / (double)cfg->head_dim);
+    if (cudaMemcpyAsync(ws.inv_freq, ctx->inv_freq_host.data(), ctx->inv_freq_host.size() * 8, cudaMemcpyHostToDevice,
+                        ctx->stream) != cudaSuccess) {
+        delete ctx;
+        return GLANCE_E_CUDA;
+    }
     // counters and the status word start at zero
     if (cudaMemsetAsync(ws.walk_ctr, 0, (size_t)cfg->max_batch * 4, ctx->stream) != cudaSuccess ||
         cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess ||

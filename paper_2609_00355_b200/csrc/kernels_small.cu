@@ -5,19 +5,25 @@ namespace glance {
 
 // ------------------------------------------------------------------------------------------
 // Row setup shared by the verify and draft passes.  One block per row:
-//   * rotary table of the row: angle = pos * theta^(-2i/d), evaluated in double
+//   * rotary table of the row: angle = pos * theta^(-2i/d), argument reduction in double
 //   * element offset of the row's K slot (kv head 0) inside a layer of the paged pool
 //   * fp32 residual row x, its bf16 copy scaled by the first norm's gain, and its sum of squares
 //     (the consumer GEMM multiplies its results by 1/rms, so no separate normalisation pass exists)
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ void fill_rope_row(const RowMeta &m, int r, int pos, int d, float theta) {
+    // angle = pos * theta^(-2i/d): the product and its reduction modulo 2 pi are done in double (a handful of
+    // FP64 instructions) with the per-dimension frequencies precomputed in double on the host; the reduced
+    // angle lies in [-pi, pi], where single-precision sincos is accurate to ~1e-7.
+    (void)theta;
     const int half = d >> 1;
     for (int i = threadIdx.x; i < half; i += blockDim.x) {
-        double inv = pow((double)theta, -(2.0 * i) / (double)d);
-        double s, c;
-        sincos((double)pos * inv, &s, &c);
-        m.rope_cos[(size_t)r * half + i] = (float)c;
-        m.rope_sin[(size_t)r * half + i] = (float)s;
+        const double x = (double)pos * m.inv_freq[i];
+        const double k = rint(x * 0.15915494309189535);           // 1 / (2 pi)
+        const double red = fma(-k, 1.2246467991473532e-16 * 2.0, fma(-k, 6.283185307179586, x));
+        float s, c;
+        sincosf((float)red, &s, &c);
+        m.rope_cos[(size_t)r * half + i] = c;
+        m.rope_sin[(size_t)r * half + i] = s;
     }
 }
 
@@ -33,15 +39,45 @@ __device__ __forceinline__ long long kv_row_offset(const KvGeom &g, const int32_
 
 // x[c] = src[c] (or 0), xb[c] = bf16(x[c] * gain[c]), ssq[0][r] = sum x^2, ssq[i>0][r] = 0
 __device__ __forceinline__ void emit_row(const RowOut &o, int r, const bf16 *src, const bf16 *gain) {
+    // H is a multiple of 64: the row is handled in 16-byte groups of eight bf16, up to four groups per thread
+    // with all loads issued before the first use (the source row usually comes from HBM)
     __shared__ float red[4];
     float *x = o.x + (size_t)r * o.H;
     bf16 *xb = o.xb + (size_t)r * o.H;
+    const int groups = o.H >> 3;
     float ss = 0.f;
-    for (int c = threadIdx.x; c < o.H; c += blockDim.x) {
-        const float v = src ? __bfloat162float(src[c]) : 0.f;
-        x[c] = v;
-        xb[c] = __float2bfloat16(v * __bfloat162float(gain[c]));
-        ss += v * v;
+    for (int g0 = threadIdx.x; g0 < groups; g0 += 4 * blockDim.x) {
+        uint4 raw[4], gn[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int g = g0 + u * blockDim.x;
+            raw[u] = make_uint4(0, 0, 0, 0);
+            gn[u] = make_uint4(0, 0, 0, 0);
+            if (g < groups) {
+                if (src) raw[u] = *reinterpret_cast<const uint4 *>(src + g * 8);
+                gn[u] = *reinterpret_cast<const uint4 *>(gain + g * 8);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int g = g0 + u * blockDim.x;
+            if (g >= groups) continue;
+            const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&raw[u]);
+            const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gn[u]);
+            float f[8];
+            uint32_t ob[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                f[2 * j] = __low2float(v2[j]);
+                f[2 * j + 1] = __high2float(v2[j]);
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * j] * __low2float(g2[j]), f[2 * j + 1] * __high2float(g2[j]));
+                ob[j] = *reinterpret_cast<uint32_t *>(&h2);
+                ss += f[2 * j] * f[2 * j] + f[2 * j + 1] * f[2 * j + 1];
+            }
+            *reinterpret_cast<float4 *>(x + g * 8) = make_float4(f[0], f[1], f[2], f[3]);
+            *reinterpret_cast<float4 *>(x + g * 8 + 4) = make_float4(f[4], f[5], f[6], f[7]);
+            *reinterpret_cast<uint4 *>(xb + g * 8) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+        }
     }
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
