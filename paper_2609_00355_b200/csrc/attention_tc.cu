@@ -360,21 +360,18 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         // ---------------- epilogue ----------------
         if (p.S == 1 && ok) {
             const float inv = 1.f / l_row;
-            bf16 *dst = p.out + ((size_t)(s * p.T + node) * p.Hq + kvh * G + g) * D + cg * OC;
+            const size_t off = ((size_t)(s * p.T + node) * p.Hq + kvh * G + g) * D + cg * OC;
 #pragma unroll
             for (int c = 0; c < OC; c += 16) {
                 uint32_t v[16];
                 tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
                 tmem_ld_wait();
                 if (row_valid) {
-                    uint32_t w[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(v[2 * j]) * inv, __uint_as_float(v[2 * j + 1]) * inv);
-                        w[j] = *reinterpret_cast<uint32_t *>(&h2);
-                    }
-                    *reinterpret_cast<uint4 *>(dst + c) = make_uint4(w[0], w[1], w[2], w[3]);
-                    *reinterpret_cast<uint4 *>(dst + c + 8) = make_uint4(w[4], w[5], w[6], w[7]);
+                    for (int j = 0; j < 16; j += 4)
+                        store_two_term(p.out + off + c + j, p.out_lo ? p.out_lo + off + c + j : nullptr,
+                                       make_float4(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv,
+                                                   __uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv));
                 }
             }
         }
@@ -448,12 +445,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 }
                 const float inv = 1.f / den;
                 const int prr = qt * QT + row_lo + lr;
-                bf16 *dst = p.out + ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c0;
-                __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-                uint2 o;
-                o.x = *reinterpret_cast<uint32_t *>(&lo);
-                o.y = *reinterpret_cast<uint32_t *>(&hi);
-                *reinterpret_cast<uint2 *>(dst) = o;
+                const size_t off = ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c0;
+                store_two_term(p.out + off, p.out_lo ? p.out_lo + off : nullptr,
+                               make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
             }
         }
     }

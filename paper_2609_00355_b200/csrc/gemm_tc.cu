@@ -53,8 +53,11 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     // MODE 1 stacks 64 gate rows and the matching 64 up rows into one 128-row weight tile (two TMA boxes)
     constexpr int FT = (MODE == 1) ? 64 : BM;            // output features per CTA
     constexpr bool CLUSTERED = (MODE >= 3);
-    const int NP = a.np;                                 // UMMA N (activation rows, padded to 16)
-    const int stage_bytes = BM * 128 + NP * 128;
+    const int NP = a.np;                                 // activation rows per CTA, padded to 16
+    // With two-term activations (x = hi + lo, both bf16) the lo rows ride along as NP more rows of the B
+    // operand: the accumulator gets NP more columns, which the epilogue adds to the first NP.
+    const int NB = a.x_lo_row > 0 ? 2 * NP : NP;         // UMMA N
+    const int stage_bytes = BM * 128 + NB * 128;
     const int stages = a.stages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int f0 = blockIdx.x * FT;
@@ -113,7 +116,11 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
             pdl_wait();
             if (trace) trace[2] = global_ns();
             for (int i = 0; i < pre; ++i)
-                tma_load_2d(smem + (size_t)i * stage_bytes + BM * 128, &map_x, &bars.full[i], (kt0 + i) * BK, r0);
+            {
+                unsigned char *xs = smem + (size_t)i * stage_bytes + BM * 128;
+                tma_load_2d(xs, &map_x, &bars.full[i], (kt0 + i) * BK, r0);
+                if (NB > NP) tma_load_2d(xs + NP * 128, &map_x, &bars.full[i], (kt0 + i) * BK, a.x_lo_row + r0);
+            }
             int issued = pre;
             for (int i = pre; i < nk; ++i) {
                 const int s = i % stages;
@@ -123,6 +130,7 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                 mbar_expect_tx(&bars.full[s], (uint32_t)stage_bytes);
                 load_w(i, slot, &bars.full[s]);
                 tma_load_2d(slot + BM * 128, &map_x, &bars.full[s], (kt0 + i) * BK, r0);
+                if (NB > NP) tma_load_2d(slot + BM * 128 + NP * 128, &map_x, &bars.full[s], (kt0 + i) * BK, a.x_lo_row + r0);
                 issued = i + 1;
             }
             if (*abort_flag) {
@@ -137,7 +145,7 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc(NP);
+            const uint32_t idesc = umma_idesc(NB);
             bool mok = true;
             for (int i = 0; i < nk && mok; ++i) {
                 const int s = i % stages;
@@ -197,7 +205,15 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
             uint32_t v[16];
             if (nk > 0 && ok) {
                 tmem_ld16(lane_addr + (uint32_t)c, v);
-                tmem_ld_wait();
+                if (NB > NP) {                           // hi part + lo part of the two-term activations
+                    uint32_t w[16];
+                    tmem_ld16(lane_addr + (uint32_t)(NP + c), w);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+                } else {
+                    tmem_ld_wait();
+                }
             } else {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = 0u;
@@ -266,12 +282,9 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                 const int f = f0 + fg;
                 if (f < a.F) {          // F is a multiple of 4
                     const float g0 = g.x * sc, g1 = g.y * sc, g2 = g.z * sc, g3 = g.w * sc;
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(g0 / (1.f + __expf(-g0)) * (u.x * sc), g1 / (1.f + __expf(-g1)) * (u.y * sc));
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(g2 / (1.f + __expf(-g2)) * (u.z * sc), g3 / (1.f + __expf(-g3)) * (u.w * sc));
-                    uint2 o;
-                    o.x = *reinterpret_cast<uint32_t *>(&lo);
-                    o.y = *reinterpret_cast<uint32_t *>(&hi);
-                    *reinterpret_cast<uint2 *>(a.act + (size_t)(r0 + r) * a.F + f) = o;
+                    const float4 val = make_float4(g0 / (1.f + __expf(-g0)) * (u.x * sc), g1 / (1.f + __expf(-g1)) * (u.y * sc),
+                                                   g2 / (1.f + __expf(-g2)) * (u.z * sc), g3 / (1.f + __expf(-g3)) * (u.w * sc));
+                    store_two_term(a.act + (size_t)(r0 + r) * a.F + f, a.act_lo ? a.act_lo + (size_t)(r0 + r) * a.F + f : nullptr, val);
                 }
             }
         } else if (MODE == 3) {
@@ -297,15 +310,12 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                 if (valid) {
                     xv.x += v.x; xv.y += v.y; xv.z += v.z; xv.w += v.w;
                     *reinterpret_cast<float4 *>(a.x + o) = xv;
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(xv.x * gain.x, xv.y * gain.y);
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(xv.z * gain.z, xv.w * gain.w);
-                    uint2 ob;
-                    ob.x = *reinterpret_cast<uint32_t *>(&lo);
-                    ob.y = *reinterpret_cast<uint32_t *>(&hi);
-                    *reinterpret_cast<uint2 *>(a.xb + o) = ob;
+                    store_two_term(a.xb + o, a.xb_lo ? a.xb_lo + o : nullptr,
+                                   make_float4(xv.x * gain.x, xv.y * gain.y, xv.z * gain.z, xv.w * gain.w));
                     if (a.hidden_out) {
-                        lo = __floats2bfloat162_rn(xv.x, xv.y);
-                        hi = __floats2bfloat162_rn(xv.z, xv.w);
+                        uint2 ob;
+                        __nv_bfloat162 lo = __floats2bfloat162_rn(xv.x, xv.y);
+                        __nv_bfloat162 hi = __floats2bfloat162_rn(xv.z, xv.w);
                         ob.x = *reinterpret_cast<uint32_t *>(&lo);
                         ob.y = *reinterpret_cast<uint32_t *>(&hi);
                         *reinterpret_cast<uint2 *>(a.hidden_out + o) = ob;
@@ -459,7 +469,8 @@ int tc_row_pad(int R) {
 
 cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, const CUtensorMap &map_x, cudaStream_t st) {
     a.np = tc_row_pad(a.R);
-    const int stage_bytes = BM * 128 + a.np * 128;
+    const int nb = a.x_lo_row > 0 ? 2 * a.np : a.np;
+    const int stage_bytes = BM * 128 + nb * 128;
     // The ring stays under half of an SM's shared memory so that two CTAs fit per SM: a GPC then offers enough
     // CTA slots for every cluster of a launch to be resident in one wave, and one CTA's prologue and epilogue
     // overlap the other's streaming.
@@ -467,7 +478,7 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     stages = stages > 12 ? 12 : (stages < 2 ? 2 : stages);
     a.stages = stages;
     uint32_t cols = 32;
-    while ((int)cols < a.np) cols <<= 1;
+    while ((int)cols < nb) cols <<= 1;
     a.tmem_cols = cols;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     const int tiles = mode == 1 ? (a.F + 63) / 64 : (a.Nout + BM - 1) / BM;

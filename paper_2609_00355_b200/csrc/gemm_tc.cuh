@@ -7,13 +7,14 @@
 namespace glance {
 
 struct TcGemmArgs {
-    int Nout, K, R, S;          // W [Nout][K], X [R][K]; S = split-K factor (mode 0 only; 1 otherwise)
+    int Nout, K, R, S;          // W [Nout][K], X [R][K]; S = split-K factor (modes 0, 3, 4; 1 otherwise)
+    int x_lo_row;               // > 0: X is two-term (hi + lo, both bf16); the lo plane starts at this row of the X map
     // mode 0: fp32 planes Y[split][r][f]; mode 2: optional fp32 logits Y[r][f] (may be nullptr)
     float *Y;
     int ldy;
     size_t split_stride;
     // mode 1 (SwiGLU): W holds F gate rows then F up rows; act[r][f] = silu(gate) * up
-    bf16 *act;
+    bf16 *act, *act_lo;         // act_lo: second term of the two-term output, or nullptr
     int F;
     // mode 2 (arg-max over f): keys[r] packed (value, id) merged with atomicMax; the last CTA writes argmax[r]
     unsigned long long *keys;
@@ -27,7 +28,7 @@ struct TcGemmArgs {
     // mode 3 (residual): x[r][f] += result; xb = bf16(x * gain[f]); ssq_out[tile][r] = sum over the tile of x^2
     float *x;
     const bf16 *gain;
-    bf16 *xb, *hidden_out;
+    bf16 *xb, *xb_lo, *hidden_out;
     float *ssq_out;
     // mode 4 (rotary + K/V write): features are q heads, then k heads, then v heads, head_dim wide
     bf16 *q;

@@ -30,7 +30,7 @@ int choose_split(int Nout, int K, int rows) {
 
 struct Workspace {
     float *x;            // [Rmax][H] residual stream
-    bf16 *xn;            // [Rmax][H]
+    bf16 *xn;            // [2][Rmax][H] bf16(x * gain) as two terms (hi plane, lo plane); so are attn and act
     bf16 *q;             // [Rmax][Hq d]
     bf16 *attn;          // [Rmax][Hq d]
     bf16 *act;           // [Rmax][F]
@@ -79,10 +79,10 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     };
     const size_t R = d.Rmax, H = c.hidden;
     w.x = (float *)take(R * H * 4);
-    w.xn = (bf16 *)take(R * H * 2);
+    w.xn = (bf16 *)take(2 * R * H * 2);                 // two planes: hi, lo
     w.q = (bf16 *)take(R * d.qd * 2);
-    w.attn = (bf16 *)take(R * d.qd * 2);
-    w.act = (bf16 *)take(R * (size_t)c.ffn * 2);
+    w.attn = (bf16 *)take(2 * R * d.qd * 2);            // two planes
+    w.act = (bf16 *)take(2 * R * (size_t)c.ffn * 2);    // two planes
     w.logits = (float *)take((size_t)d.Rlog * c.vocab * 4);
     w.walk_ctr = (int32_t *)take((size_t)c.max_batch * 4);
     w.row_seq = (int32_t *)take(R * 4);
@@ -187,7 +187,7 @@ const CUtensorMap *get_map(glance_ctx *ctx, const void *base, int inner, int row
 // allocated behind X) and W [Nout][K], and tallies its algorithmic bytes.
 void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, TcGemmArgs a) {
     const CUtensorMap *mw = get_map(ctx, W, a.K, a.Nout, mode == 1 ? 64 : 128);
-    const CUtensorMap *mx = get_map(ctx, X, a.K, x_rows, tc_row_pad(a.R));
+    const CUtensorMap *mx = get_map(ctx, X, a.K, a.x_lo_row > 0 ? 2 * x_rows : x_rows, tc_row_pad(a.R));
     if (!mw || !mx) return;
     a.keys = ctx->ws.am_keys; a.counter = ctx->ws.am_counter; a.status = ctx->ws.status;
     if (ctx->trace && ctx->trace_slots > 0) {
@@ -262,6 +262,7 @@ RowOut rowout_of(const glance_ctx *ctx) {
     o.H = ctx->cfg.hidden;
     o.x = ctx->ws.x;
     o.xb = ctx->ws.xn;
+    o.xb_lo = ctx->ws.xn + (size_t)ctx->dims.Rmax * ctx->cfg.hidden;
     o.ssq = ctx->ws.ssq;
     o.n_ssq = ctx->dims.n_ssq;
     o.ssq_stride = ctx->dims.Rmax;
@@ -287,6 +288,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
         TcGemmArgs g{};
         g.Nout = d.qkv_out; g.K = c.hidden; g.R = ps.R; g.S = choose_split(d.qkv_out, c.hidden, ps.R);
         with_row_scales(ctx, g);
+        g.x_lo_row = xr;
         g.q = ws.q; g.pool_layer = pool_layer; g.kvrow = ws.row_kvrow;
         g.v_off = (size_t)c.n_kv_heads * kPage * c.head_dim; g.head_stride = (size_t)kPage * c.head_dim;
         g.rope_cos = ws.rope_cos; g.rope_sin = ws.rope_sin;
@@ -297,7 +299,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     AttnParams ap;
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
-    ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn;
+    ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn; ap.out_lo = ws.attn + (size_t)xr * d.qd;
     ap.S = attention_tc_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch, c.head_dim);
     ap.status = ws.status;
     attention(ctx, ap);
@@ -305,19 +307,22 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     {
         TcGemmArgs g{};
         g.Nout = c.hidden; g.K = d.qd; g.R = R; g.S = choose_split(c.hidden, d.qd, R);
-        g.x = ws.x; g.gain = w.ln2; g.xb = ws.xn; g.ssq_out = ws.ssq; g.ssq_stride = d.Rmax;
+        g.x = ws.x; g.gain = w.ln2; g.xb = ws.xn; g.xb_lo = ws.xn + (size_t)xr * c.hidden; g.ssq_out = ws.ssq;
+        g.ssq_stride = d.Rmax; g.x_lo_row = xr;
         gemm(ctx, 3, w.wo, ws.attn, xr, g);
     }
     {
         TcGemmArgs g{};
-        g.Nout = 2 * c.ffn; g.K = c.hidden; g.R = R; g.S = 1; g.act = ws.act; g.F = c.ffn;
+        g.Nout = 2 * c.ffn; g.K = c.hidden; g.R = R; g.S = 1; g.act = ws.act; g.act_lo = ws.act + (size_t)xr * c.ffn;
+        g.F = c.ffn; g.x_lo_row = xr;
         with_row_scales(ctx, g);
         gemm(ctx, 1, w.wgu, ws.xn, xr, g);
     }
     {
         TcGemmArgs g{};
         g.Nout = c.hidden; g.K = c.ffn; g.R = R; g.S = choose_split(c.hidden, c.ffn, R);
-        g.x = ws.x; g.gain = next_gain; g.xb = ws.xn; g.hidden_out = hidden_out; g.ssq_out = ws.ssq; g.ssq_stride = d.Rmax;
+        g.x = ws.x; g.gain = next_gain; g.xb = ws.xn; g.xb_lo = ws.xn + (size_t)xr * c.hidden; g.hidden_out = hidden_out;
+        g.ssq_out = ws.ssq; g.ssq_stride = d.Rmax; g.x_lo_row = xr;
         gemm(ctx, 3, w.wd, ws.act, xr, g);
     }
 }
@@ -335,6 +340,7 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
     if (argmax) {   // logits are stored only on request
         TcGemmArgs g{};
         g.Nout = c.vocab; g.K = c.hidden; g.R = ps.R; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.argmax = argmax;
+        g.x_lo_row = ctx->dims.Rmax;
         with_row_scales(ctx, g);
         gemm(ctx, 2, ctx->lm_head, ctx->ws.xn, ctx->dims.Rmax, g);
     }
@@ -530,6 +536,7 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
     {
         TcGemmArgs g{};
         g.Nout = c.vocab; g.K = c.hidden; g.R = R1; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.split_stride = 0;
+        g.x_lo_row = ctx->dims.Rmax;
         with_row_scales(ctx, g);
         gemm(ctx, 0, ctx->lm_head, ws.xn, ctx->dims.Rmax, g);
     }
@@ -629,7 +636,7 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     ap.batch = seqs->batch; ap.T = T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
     ap.q = (const bf16 *)q; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
-    ap.out = (bf16 *)out; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
+    ap.out = (bf16 *)out; ap.out_lo = nullptr; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
     ap.status = ctx->ws.status;
     attention(ctx, ap);
     return finish(ctx);

@@ -11,7 +11,8 @@ namespace glance {
 struct RowOut {
     int H;
     float *x;            // [R][H]
-    bf16 *xb;            // [R][H]
+    bf16 *xb;            // [R][H] first term of bf16(x * gain)
+    bf16 *xb_lo;         // [R][H] second term (x * gain - first term), or nullptr
     float *ssq;          // [n_ssq][ssq_stride]: plane 0 gets the row's full sum of squares, the others 0
     int n_ssq, ssq_stride;
 };
@@ -102,6 +103,7 @@ struct AttnParams {
     const uint64_t *anc;         // [batch][T][W] or nullptr (all T extra keys visible)
     int W;
     bf16 *out;                   // [batch*T][Hq*d]
+    bf16 *out_lo;                // second term of the two-term output, or nullptr
     int S;                       // key splits (= cluster size)
     int32_t *status;
     unsigned long long *trace;   // test hook: phase timestamps of the first CTA, or nullptr

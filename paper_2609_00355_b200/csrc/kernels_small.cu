@@ -1,5 +1,6 @@
 // Row setup, normalisation, rotary + paged K/V write, SwiGLU, argmax and top-k kernels of the round.
 #include "kernels.cuh"
+#include "tc_ptx.cuh"
 
 namespace glance {
 
@@ -44,6 +45,7 @@ __device__ __forceinline__ void emit_row(const RowOut &o, int r, const bf16 *src
     __shared__ float red[4];
     float *x = o.x + (size_t)r * o.H;
     bf16 *xb = o.xb + (size_t)r * o.H;
+    bf16 *xl = o.xb_lo ? o.xb_lo + (size_t)r * o.H : nullptr;
     const int groups = o.H >> 3;
     float ss = 0.f;
     for (int g0 = threadIdx.x; g0 < groups; g0 += 4 * blockDim.x) {
@@ -64,19 +66,19 @@ __device__ __forceinline__ void emit_row(const RowOut &o, int r, const bf16 *src
             if (g >= groups) continue;
             const __nv_bfloat162 *v2 = reinterpret_cast<const __nv_bfloat162 *>(&raw[u]);
             const __nv_bfloat162 *g2 = reinterpret_cast<const __nv_bfloat162 *>(&gn[u]);
-            float f[8];
-            uint32_t ob[4];
+            float f[8], sg[8];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 f[2 * j] = __low2float(v2[j]);
                 f[2 * j + 1] = __high2float(v2[j]);
-                __nv_bfloat162 h2 = __floats2bfloat162_rn(f[2 * j] * __low2float(g2[j]), f[2 * j + 1] * __high2float(g2[j]));
-                ob[j] = *reinterpret_cast<uint32_t *>(&h2);
+                sg[2 * j] = f[2 * j] * __low2float(g2[j]);
+                sg[2 * j + 1] = f[2 * j + 1] * __high2float(g2[j]);
                 ss += f[2 * j] * f[2 * j] + f[2 * j + 1] * f[2 * j + 1];
             }
             *reinterpret_cast<float4 *>(x + g * 8) = make_float4(f[0], f[1], f[2], f[3]);
             *reinterpret_cast<float4 *>(x + g * 8 + 4) = make_float4(f[4], f[5], f[6], f[7]);
-            *reinterpret_cast<uint4 *>(xb + g * 8) = make_uint4(ob[0], ob[1], ob[2], ob[3]);
+            tc::store_two_term(xb + g * 8, xl ? xl + g * 8 : nullptr, make_float4(sg[0], sg[1], sg[2], sg[3]));
+            tc::store_two_term(xb + g * 8 + 4, xl ? xl + g * 8 + 4 : nullptr, make_float4(sg[4], sg[5], sg[6], sg[7]));
         }
     }
     ss = warp_sum(ss);

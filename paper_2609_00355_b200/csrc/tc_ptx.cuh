@@ -141,6 +141,23 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
           "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]) : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Two-term bf16 representation of four fp32 values: hi = bf16(v), lo = bf16(v - hi).  hi + lo carries about 16
+// mantissa bits, so activations that feed a GEMM lose almost nothing to rounding.  lo may be nullptr.
+__device__ __forceinline__ void store_two_term(bf16 *hi, bf16 *lo, float4 v) {
+    __nv_bfloat162 h01 = __floats2bfloat162_rn(v.x, v.y), h23 = __floats2bfloat162_rn(v.z, v.w);
+    uint2 o;
+    o.x = *reinterpret_cast<uint32_t *>(&h01);
+    o.y = *reinterpret_cast<uint32_t *>(&h23);
+    *reinterpret_cast<uint2 *>(hi) = o;
+    if (lo) {
+        __nv_bfloat162 l01 = __floats2bfloat162_rn(v.x - __low2float(h01), v.y - __high2float(h01));
+        __nv_bfloat162 l23 = __floats2bfloat162_rn(v.z - __low2float(h23), v.w - __high2float(h23));
+        o.x = *reinterpret_cast<uint32_t *>(&l01);
+        o.y = *reinterpret_cast<uint32_t *>(&l23);
+        *reinterpret_cast<uint2 *>(lo) = o;
+    }
+}
+
 // makes generic-proxy shared-memory writes visible to the async proxy (TMA / tcgen05.mma operand reads)
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
