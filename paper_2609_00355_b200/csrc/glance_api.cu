@@ -288,7 +288,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
         TcGemmArgs g{};
         g.Nout = d.qkv_out; g.K = c.hidden; g.R = ps.R; g.S = choose_split(d.qkv_out, c.hidden, ps.R);
         with_row_scales(ctx, g);
-        g.x_lo_row = xr;
+        g.x_lo_row = 0;      // q, K, V are rounded to bf16 right after: the second term of x would buy nothing
         g.q = ws.q; g.pool_layer = pool_layer; g.kvrow = ws.row_kvrow;
         g.v_off = (size_t)c.n_kv_heads * kPage * c.head_dim; g.head_stride = (size_t)kPage * c.head_dim;
         g.rope_cos = ws.rope_cos; g.rope_sin = ws.rope_sin;
@@ -340,7 +340,7 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
     if (argmax) {   // logits are stored only on request
         TcGemmArgs g{};
         g.Nout = c.vocab; g.K = c.hidden; g.R = ps.R; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.argmax = argmax;
-        g.x_lo_row = ctx->dims.Rmax;
+        g.x_lo_row = 0;      // logits only decide an arg-max / top-k: one term is enough
         with_row_scales(ctx, g);
         gemm(ctx, 2, ctx->lm_head, ctx->ws.xn, ctx->dims.Rmax, g);
     }
@@ -536,7 +536,7 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
     {
         TcGemmArgs g{};
         g.Nout = c.vocab; g.K = c.hidden; g.R = R1; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.split_stride = 0;
-        g.x_lo_row = ctx->dims.Rmax;
+        g.x_lo_row = 0;
         with_row_scales(ctx, g);
         gemm(ctx, 0, ctx->lm_head, ws.xn, ctx->dims.Rmax, g);
     }
