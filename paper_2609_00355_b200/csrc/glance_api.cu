@@ -16,14 +16,14 @@ namespace {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// split-K factor of a weight-streaming GEMM: as many CTAs as fit one wave of the 148 SMs, at least 8 k-tiles
-// per split
+// split-K factor of a weight-streaming GEMM: as many CTAs as fit one wave at two CTAs per SM (one CTA per SM
+// keeps too few weight bytes in flight to cover the HBM latency), at least 8 k-tiles per split
 // The splits of one tile form a thread-block cluster (<= 8 CTAs) that reduces them through shared memory.
 int choose_split(int Nout, int K, int rows) {
     const int tiles = (Nout + 127) / 128;
     const int ktiles = K / 64;
     (void)rows;
-    int s = 148 / tiles;
+    int s = (2 * 148) / tiles;
     s = std::min(s, std::max(1, ktiles / 8));
     return std::max(1, std::min(s, 8));
 }
