@@ -27,6 +27,12 @@ constexpr int QT = 128;          // packed query rows per CTA (UMMA M)
 constexpr int KT = kPage;        // keys per tile (UMMA N of S, K of P V)
 constexpr int MAX_SPLITS = 8;     // the splits of a tile form one thread-block cluster
 constexpr float kRescaleThreshold = 8.f;   // log2 units
+
+__device__ __forceinline__ float ex2_approx(float x) {   // 2^x, hardware approximation; 2^-inf = +0
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 constexpr int NSOFT = 512;       // softmax / epilogue threads (16 warps)
 constexpr int NTHREADS = 64 + NSOFT;
 
@@ -273,6 +279,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
                 for (int j = 0; j < 16; ++j) sc[j] = __uint_as_float(v[j]);
             }
+            if (trace && threadIdx.x == 64 && i == 0) trace[12] = global_ns();
             const bool need_mask = key0 + KT > P;
             float mt = -INFINITY;
 #pragma unroll
@@ -293,8 +300,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             }
             // row maximum of the tile across the four column groups
             red[i & 1][cg][row] = mt;
-            asm volatile("bar.sync 1, 512;" ::: "memory");
-            if (*abort_flag) break;                       // uniform across the 16 warps: read right after the barrier
+            asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");   // only the four warps of this lane quarter share rows
+            if (trace && threadIdx.x == 64 && i == 0) trace[13] = global_ns();
+            if (*abort_flag) break;                       // a quarter that leaves stops arriving at p_full: every wait is bounded
             mt = fmaxf(fmaxf(red[i & 1][0][row], red[i & 1][1][row]), fmaxf(red[i & 1][2][row], red[i & 1][3][row]));
             if (i > 0) {
                 // P and O are in use by the previous tile's second MMA until o_done
@@ -325,14 +333,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             // P = 2^(S' - m_ref), bf16: this thread's 16 keys = two 16-byte chunks of its row of the A operand
             float rs = 0.f;
             unsigned char *prow = sP + row * 128;
+            const float m_sub = (m_ref == -INFINITY) ? 0.f : m_ref;   // a fully masked row keeps -inf - 0 = -inf -> 2^-inf = 0
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
                 uint32_t w[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float a = sc[c * 8 + 2 * j], b = sc[c * 8 + 2 * j + 1];
-                    const float pa = (a == -INFINITY) ? 0.f : exp2f(a - m_ref);
-                    const float pb = (b == -INFINITY) ? 0.f : exp2f(b - m_ref);
+                    const float pa = ex2_approx(a - m_sub);
+                    const float pb = ex2_approx(b - m_sub);
                     rs += pa + pb;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
                     w[j] = *reinterpret_cast<uint32_t *>(&h2);
@@ -340,6 +349,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 *reinterpret_cast<uint4 *>(prow + (((cg * 2 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
             l_run += rs;
+            if (trace && threadIdx.x == 64 && i == 0) trace[14] = global_ns();
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bars.p_full);                    // always arrive: the MMA issuer counts 512 arrivals
