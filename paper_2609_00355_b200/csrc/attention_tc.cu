@@ -42,12 +42,16 @@ struct Smem {
     static constexpr int Q_BYTES = SLABS * QT * 128;     // 32 KB at d = 128
     static constexpr int KV_BYTES = SLABS * KT * 128;    // one K or V page: 16 KB at d = 128
     static constexpr int P_BYTES = QT * 128;             // 128 rows x 64 keys bf16
-    static constexpr int TOTAL = Q_BYTES + 4 * KV_BYTES + P_BYTES + 1024;
+    static constexpr int OPER_BYTES = Q_BYTES + 4 * KV_BYTES + P_BYTES;   // operand buffers (and merge staging)
+    static constexpr int ROWF = D + 4;                   // floats per merged row: O, m, l, padding
+    // split merge: rows received from the cluster's CTAs (each owner gets <= ceil(QT/S) rows from each of S CTAs)
+    static constexpr int RECV_BYTES = (QT + MAX_SPLITS) * ROWF * 4;
+    static constexpr int TOTAL = OPER_BYTES + RECV_BYTES + 1024;
     static constexpr uint32_t TMEM_COLS = 256;           // two S buffers (2 x 64) + O (d)
 };
 
 struct alignas(8) AttnBars {
-    uint64_t q_ready, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full, o_done;
+    uint64_t q_ready, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full, o_done, merge;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -85,15 +89,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         }
         mbar_init(&bars.p_full, NSOFT);
         mbar_init(&bars.o_done, 1);
+        mbar_init(&bars.merge, 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (p.S > 1) {
+            // split merge: this CTA owns a band of the tile's rows and receives that band from each of the S CTAs
+            const int rpc = (QT + p.S - 1) / p.S;
+            const int mine = max(0, min(rpc, QT - (int)cluster_rank() * rpc));
+            if (mine > 0) mbar_expect_tx(&bars.merge, (uint32_t)(p.S * mine * Smem<D>::ROWF * 4));
+        }
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&bars.tmem_base)), "r"(Smem<D>::TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
-    __syncthreads();
+    if (p.S > 1) cluster_sync_all();                     // peers' merge barriers exist before anybody can signal them
+    else __syncthreads();
     tc_fence_after();
     const uint32_t tmem_S = bars.tmem_base, tmem_O = bars.tmem_base + 128;   // S is double-buffered: columns 0-63, 64-127
     volatile int *abort_flag = &bars.abort_flag;
@@ -393,23 +405,24 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 
     if (p.S > 1) {
         // ---------------- merge of the key splits inside the cluster (reduce-scatter by rows) ----------------
-        // The S CTAs of one (sequence, kv head, q tile) form a cluster.  CTA `rank` owns rows [rank*RPC, +RPC):
-        // every CTA ships, per row, its unnormalised O row and (m, l) to the owner's shared memory (on top of
-        // the idle Q/K/V buffers), the owner combines the S partial rows in split order.
-        constexpr int ROWF = D + 4;                       // floats per shipped row: O, m, l, padding
+        // The S CTAs of one (sequence, kv head, q tile) form a cluster.  CTA `rank` owns rows [rank*RPC, +RPC).
+        // Every CTA stages its unnormalised O rows with (m, l) in its own (now idle) operand buffers, then one
+        // asynchronous shared-to-shared copy per owner ships that owner's band into the owner's receive region
+        // and counts its bytes on the owner's merge barrier; the owner combines the S bands in split order.
+        constexpr int ROWF = Smem<D>::ROWF;
         constexpr int OC = D / 4;
         const int RPC = (QT + p.S - 1) / p.S;
         const uint32_t rank = cluster_rank();
+        float *stage = reinterpret_cast<float *>(smem);
+        unsigned char *recv = smem + Smem<D>::OPER_BYTES;
         if (trace && threadIdx.x == 64) trace[7] = global_ns();
-        cluster_sync_all();                               // all MMAs of the cluster are done: buffers are idle
-        if (trace && threadIdx.x == 64) trace[8] = global_ns();
         if (warp >= 2) {
+            // this CTA's MMAs have all completed (o_done above) and every page it asked for has been consumed
             const int q = warp & 3, cg = (warp - 2) >> 2;
             const int row = q * 32 + lane;
             const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-            const uint32_t owner = (uint32_t)(row / RPC);
-            const uint32_t dst = map_to_rank(smem_u32(smem) + (uint32_t)(((rank * RPC + (row - owner * RPC)) * ROWF) * 4), owner);
             const bool live = nt > 0 && sm_ok;
+            float *dst = stage + (size_t)row * ROWF + cg * OC;
 #pragma unroll
             for (int c = 0; c < OC; c += 16) {
                 uint32_t v[16];
@@ -422,22 +435,32 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 }
 #pragma unroll
                 for (int j = 0; j < 16; j += 4)
-                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + (uint32_t)((cg * OC + c + j) * 4)), "r"(v[j]),
-                                 "r"(v[j + 1]), "r"(v[j + 2]), "r"(v[j + 3]) : "memory");
+                    *reinterpret_cast<uint4 *>(dst + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
             if (cg == 0) {
-                st_cluster_f32(dst + D * 4, live ? sm_m : -INFINITY);
-                st_cluster_f32(dst + D * 4 + 4, live ? sm_l : 0.f);
+                stage[(size_t)row * ROWF + D] = live ? sm_m : -INFINITY;
+                stage[(size_t)row * ROWF + D + 1] = live ? sm_l : 0.f;
             }
-        }
-        if (trace && threadIdx.x == 64) trace[9] = global_ns();
-        cluster_sync_all();                               // shipped rows are visible to their owners
-        if (trace && threadIdx.x == 64) trace[10] = global_ns();
-        if (warp >= 2) {
-            const int tsm = threadIdx.x - 64;
-            const float *rows = reinterpret_cast<const float *>(smem);
+            fence_async_smem();                           // staged rows visible to the asynchronous copy engine
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (trace && threadIdx.x == 64) trace[8] = global_ns();
+            if (warp == 2 && lane < p.S) {
+                const uint32_t owner = (uint32_t)lane;
+                const int rows = max(0, min(RPC, QT - (int)owner * RPC));
+                if (rows > 0)
+                    dsmem_bulk_copy(map_to_rank(smem_u32(recv) + (uint32_t)(rank * RPC * ROWF * 4), owner),
+                                    smem_u32(stage) + (uint32_t)(owner * RPC * ROWF * 4), (uint32_t)(rows * ROWF * 4),
+                                    map_to_rank(smem_u32(&bars.merge), owner));
+            }
+            if (trace && threadIdx.x == 64) trace[9] = global_ns();
             const int row_lo = (int)rank * RPC;
-            const int my_rows = max(0, min(min(RPC, QT - row_lo), PR - qt * QT - row_lo));
+            const int own_rows = max(0, min(RPC, QT - row_lo));
+            bool got = true;
+            if (own_rows > 0) got = mbar_wait(&bars.merge, 0, abort_flag, p.status);
+            if (trace && threadIdx.x == 64) trace[10] = global_ns();
+            const int tsm = threadIdx.x - 64;
+            const float *rows = reinterpret_cast<const float *>(recv);
+            const int my_rows = got ? max(0, min(own_rows, PR - qt * QT - row_lo)) : 0;
             constexpr int SEG = D / 4;                    // 4-float segments per row
             for (int item = tsm; item < my_rows * SEG; item += NSOFT) {
                 const int lr = item / SEG, c0 = (item % SEG) * 4;
@@ -463,7 +486,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     }
     if (trace && threadIdx.x == 64) trace[11] = global_ns();
     tc_fence_before();
-    __syncthreads();
+    // no CTA leaves while its staged rows may still be read by a copy in flight, or a peer may still write to it
+    if (p.S > 1) cluster_sync_all();
+    else __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(bars.tmem_base), "r"(Smem<D>::TMEM_COLS) : "memory");
