@@ -23,102 +23,133 @@ __device__ __forceinline__ bool cand_before(const Cand &a, const Cand &b) {
     return a.key < b.key;
 }
 
+// Everything the loop touches lives in shared memory (candidate tables, node arrays, ancestor masks): an
+// iteration is a handful of shared-memory accesses and one warp reduction; the tree is written out once at the end.
 __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, const int32_t *root, const int32_t *ids,
                                                         const float *lp, glance_tree out) {
     constexpr int CAP = kMaxTreeN + 4;
     __shared__ float f_score[CAP];
     __shared__ int f_depth[CAP], f_rank[CAP], f_parent[CAP];
     __shared__ unsigned long long f_key[CAP];
+    __shared__ uint32_t f_sk[CAP];                   // order-preserving image of f_score
+    __shared__ unsigned long long f_t[CAP];          // tie word: (15 - depth) << 60 | ~key
     __shared__ float n_score[kMaxTreeN];
-    __shared__ int n_count, f_count;
-
+    __shared__ int n_token[kMaxTreeN], n_parent[kMaxTreeN], n_depth[kMaxTreeN], n_rank[kMaxTreeN];
+    __shared__ unsigned long long n_anc[kMaxTreeN * 2];
+    __shared__ float s_lp[kMaxBlock * kMaxTopk];
+    __shared__ int s_id[kMaxBlock * kMaxTopk];
     const int s = blockIdx.x, lane = threadIdx.x;
     const int W = (N + 63) >> 6;
     const int32_t *sid = ids + (size_t)s * L * k;
     const float *slp = lp + (size_t)s * L * k;
-    int32_t *token = out.token + (size_t)s * N, *parent = out.parent + (size_t)s * N;
-    int32_t *depth = out.depth + (size_t)s * N, *rank = out.rank + (size_t)s * N;
-    float *score = out.score + (size_t)s * N;
-    uint64_t *anc = out.anc + (size_t)s * N * W;
-
-    if (lane == 0) {
-        token[0] = root[s]; parent[0] = -1; depth[0] = 0; rank[0] = 0; score[0] = 0.f;
-        n_score[0] = 0.f;
-        n_count = 1;
-        f_count = 0;
-        if (L >= 1 && N > 1) {
-            f_score[0] = __fadd_rn(0.f, slp[0]);
-            f_depth[0] = 1; f_rank[0] = 0; f_parent[0] = 0; f_key[0] = 0ull;
-            f_count = 1;
-        }
+    for (int e = lane; e < L * k; e += 32) {
+        s_lp[e] = slp[e];
+        s_id[e] = sid[e];
     }
-    if (lane < W) anc[lane] = (lane == 0) ? 1ull : 0ull;
+    const int32_t root_tok = root[s];
     __syncwarp();
 
-    while (true) {
-        const int fc = f_count, nc = n_count;
-        if (fc == 0 || nc >= N) break;
-        // warp arg-best over the frontier
-        Cand best;
-        best.score = -INFINITY; best.depth = 1 << 30; best.key = ~0ull;
+    auto tie_word = [](int depth, unsigned long long key) {
+        return ((unsigned long long)(15 - depth) << 60) | (~key & 0x0fffffffffffffffull);
+    };
+    int nc = 1, fc = 0;                                  // node / frontier counts: the same in every lane
+    if (L >= 1 && N > 1) fc = 1;
+    if (lane == 0) {
+        n_token[0] = root_tok; n_parent[0] = -1; n_depth[0] = 0; n_rank[0] = 0; n_score[0] = 0.f;
+        if (fc) {
+            const float sc0 = __fadd_rn(0.f, s_lp[0]);
+            f_score[0] = sc0; f_sk[0] = float_key(sc0);
+            f_depth[0] = 1; f_rank[0] = 0; f_parent[0] = 0; f_key[0] = 0ull; f_t[0] = tie_word(1, 0ull);
+        }
+    }
+    if (lane < W) n_anc[lane] = (lane == 0) ? 1ull : 0ull;
+    __syncwarp();
+
+    // The order (score desc, depth asc, key asc) as integers: a 32-bit order-preserving image of the score and a
+    // 64-bit tie word (15 - depth in the top four bits, the complemented 60-bit path key below); larger wins.
+    while (fc > 0 && nc < N) {
+        uint32_t bsk = 0;
+        unsigned long long bt = 0ull;
         int bi = -1;
         for (int e = lane; e < fc; e += 32) {
-            Cand c; c.score = f_score[e]; c.depth = f_depth[e]; c.key = f_key[e];
-            if (bi < 0 || cand_before(c, best)) { best = c; bi = e; }
+            const uint32_t sk = f_sk[e];
+            const unsigned long long t = f_t[e];
+            if (bi < 0 || sk > bsk || (sk == bsk && t > bt)) { bsk = sk; bt = t; bi = e; }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            Cand c;
-            c.score = __shfl_xor_sync(0xffffffffu, best.score, o);
-            c.depth = __shfl_xor_sync(0xffffffffu, best.depth, o);
-            c.key = __shfl_xor_sync(0xffffffffu, best.key, o);
-            const int ci = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ci >= 0 && (bi < 0 || cand_before(c, best))) { best = c; bi = ci; }
+        // warp arg-best: hardware max over the score image, then (rarely) over the halves of the tie word
+        const uint32_t m1 = __reduce_max_sync(0xffffffffu, bi >= 0 ? bsk : 0u);
+        uint32_t live = __ballot_sync(0xffffffffu, bi >= 0 && bsk == m1);
+        if (__popc(live) > 1) {
+            const bool in = (live >> lane) & 1u;
+            const uint32_t m2 = __reduce_max_sync(0xffffffffu, in ? (uint32_t)(bt >> 32) : 0u);
+            live = __ballot_sync(0xffffffffu, in && (uint32_t)(bt >> 32) == m2);
+            if (__popc(live) > 1) {
+                const bool in2 = (live >> lane) & 1u;
+                const uint32_t m3 = __reduce_max_sync(0xffffffffu, in2 ? (uint32_t)bt : 0u);
+                live = __ballot_sync(0xffffffffu, in2 && (uint32_t)bt == m3);
+            }
         }
-        // (score, depth, key) identifies a candidate uniquely, so every lane now agrees on bi
+        // (score, depth, key) identifies a candidate uniquely: exactly one lane is left
+        bi = __shfl_sync(0xffffffffu, bi, __ffs(live) - 1);
         const int i = nc;
         const int dpt = f_depth[bi], rk = f_rank[bi], par = f_parent[bi];
         const float sc = f_score[bi];
         const unsigned long long key = f_key[bi];
-        __syncwarp();
+        // the popped entry is replaced by the last one; the child and the next sibling are appended
+        const int last = fc - 1;
+        const bool has_child = dpt < L, has_sib = rk + 1 < k;
+        float mv_score = 0.f; int mv_depth = 0, mv_rank = 0, mv_parent = 0; unsigned long long mv_key = 0ull, mv_t = 0ull;
+        uint32_t mv_sk = 0u;
+        if (lane == 3 && bi != last) {
+            mv_score = f_score[last]; mv_depth = f_depth[last]; mv_rank = f_rank[last];
+            mv_parent = f_parent[last]; mv_key = f_key[last]; mv_sk = f_sk[last]; mv_t = f_t[last];
+        }
+        unsigned long long aw = 0ull;
         if (lane < W) {
-            uint64_t w = anc[(size_t)par * W + lane];
-            if ((i >> 6) == lane) w |= 1ull << (i & 63);
-            anc[(size_t)i * W + lane] = w;
+            aw = n_anc[par * W + lane];
+            if ((i >> 6) == lane) aw |= 1ull << (i & 63);
         }
+        const float par_score = n_score[par];
+        __syncwarp();                                    // all reads of the old frontier are done
+        if (lane < W) n_anc[i * W + lane] = aw;
         if (lane == 0) {
-            token[i] = sid[(dpt - 1) * k + rk];
-            parent[i] = par; depth[i] = dpt; rank[i] = rk; score[i] = sc;
-            n_score[i] = sc;
-            n_count = nc + 1;
-            // remove the popped entry (swap with the last), then push child and sibling
-            int cnt = fc - 1;
-            if (bi != cnt) {
-                f_score[bi] = f_score[cnt]; f_depth[bi] = f_depth[cnt]; f_rank[bi] = f_rank[cnt];
-                f_parent[bi] = f_parent[cnt]; f_key[bi] = f_key[cnt];
-            }
-            if (dpt < L) {
-                f_score[cnt] = __fadd_rn(sc, slp[dpt * k + 0]);
-                f_depth[cnt] = dpt + 1; f_rank[cnt] = 0; f_parent[cnt] = i; f_key[cnt] = key;
-                ++cnt;
-            }
-            if (rk + 1 < k) {
-                f_score[cnt] = __fadd_rn(n_score[par], slp[(dpt - 1) * k + rk + 1]);
-                f_depth[cnt] = dpt; f_rank[cnt] = rk + 1; f_parent[cnt] = par;
-                f_key[cnt] = key + (1ull << (4 * (15 - dpt)));
-                ++cnt;
-            }
-            f_count = cnt;
+            n_token[i] = s_id[(dpt - 1) * k + rk];
+            n_parent[i] = par; n_depth[i] = dpt; n_rank[i] = rk; n_score[i] = sc;
+        } else if (lane == 1 && has_child) {
+            const float cs = __fadd_rn(sc, s_lp[dpt * k + 0]);
+            f_score[last] = cs; f_sk[last] = float_key(cs);
+            f_depth[last] = dpt + 1; f_rank[last] = 0; f_parent[last] = i; f_key[last] = key; f_t[last] = tie_word(dpt + 1, key);
+        } else if (lane == 2 && has_sib) {
+            const int at = last + (has_child ? 1 : 0);
+            const float ss = __fadd_rn(par_score, s_lp[(dpt - 1) * k + rk + 1]);
+            const unsigned long long sk2 = key + (1ull << (4 * (15 - dpt)));
+            f_score[at] = ss; f_sk[at] = float_key(ss);
+            f_depth[at] = dpt; f_rank[at] = rk + 1; f_parent[at] = par;
+            f_key[at] = sk2; f_t[at] = tie_word(dpt, sk2);
+        } else if (lane == 3 && bi != last) {
+            f_score[bi] = mv_score; f_depth[bi] = mv_depth; f_rank[bi] = mv_rank; f_parent[bi] = mv_parent; f_key[bi] = mv_key;
+            f_sk[bi] = mv_sk; f_t[bi] = mv_t;
         }
+        nc = nc + 1;
+        fc = last + (has_child ? 1 : 0) + (has_sib ? 1 : 0);
         __syncwarp();
     }
     __syncwarp();
-    const int nc = n_count;
     if (lane == 0) out.n_nodes[s] = nc;
-    // padding rows: never entered by the walk, visible to themselves only
-    for (int i = nc + lane; i < N; i += 32) {
-        token[i] = 0; parent[i] = -1; depth[i] = 0; rank[i] = 0; score[i] = 0.f;
-        for (int w = 0; w < W; ++w) anc[(size_t)i * W + w] = ((i >> 6) == w) ? (1ull << (i & 63)) : 0ull;
+    int32_t *token = out.token + (size_t)s * N, *parent = out.parent + (size_t)s * N;
+    int32_t *depth = out.depth + (size_t)s * N, *rank = out.rank + (size_t)s * N;
+    float *score = out.score + (size_t)s * N;
+    uint64_t *anc = out.anc + (size_t)s * N * W;
+    for (int i = lane; i < N; i += 32) {
+        // padding rows: never entered by the walk, visible to themselves only
+        const bool real = i < nc;
+        token[i] = real ? n_token[i] : 0;
+        parent[i] = real ? n_parent[i] : -1;
+        depth[i] = real ? n_depth[i] : 0;
+        rank[i] = real ? n_rank[i] : 0;
+        score[i] = real ? n_score[i] : 0.f;
+        for (int w = 0; w < W; ++w)
+            anc[(size_t)i * W + w] = real ? n_anc[i * W + w] : (((i >> 6) == w) ? (1ull << (i & 63)) : 0ull);
     }
 }
 
