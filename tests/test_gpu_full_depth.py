@@ -1,0 +1,105 @@
+"""Full-depth parity at the benchmark shape: one verify pass of the 7B configuration (28 layers, N = 64 tree
+rows against a 1536-token context) through the C ABI, compared with the fp32 CPU oracle.
+
+The committed context is synthetic: every layer's K/V cache rows are seeded random bf16 values handed to both
+sides (prefilling 1536 positions through the oracle would take minutes and test nothing new), so the comparison
+covers exactly what the timed round runs per verify pass: tree packing, 28 decoder layers with tree attention
+over the paged cache, the final norm, the LM head and its arg-max.  The oracle widens one layer's weights to
+fp32 at a time to keep the host footprint bounded.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import glance_oracle as O
+from paper_2609_00355_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+class LazyLayers:
+    """Sequence of per-layer weight dicts, converted to fp32 CPU tensors one layer at a time."""
+
+    def __init__(self, layers):
+        self.layers = layers
+
+    def __len__(self):
+        return len(self.layers)
+
+    def __iter__(self):
+        for lw in self.layers:
+            yield {k: v.detach().cpu().float() for k, v in lw.items()}
+
+    def __getitem__(self, i):
+        return {k: v.detach().cpu().float() for k, v in self.layers[i].items()}
+
+
+def test_verify_pass_7b_full_depth():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_00355_b200.binding import Engine
+    from tests import parity_harness as H
+
+    cfg = synth.CONFIGS["7b"]
+    dev = torch.device("cuda:0")
+    tw, hw = synth.make_weights(cfg, dev)
+    eng = Engine(cfg, tw, hw, batch=1)
+    P = cfg.ctx
+
+    # committed state: the same seeded random K/V bits for both sides
+    g = torch.Generator(device=dev).manual_seed(11)
+    page = cfg.page_size
+    pos = torch.arange(P, device=dev)
+    pages = eng.page_table[0].long()[pos // page]
+    Ks, Vs = [], []
+    for l in range(cfg.n_layers):
+        K = (torch.randn(P, cfg.n_kv_heads, cfg.head_dim, generator=g, device=dev) * 0.5).to(torch.bfloat16)
+        V = (torch.randn(P, cfg.n_kv_heads, cfg.head_dim, generator=g, device=dev) * 0.5).to(torch.bfloat16)
+        eng.kv_pool[l, pages, 0, :, pos % page, :] = K
+        eng.kv_pool[l, pages, 1, :, pos % page, :] = V
+        Ks.append(K.cpu())
+        Vs.append(V.cpu())
+    eng.seq_len[0] = P
+    root = 1234
+    eng.root[0] = root
+
+    rng = np.random.default_rng(5)
+    ids, lp = synth.random_topk(cfg.L, cfg.topk, cfg.vocab, rng)
+    eng.glance_build_tree(torch.from_numpy(ids[None]).to(dev), torch.from_numpy(lp[None]).to(dev))
+    vlog = torch.zeros(1, cfg.tree_N, cfg.vocab, dtype=torch.float32, device=dev)
+    eng.glance_verify_tree(logits_dbg=vlog)
+    eng.check_device_status()
+    torch.cuda.synchronize()
+
+    # oracle on the same tree and state
+    tree = O.build_tree(root, ids, lp, cfg.tree_N)
+    H.assert_tree_bits(H.tree_from_device(eng.tree, 0), tree)
+    otw = {"embed": tw["embed"].cpu().float(), "lm_head": tw["lm_head"].cpu().float(),
+           "final_norm": tw["final_norm"].cpu().float(), "layers": LazyLayers(tw["layers"])}
+    cap = P + cfg.tree_N + 8
+    st = O.SeqState(P, root, [], [], torch.zeros(1), torch.zeros(1), torch.zeros(1))
+    for l in range(cfg.n_layers):
+        Kc = torch.zeros(cap, cfg.n_kv_heads, cfg.head_dim)
+        Kc[:P] = Ks[l].float()
+        st.K.append(Kc)
+        Vc = torch.zeros(cap, cfg.n_kv_heads, cfg.head_dim)
+        Vc[:P] = Vs[l].float()
+        st.V.append(Vc)
+    ol, oh = O.verify_tree(O.Shape.of(cfg), otw, st, tree)
+
+    n = tree.n_nodes
+    assert n == cfg.tree_N
+    scale = float(ol[:n].abs().max())
+    err = float((vlog[0, :n].cpu() - ol[:n]).abs().max())
+    assert err <= H.REL_TOL * scale, f"logits: max-abs error {err:.4g} > {H.REL_TOL} x {scale:.4g}"
+    hscale = float(oh[:n].abs().max())
+    herr = float((eng.hidden[0, :n].float().cpu() - oh[:n]).abs().max())
+    assert herr <= H.REL_TOL * hscale, f"hidden: max-abs error {herr:.4g} > {H.REL_TOL} x {hscale:.4g}"
+    # the arg-max must agree wherever the oracle's decision is clear
+    oam = O.argmax_lowest(ol)
+    top2 = torch.topk(ol, 2, dim=-1).values
+    margin = (top2[:, 0] - top2[:, 1]).numpy()
+    am = eng.argmax[0].cpu().numpy()
+    for i in range(n):
+        if margin[i] > H.MARGIN:
+            assert am[i] == int(oam[i]), f"node {i}: arg-max differs at margin {margin[i]:.3g}"
