@@ -103,7 +103,9 @@ size_t glance_workspace_bytes(const glance_config *cfg);
 
 /* Creates a context on the current device.  `workspace` (device, 256-byte aligned, at least
  * glance_workspace_bytes(cfg)) and all weights stay borrowed until glance_destroy.
- * `cuda_stream` is a cudaStream_t (NULL = default stream).  Allocates only host memory. */
+ * `cuda_stream` is a cudaStream_t (NULL = default stream).  Allocates only host memory; enqueues one small
+ * host-to-device copy on that stream (the rotary frequencies theta^(-2i/d), computed in double) and the
+ * clearing of the workspace's counters. */
 int32_t glance_create(const glance_config *cfg, const glance_target_weights *target,
                       const glance_head_weights *head, void *workspace, size_t workspace_bytes,
                       void *cuda_stream, glance_ctx **out);
