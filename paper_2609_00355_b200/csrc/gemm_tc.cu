@@ -194,6 +194,42 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16);
     const uint32_t rank = CLUSTERED ? cluster_rank() : 0u;
     const int RP = CLUSTERED ? (NP + a.S - 1) / a.S : NP; // rows per owner CTA
+    // Rows this CTA finishes (all NP, or its band of the cluster's reduce-scatter) and, for the first two rows
+    // of each epilogue warp, the global operands of the row processing (residual, gain, rotary table, K/V row):
+    // they are fetched here, ahead of the merge, so that their L2 latency hides under it.
+    const int ew = warp - 2;                             // epilogue warp 0..7
+    const int row_lo = (int)rank * RP;                   // first owned row (tile-local)
+    const int my_rows = max(0, min(min(RP, NP - row_lo), a.R - r0 - row_lo));
+    const int fo = 4 * lane;                             // first of this thread's four features (tile-local)
+    float4 pre_a[2], pre_b[2], gain = make_float4(0.f, 0.f, 0.f, 0.f);
+    long long pre_kv[2] = {-1, -1};
+    pre_a[0] = pre_a[1] = pre_b[0] = pre_b[1] = gain;
+    if (warp >= 2 && f0 + fo < a.Nout) {
+        if (MODE == 3) {
+            const uint2 gg = *reinterpret_cast<const uint2 *>(a.gain + f0 + fo);
+            const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x);
+            const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
+            gain = make_float4(__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23));
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+                if (ew + u * NEPI < my_rows)
+                    pre_a[u] = __ldcg(reinterpret_cast<const float4 *>(a.x + (size_t)(r0 + row_lo + ew + u * NEPI) * a.Nout + f0 + fo));
+        } else if (MODE == 4) {
+            const int d = a.head_dim, half = d >> 1;
+            const int h = (f0 + fo) / d, i = (f0 + fo) % d;
+            const int ci = (i < half) ? i : i - half;
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+                if (ew + u * NEPI < my_rows) {
+                    const int rr = r0 + row_lo + ew + u * NEPI;
+                    if (h < a.Hq + a.Hkv) {
+                        pre_a[u] = *reinterpret_cast<const float4 *>(a.rope_cos + (size_t)rr * half + ci);
+                        pre_b[u] = *reinterpret_cast<const float4 *>(a.rope_sin + (size_t)rr * half + ci);
+                    }
+                    if (h >= a.Hq) pre_kv[u] = a.kvrow[rr];
+                }
+        }
+    }
     if (CLUSTERED) {
         cluster_sync_all();                              // every CTA's MMAs are done: all rings are idle
         if (trace && threadIdx.x == 64) trace[5] = global_ns();
@@ -239,10 +275,6 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     }
     if (warp >= 2 && ok) {
         const float *tile = reinterpret_cast<const float *>(smem);
-        const int ew = warp - 2;                         // epilogue warp 0..7
-        const int row_lo = (int)rank * RP;               // first owned row (tile-local)
-        const int my_rows = max(0, min(min(RP, NP - row_lo), a.R - r0 - row_lo));
-        const int fo = 4 * lane;                         // first of this thread's four features (tile-local)
         if (MODE == 0 || MODE == 2) {
             const bool vec = (a.ldy & 3) == 0;
             for (int r = ew; r < my_rows; r += NEPI) {
@@ -290,17 +322,13 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
         } else if (MODE == 3) {
             const int f = f0 + fo;
             const bool valid = f < a.Nout;               // Nout is a multiple of 4
-            float4 gain = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (valid) {
-                const uint2 gg = *reinterpret_cast<const uint2 *>(a.gain + f);
-                const __nv_bfloat162 g01 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.x);
-                const __nv_bfloat162 g23 = *reinterpret_cast<const __nv_bfloat162 *>(&gg.y);
-                gain = make_float4(__low2float(g01), __high2float(g01), __low2float(g23), __high2float(g23));
-            }
-            for (int lr = ew; lr < my_rows; lr += NEPI) {
+            int it = 0;
+            for (int lr = ew; lr < my_rows; lr += NEPI, ++it) {
                 const size_t o = (size_t)(r0 + row_lo + lr) * a.Nout + f;
                 float4 xv = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (valid) xv = __ldcg(reinterpret_cast<const float4 *>(a.x + o));
+                if (it == 0) xv = pre_a[0];
+                else if (it == 1) xv = pre_a[1];
+                else if (valid) xv = __ldcg(reinterpret_cast<const float4 *>(a.x + o));
                 float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
                 for (int k = 0; k < a.S; ++k) {          // split order: bit-reproducible
                     const float4 p = *reinterpret_cast<const float4 *>(tile + (size_t)(k * RP + lr) * BM + fo);
@@ -335,7 +363,8 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
             const int pfo = (i < half) ? fo + half : fo - half;
             const int ci = (i < half) ? i : i - half;
             const int kvh = is_k ? h - a.Hq : h - a.Hq - a.Hkv;
-            for (int lr = ew; lr < my_rows; lr += NEPI) {
+            int it = 0;
+            for (int lr = ew; lr < my_rows; lr += NEPI, ++it) {
                 const int rr = r0 + row_lo + lr;
                 float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
                 for (int k = 0; k < a.S; ++k) {
@@ -351,8 +380,8 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                 vb.x *= sc; vb.y *= sc; vb.z *= sc; vb.w *= sc;
                 float4 out = va;
                 if (is_q || is_k) {
-                    const float4 cs = *reinterpret_cast<const float4 *>(a.rope_cos + (size_t)rr * half + ci);
-                    const float4 sn = *reinterpret_cast<const float4 *>(a.rope_sin + (size_t)rr * half + ci);
+                    const float4 cs = it == 0 ? pre_a[0] : it == 1 ? pre_a[1] : *reinterpret_cast<const float4 *>(a.rope_cos + (size_t)rr * half + ci);
+                    const float4 sn = it == 0 ? pre_b[0] : it == 1 ? pre_b[1] : *reinterpret_cast<const float4 *>(a.rope_sin + (size_t)rr * half + ci);
                     if (i < half) {
                         out.x = va.x * cs.x - vb.x * sn.x; out.y = va.y * cs.y - vb.y * sn.y;
                         out.z = va.z * cs.z - vb.z * sn.z; out.w = va.w * cs.w - vb.w * sn.w;
@@ -368,7 +397,7 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                 if (is_q) {
                     if (rr < a.Rq) *reinterpret_cast<uint2 *>(a.q + ((size_t)rr * a.Hq + h) * d + i) = ob;
                 } else {
-                    const long long base = a.kvrow[rr];
+                    const long long base = it == 0 ? pre_kv[0] : it == 1 ? pre_kv[1] : a.kvrow[rr];
                     if (base >= 0)
                         *reinterpret_cast<uint2 *>(a.pool_layer + (size_t)base + (is_k ? 0 : a.v_off) + (size_t)kvh * a.head_stride + i) = ob;
                 }
