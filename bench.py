@@ -32,9 +32,9 @@ import torch
 from paper_2609_00355_b200 import synth
 
 # dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch, averaged over the 118 GEMM launches of a round,
-# from the ncu capture summarised in profiles/gemm_tc_and_attn_7b_2layers_ncu_full.md (2-layer case scaled to
+# from the ncu capture summarised in profiles/gemm_tc_and_attn_tc_7b_2layers_ncu_full.md (2-layer case scaled to
 # 29 layers' worth of launches + the two LM-head passes; traffic grows in proportion to the layer count)
-TRAFFIC_PER_LAUNCH = {"7b": 136.8e6}
+TRAFFIC_PER_LAUNCH = {"7b": 137.7e6}
 
 METRIC = "committed_tokens_per_s"
 UNIT = "tokens/s"

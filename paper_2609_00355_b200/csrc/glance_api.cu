@@ -196,11 +196,12 @@ void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, T
     }
     const bool prof = prof_begin(ctx);
     if (launch_gemm_tc(mode, a, *mw, *mx, ctx->stream) != cudaSuccess) ctx->map_error = true;
-    double bytes = 2.0 * a.Nout * a.K + 2.0 * a.R * a.K;
+    // weights once, activations in (both planes when two-term), results out
+    double bytes = 2.0 * a.Nout * a.K + (a.x_lo_row > 0 ? 4.0 : 2.0) * a.R * a.K;
     if (mode == 0) bytes += 4.0 * a.S * a.R * a.Nout;
-    else if (mode == 1) bytes += 2.0 * a.R * a.F;
+    else if (mode == 1) bytes += (a.act_lo ? 4.0 : 2.0) * a.R * a.F;
     else if (mode == 2) bytes += 4.0 * a.R + (a.Y ? 4.0 * a.R * a.Nout : 0.0);
-    else if (mode == 3) bytes += (4.0 + 4.0 + 2.0) * a.R * a.Nout;     // residual in/out + bf16 copy
+    else if (mode == 3) bytes += (4.0 + 4.0 + (a.xb_lo ? 4.0 : 2.0)) * a.R * a.Nout;   // residual in/out + bf16 copy
     else bytes += 2.0 * a.R * a.Nout;
     prof_end(ctx, prof, KIND_GEMM, bytes);
 }
