@@ -181,7 +181,10 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
 /* Test hook: phase timestamps of the GEMM kernel.  While a buffer (device, slots x 16 uint64) is set, the
  * n-th GEMM launch after this call makes its first CTA write nanosecond timestamps (entry, set-up done,
  * predecessor finished, first tile landed, accumulator ready, cluster barrier 1, tile shipped, cluster
- * barrier 2, epilogue done, exit) into slot n % slots.  buffer = NULL, slots = 0 switches it off. */
+ * barrier 2, epilogue done, exit) into entries 0-11 of slot n % slots (attention launches count too and record
+ * their own phases).  Entries 12-15 are merged over ALL CTAs of the launch with atomic max / min, so the caller
+ * presets them (12, 15 to 0; 13, 14 to all ones): 12 = last main loop end, 13 = first main loop end, 14 = first
+ * CTA start, 15 = last CTA end.  buffer = NULL, slots = 0 switches it off. */
 int32_t glance_debug_trace(glance_ctx *ctx, uint64_t *buffer, int32_t slots);
 
 /* Measurement aid.  While enabled, every kernel launch is bracketed by a pair of CUDA events on the context's

@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 
     unsigned long long *trace = (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? p.trace : nullptr;
     if (trace && threadIdx.x == 0) trace[0] = global_ns();
+    if (p.trace && threadIdx.x == 0) atomicMin(p.trace + 14, (unsigned long long)global_ns());   // grid span: first start
     pdl_launch_dependents();
     const int G = p.Hq / p.Hkv;
     const int PR = p.T * G;
@@ -291,7 +292,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
                 for (int j = 0; j < 16; ++j) sc[j] = __uint_as_float(v[j]);
             }
-            if (trace && threadIdx.x == 64 && i == 0) trace[12] = global_ns();
             const bool need_mask = key0 + KT > P;
             float mt = -INFINITY;
 #pragma unroll
@@ -313,7 +313,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             // row maximum of the tile across the four column groups
             red[i & 1][cg][row] = mt;
             asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");   // only the four warps of this lane quarter share rows
-            if (trace && threadIdx.x == 64 && i == 0) trace[13] = global_ns();
             if (*abort_flag) break;                       // a quarter that leaves stops arriving at p_full: every wait is bounded
             mt = fmaxf(fmaxf(red[i & 1][0][row], red[i & 1][1][row]), fmaxf(red[i & 1][2][row], red[i & 1][3][row]));
             if (i > 0) {
@@ -361,7 +360,6 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 *reinterpret_cast<uint4 *>(prow + (((cg * 2 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
             l_run += rs;
-            if (trace && threadIdx.x == 64 && i == 0) trace[14] = global_ns();
             fence_async_smem();
             tc_fence_before();
             mbar_arrive(&bars.p_full);                    // always arrive: the MMA issuer counts 512 arrivals
@@ -485,6 +483,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         }
     }
     if (trace && threadIdx.x == 64) trace[11] = global_ns();
+    if (p.trace && threadIdx.x == 64) atomicMax(p.trace + 15, (unsigned long long)global_ns());  // grid span: last end
     tc_fence_before();
     // no CTA leaves while its staged rows may still be read by a copy in flight, or a peer may still write to it
     if (p.S > 1) cluster_sync_all();

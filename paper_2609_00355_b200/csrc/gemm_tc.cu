@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     // optional phase timestamps of CTA (0,0,0) (test hook; a.trace is nullptr in normal use)
     unsigned long long *trace = (a.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? a.trace : nullptr;
     if (trace && threadIdx.x == 0) trace[0] = global_ns();
+    if (a.trace && threadIdx.x == 0) atomicMin(a.trace + 14, (unsigned long long)global_ns());   // grid span: first start
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -181,6 +182,10 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
         tc_fence_after();
         asm volatile("bar.sync 1, 256;" ::: "memory");   // inv_rms visible to all epilogue warps
         if (trace && threadIdx.x == 64) trace[4] = global_ns();
+        if (a.trace && threadIdx.x == 64 && nk > 0) {                                                 // main loop end: last / first CTA
+            atomicMax(a.trace + 12, (unsigned long long)global_ns());
+            atomicMin(a.trace + 13, (unsigned long long)global_ns());
+        }
     }
 
     // ---------------- epilogue, part 2 ----------------
@@ -235,7 +240,8 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
         if (trace && threadIdx.x == 64) trace[5] = global_ns();
     }
     if (warp >= 2) {
-        const uint32_t local = smem_u32(smem) + (uint32_t)((rank * RP) * BM * 4) + (uint32_t)(fl * 4);
+        // this CTA's plane inside an owner's ring, at the first of the lane quad's four features
+        const uint32_t quad_base = smem_u32(smem) + (uint32_t)((rank * RP) * BM * 4) + (uint32_t)((q * 32 + (lane & ~3)) * 4);
         const int chalf = (warp - 2) >> 2;               // the two warps of a lane quarter alternate 16-column chunks
         for (int c = chalf * 16; c < NP; c += 32) {
             uint32_t v[16];
@@ -254,15 +260,32 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 16; ++j) v[j] = 0u;
             }
+            if (CLUSTERED) {
+                // 4 x 4 transposes inside each lane quad: lane i of a quad ends up with rows c+4m+i (m = 0..3) of
+                // the quad's four consecutive features, so that a remote store carries 16 bytes instead of 4
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-                const int r = c + j;
-                if (CLUSTERED) {
+                for (int m = 0; m < 4; ++m) {
+                    uint32_t *e = v + 4 * m;
+#pragma unroll
+                    for (int k = 0; k < 4; k += 2) {
+                        const uint32_t x = (lane & 1) ? e[k] : e[k + 1];
+                        const uint32_t y = __shfl_xor_sync(0xffffffffu, x, 1);
+                        if (lane & 1) e[k] = y; else e[k + 1] = y;
+                    }
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const uint32_t x = (lane & 2) ? e[k] : e[k + 2];
+                        const uint32_t y = __shfl_xor_sync(0xffffffffu, x, 2);
+                        if (lane & 2) e[k] = y; else e[k + 2] = y;
+                    }
+                    const int r = c + 4 * m + (lane & 3);
                     const uint32_t owner = (uint32_t)(r / RP);
-                    st_cluster_f32(map_to_rank(local + (uint32_t)((r - owner * RP) * BM * 4), owner), __uint_as_float(v[j]));
-                } else {
-                    reinterpret_cast<float *>(smem)[r * BM + fl] = __uint_as_float(v[j]);
+                    const uint32_t dst = map_to_rank(quad_base + (uint32_t)((r - owner * RP) * BM * 4), owner);
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(e[0]), "r"(e[1]), "r"(e[2]), "r"(e[3]) : "memory");
                 }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) reinterpret_cast<float *>(smem)[(c + j) * BM + fl] = __uint_as_float(v[j]);
             }
         }
     }
@@ -406,6 +429,9 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     }
 
     if (trace && threadIdx.x == 64) trace[8] = global_ns();
+    if (a.trace && threadIdx.x == 64) {
+        atomicMax(a.trace + 15, (unsigned long long)global_ns());                                 // grid span: last end
+    }
     tc_fence_before();
     __syncthreads();
     if (trace && threadIdx.x == 0) trace[9] = global_ns();
