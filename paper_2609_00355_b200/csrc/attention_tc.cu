@@ -42,7 +42,7 @@ struct Smem {
     static constexpr int Q_BYTES = SLABS * QT * 128;     // 32 KB at d = 128
     static constexpr int KV_BYTES = SLABS * KT * 128;    // one K or V page: 16 KB at d = 128
     static constexpr int P_BYTES = QT * 128;             // 128 rows x 64 keys bf16
-    static constexpr int OPER_BYTES = Q_BYTES + 4 * KV_BYTES + P_BYTES;   // operand buffers (and merge staging)
+    static constexpr int OPER_BYTES = Q_BYTES + 4 * KV_BYTES + 2 * P_BYTES;   // P is double-buffered;   // operand buffers (and merge staging)
     static constexpr int ROWF = D + 4;                   // floats per merged row: O, m, l, padding
     // split merge: rows received from the cluster's CTAs (each owner gets <= ceil(QT/S) rows from each of S CTAs)
     static constexpr int RECV_BYTES = (QT + MAX_SPLITS) * ROWF * 4;
@@ -51,7 +51,7 @@ struct Smem {
 };
 
 struct alignas(8) AttnBars {
-    uint64_t q_ready, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full, o_done, merge;
+    uint64_t q_ready, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], merge;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -88,8 +88,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             mbar_init(&bars.v_empty[b], 1);
             mbar_init(&bars.s_full[b], 1);
         }
-        mbar_init(&bars.p_full, NSOFT);
-        mbar_init(&bars.o_done, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&bars.p_full[b], NSOFT);
+            mbar_init(&bars.o_done[b], 1);
+        }
         mbar_init(&bars.merge, 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -209,16 +211,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             for (int i = 0; i < nt && ok; ++i) {
                 const int st = i & 1;
                 if (i + 1 < nt && !issue_s(i + 1)) { ok = false; break; }
-                if (!mbar_wait(&bars.p_full, (uint32_t)i & 1u, abort_flag, p.status)) { ok = false; break; }
+                if (!mbar_wait(&bars.p_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
                 if (!mbar_wait(&bars.v_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t vbase = smem_u32(sV + st * Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < KT / 16; ++kk)
-                    umma_f16(tmem_O, umma_desc(smem_u32(sP)) + (uint64_t)(kk * 2), umma_desc_mn(vbase + kk * 16 * 128, KT * 128),
+                    umma_f16(tmem_O, umma_desc(smem_u32(sP) + st * Smem<D>::P_BYTES) + (uint64_t)(kk * 2), umma_desc_mn(vbase + kk * 16 * 128, KT * 128),
                              idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(&bars.v_empty[st]);           // V page free once these MMAs have read it
-                umma_commit(&bars.o_done);                // P free, O updated
+                umma_commit(&bars.o_done[st]);            // this P buffer free, O updated
             }
         }
     } else {
@@ -315,11 +317,10 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");   // only the four warps of this lane quarter share rows
             if (*abort_flag) break;                       // a quarter that leaves stops arriving at p_full: every wait is bounded
             mt = fmaxf(fmaxf(red[i & 1][0][row], red[i & 1][1][row]), fmaxf(red[i & 1][2][row], red[i & 1][3][row]));
-            if (i > 0) {
-                // P and O are in use by the previous tile's second MMA until o_done
-                ok = ok && mbar_wait(&bars.o_done, (uint32_t)(i - 1) & 1u, abort_flag, p.status);
+            if (i > 1) {
+                // this tile's P buffer was read by the second MMA of tile i-2
+                ok = ok && mbar_wait(&bars.o_done[st], (uint32_t)((i - 2) >> 1) & 1u, abort_flag, p.status);
                 ok = __all_sync(0xffffffffu, ok);
-                tc_fence_after();
             }
             float factor = 1.f;
             if (m_ref == -INFINITY) {
@@ -328,22 +329,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 factor = exp2f(m_ref - mt);
                 m_ref = mt;
             }
-            if (__any_sync(0xffffffffu, factor != 1.f) && ok) {
-                l_run *= factor;
-#pragma unroll
-                for (int c = 0; c < OC; c += 16) {
-                    uint32_t v[16];
-                    tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * factor);
-                    tmem_st16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+            if (__any_sync(0xffffffffu, factor != 1.f)) {
+                // O may only be touched once the previous tile's second MMA has landed
+                if (i > 0) {
+                    ok = ok && mbar_wait(&bars.o_done[st ^ 1], (uint32_t)((i - 1) >> 1) & 1u, abort_flag, p.status);
+                    ok = __all_sync(0xffffffffu, ok);
                 }
-                tmem_st_wait();
+                tc_fence_after();
+                if (ok) {
+                    l_run *= factor;
+#pragma unroll
+                    for (int c = 0; c < OC; c += 16) {
+                        uint32_t v[16];
+                        tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * factor);
+                        tmem_st16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                    }
+                    tmem_st_wait();
+                }
             }
             // P = 2^(S' - m_ref), bf16: this thread's 16 keys = two 16-byte chunks of its row of the A operand
             float rs = 0.f;
-            unsigned char *prow = sP + row * 128;
+            unsigned char *prow = sP + st * Smem<D>::P_BYTES + row * 128;
             const float m_sub = (m_ref == -INFINITY) ? 0.f : m_ref;   // a fully masked row keeps -inf - 0 = -inf -> 2^-inf = 0
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
@@ -362,12 +371,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             l_run += rs;
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(&bars.p_full);                    // always arrive: the MMA issuer counts 512 arrivals
+            mbar_arrive(&bars.p_full[st]);                // always arrive: the MMA issuer counts 512 arrivals
             if (trace && threadIdx.x == 64 && i == 0) trace[5] = global_ns();
         }
         if (trace && threadIdx.x == 64) trace[6] = global_ns();
         if (ok && nt > 0) {
-            ok = mbar_wait(&bars.o_done, (uint32_t)(nt - 1) & 1u, abort_flag, p.status);
+            ok = mbar_wait(&bars.o_done[(nt - 1) & 1], (uint32_t)((nt - 1) >> 1) & 1u, abort_flag, p.status);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
         }
