@@ -350,3 +350,27 @@ def test_round_7b_shape_one_layer_slice(harness):
     for r in range(3):
         run.round(p_m=0.8, check_draft=(r == 0))
     print("7b-slice parity stats:", run.stats)
+
+
+def test_round_long_shape_slice_128_rows(harness):
+    """N = 128 tree rows at the full 7B widths (2 layers, reduced vocabulary): the 128-row GEMM tiles with
+    two-term activations (UMMA N = 256) and the two-word ancestor masks of the long-context configuration."""
+    cfg = synth.CONFIGS["long"].replace(n_layers=2, vocab=4096, n_img=300, n_txt=85, rounds=3)
+    run = harness.ParityRun(cfg)
+    run.check_state()
+    for r in range(2):
+        run.round(p_m=0.5, check_draft=(r == 0))
+    print("long-slice parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_batch3_two_row_blocks(harness):
+    """Three sequences of 64 tree rows each: 192 verify rows span two 128-row blocks of every GEMM."""
+    cfg = synth.CONFIGS["tiny"].replace(tree_N=64, block_B=8, topk=4)
+    run = harness.ParityRun(cfg, batch=3, ctx_lens=[(90, 20), (33, 9), (150, 41)])
+    run.check_state()
+    for _ in range(3):
+        run.round(p_m=0.7)
+    run.check_head_state()
+    print("batch3 x 64 rows parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
