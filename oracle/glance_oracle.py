@@ -35,9 +35,10 @@ random, chain and single-node trees; accepted length against brute-force members
 verify rows against chain_row; chain mask = causal; best-first = brute-force sort;
 attention against torch SDPA; top-k / lse against torch.topk / logsumexp; rotary
 relative-position identity; KV state after rounds = fresh prefill.
-The draft head's definition (one layer over final hidden states) has no worked example
-in the paper: **parity unpinned** for draft_block beyond internal consistency and
-library cross-checks of its attention and top-k.
+draft_block (the reading of Section 3.2 stated above; the paper prints no worked example of the head):
+equality with decoder_layer under an all-ones mask, the identity-layer closed form (W_o = W_down = 0), the
+single-key closed form (B = 1, no context) written out in float64, invariance under a permutation of the
+context rows.
 """
 from __future__ import annotations
 

@@ -403,7 +403,7 @@ def test_commit_moves_rows_in_ascending_order_hazard_case(tiny):
 
 
 def test_draft_block_internal_consistency(tiny):
-    """The head definition is unpinned by the paper; these are consistency checks only."""
+    """Consistency checks of the block head beside the pins below."""
     st = _fresh(tiny)
     dl = O.draft_block(tiny.sh, tiny.tw, tiny.hw, st, tiny.cfg.block_B)
     assert dl.shape == (tiny.cfg.block_B, tiny.cfg.vocab)
@@ -414,6 +414,94 @@ def test_draft_block_internal_consistency(tiny):
     assert all(float((dl[j] - dl2[j]).abs().max()) > 0 for j in range(tiny.cfg.block_B))
     # masked slots differ only through their rotary positions
     assert float((dl[1] - dl[2]).abs().max()) > 0
+
+
+def _head_as_layer(hw):
+    return {k: hw[k] for k in ("ln1", "wqkv", "wo", "ln2", "wgu", "wd")}
+
+
+def test_draft_block_is_one_unmasked_decoder_layer(tiny):
+    """Section 3.2 reading: the head is ONE decoder layer whose B rows see all P context keys and all B block
+    keys.  The same rows pushed through decoder_layer (pinned elsewhere against library attention and cache-free
+    chains) with the head's weights and an all-ones mask must give the same logits."""
+    st = _fresh(tiny)
+    sh, B, P = tiny.sh, tiny.cfg.block_B, st.P
+    dl = O.draft_block(sh, tiny.tw, tiny.hw, st, B)
+    X = tiny.hw["mask_embed"][None, :].repeat(B, 1)
+    X[0] = tiny.tw["embed"][st.root]
+    Kc, Vc = st.hK.clone(), st.hV.clone()
+    pos = torch.arange(P, P + B)
+    y = O.decoder_layer(sh, _head_as_layer(tiny.hw), X, pos, Kc, Vc, pos, torch.ones(B, P + B, dtype=torch.bool))
+    ref = O.rmsnorm(y, tiny.hw["final_norm"], sh.rms_eps) @ tiny.tw["lm_head"].T
+    assert float((dl - ref).abs().max()) <= 1e-5 * float(ref.abs().max())
+    # and the pass must not have touched the committed head context
+    assert torch.equal(st.hK[:P], Kc[:P]) and torch.equal(st.hV[:P], Vc[:P])
+
+
+def test_draft_block_identity_layer_closed_form(tiny):
+    """With W_o = 0 and W_down = 0 the layer is the identity: logits = lm_head . rmsnorm(input), written out in
+    float64.  Slot 0 comes from E[root], every other slot from the mask embedding (so they are all equal)."""
+    st = _fresh(tiny)
+    sh, B = tiny.sh, tiny.cfg.block_B
+    hw = dict(tiny.hw)
+    hw["wo"] = torch.zeros_like(hw["wo"])
+    hw["wd"] = torch.zeros_like(hw["wd"])
+    dl = O.draft_block(sh, tiny.tw, hw, st, B).double().numpy()
+    g = hw["final_norm"].double().numpy()
+    W = tiny.tw["lm_head"].double().numpy()
+
+    def closed(x):
+        x = x.double().numpy()
+        return W @ (x / np.sqrt(np.mean(x * x) + sh.rms_eps) * g)
+
+    ref0, ref1 = closed(tiny.tw["embed"][st.root]), closed(hw["mask_embed"])
+    scale = max(np.abs(ref0).max(), np.abs(ref1).max())
+    assert np.abs(dl[0] - ref0).max() <= 1e-5 * scale
+    for j in range(1, B):
+        assert np.abs(dl[j] - ref1).max() <= 1e-5 * scale
+
+
+def test_draft_block_single_key_closed_form(tiny):
+    """B = 1 with no context: the softmax runs over one key, so the attention output is that row's own value
+    vector (kv head h // G for q head h) and the whole pass has a closed form, written out in float64 numpy."""
+    sh = tiny.sh
+    hw, tw = tiny.hw, tiny.tw
+    root = 7
+    Hq, Hkv, d, F = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.ffn
+    st = O.SeqState(0, root, [], [], torch.zeros(4, Hkv, d), torch.zeros(4, Hkv, d), torch.zeros(4, sh.hidden))
+    dl = O.draft_block(sh, tw, hw, st, 1).double().numpy()[0]
+
+    def norm(x, g):
+        return x / np.sqrt(np.mean(x * x) + sh.rms_eps) * g.double().numpy()
+
+    x = tw["embed"][root].double().numpy()
+    Wqkv = hw["wqkv"].double().numpy()
+    v = (Wqkv[(Hq + Hkv) * d:] @ norm(x, hw["ln1"])).reshape(Hkv, d)          # value rows follow the q and k rows
+    o = np.concatenate([v[h // (Hq // Hkv)] for h in range(Hq)])                # one key: softmax weight 1
+    x = x + hw["wo"].double().numpy() @ o
+    gu = hw["wgu"].double().numpy() @ norm(x, hw["ln2"])
+    gate, up = gu[:F], gu[F:]
+    x = x + hw["wd"].double().numpy() @ (gate / (1.0 + np.exp(-gate)) * up)
+    ref = tw["lm_head"].double().numpy() @ norm(x, hw["final_norm"])
+    assert np.abs(dl - ref).max() <= 1e-4 * np.abs(ref).max()
+
+
+def test_draft_block_context_order_invariance(tiny):
+    """No mask inside [context ; block]: permuting the context rows (keys and values together) changes nothing,
+    while breaking the pairing of keys and values does."""
+    st = _fresh(tiny)
+    sh, B, P = tiny.sh, tiny.cfg.block_B, st.P
+    dl = O.draft_block(sh, tiny.tw, tiny.hw, st, B)
+    perm = torch.randperm(P, generator=torch.Generator().manual_seed(3))
+    st2 = _fresh(tiny)
+    st2.hK[:P] = st.hK[:P][perm]
+    st2.hV[:P] = st.hV[:P][perm]
+    dl2 = O.draft_block(sh, tiny.tw, tiny.hw, st2, B)
+    assert float((dl - dl2).abs().max()) <= 2e-5 * float(dl.abs().max())
+    st3 = _fresh(tiny)
+    st3.hK[:P] = torch.roll(st.hK[:P], 1, 0)        # keys and values no longer paired
+    dl3 = O.draft_block(sh, tiny.tw, tiny.hw, st3, B)
+    assert float((dl - dl3).abs().max()) > 1e-4 * float(dl.abs().max())
 
 
 def test_controlled_match_acceptance_statistics(tiny):
