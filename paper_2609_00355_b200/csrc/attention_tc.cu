@@ -11,9 +11,11 @@
 // The running reference maximum m of a row is only raised when a tile exceeds it by more than 2^8 (the
 // accumulator is then rescaled in TMEM), so exponentials stay far inside fp32/bf16 range and O is almost
 // never touched between tiles.  Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
-// warps 2..17 = softmax / epilogue (a row's scores and outputs are split over four threads).  The key splits of a tile form a thread-block cluster and are merged
-// through distributed shared memory.  Every mbarrier wait is bounded; a wait that gives up records
-// GLANCE_E_TIMEOUT.
+// warps 2..17 = softmax / epilogue (a row's scores and outputs are split over four threads).  S and P are
+// double-buffered, so the next tile's scores and probabilities are produced while the previous P V runs.
+// The key splits of a tile form a thread-block cluster and are merged through distributed shared memory
+// (one asynchronous bulk copy per owner CTA, byte-counted on the owner's mbarrier).  Every mbarrier wait is
+// bounded; a wait that gives up records GLANCE_E_TIMEOUT.
 #include "kernels.cuh"
 #include "tc_ptx.cuh"
 

@@ -5,8 +5,10 @@
 // One CTA owns a 128-row weight tile (UMMA M = 128) and up to 128 activation rows (UMMA N = NP, a
 // multiple of 16) over one K range.  Weights are read from HBM exactly once; a ring of STAGES shared
 // memory slots is filled by TMA (128-byte swizzle, one 64-wide k-slab per slot) and drained by
-// tcgen05.mma issued from a single thread; the fp32 accumulator lives in TMEM and is read back by four
-// epilogue warps (one TMEM lane = one output feature).
+// tcgen05.mma issued from a single thread; the fp32 accumulator lives in TMEM and is read back by eight
+// epilogue warps (one TMEM lane = one output feature, two warps per lane quarter).  Activations may be two-term
+// (x = hi + lo, both bf16): the lo rows are NP more rows of the same B tile, and the epilogue adds the two
+// accumulator halves.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer, warps 2..9 = epilogue.
 // Epilogues: (0) fp32 split-K plane, (1) SwiGLU over 64 gate rows and their 64 up rows stacked into one tile,
