@@ -62,9 +62,13 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
     const int stage_bytes = BM * 128 + NB * 128;
     const int stages = a.stages;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int f0 = blockIdx.x * FT;
+    // grid = (weight tiles, K splits, 128-row blocks) -- or, with more than one row block, (row blocks, K splits,
+    // weight tiles): CTAs are dispatched x-fastest, so the CTAs that stream the same weight tile for different row
+    // blocks then start together and all but the first find the tile in L2 instead of reading HBM again
+    const int tile_idx = a.rows_fastest ? blockIdx.z : blockIdx.x;
+    const int f0 = tile_idx * FT;
     const int split = blockIdx.y;
-    const int r0 = blockIdx.z * 128;
+    const int r0 = (a.rows_fastest ? blockIdx.x : blockIdx.z) * 128;
     const int ktiles = a.K / BK;
     const int kt0 = (int)((long long)split * ktiles / a.S), kt1 = (int)((long long)(split + 1) * ktiles / a.S);
     const int nk = kt1 - kt0;
@@ -376,7 +380,7 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                     sq = ((xv.x * xv.x + xv.y * xv.y) + xv.z * xv.z) + xv.w * xv.w;
                 }
                 sq = warp_sum(sq);                       // one warp spans the tile's 128 features
-                if (lane == 0) a.ssq_out[(size_t)blockIdx.x * a.ssq_stride + r0 + row_lo + lr] = sq;
+                if (lane == 0) a.ssq_out[(size_t)tile_idx * a.ssq_stride + r0 + row_lo + lr] = sq;
             }
         } else {
             // MODE 4: q heads, then k heads, then v heads; rotary pairs (i, i + d/2) lie in the same tile
@@ -539,7 +543,9 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     a.tmem_cols = cols;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     const int tiles = mode == 1 ? (a.F + 63) / 64 : (a.Nout + BM - 1) / BM;
-    dim3 grid(tiles, a.S, (a.R + 127) / 128);
+    const int row_blocks = (a.R + 127) / 128;
+    a.rows_fastest = row_blocks > 1 ? 1 : 0;
+    dim3 grid(a.rows_fastest ? row_blocks : tiles, a.S, a.rows_fastest ? tiles : row_blocks);
     if (mode >= 3) {
         // every CTA's ring must hold S planes of ceil(np/S) rows, and a cluster has at most 8 CTAs
         const size_t rp = (a.np + a.S - 1) / a.S;

@@ -39,7 +39,7 @@ struct TcGemmArgs {
     int Hq, Hkv, head_dim, Rq;
     unsigned long long *trace;   // test hook: 16 phase timestamps (ns) of CTA (0,0,0), or nullptr
     // filled by launch_gemm_tc
-    int np, stages;
+    int np, stages, rows_fastest;
     uint32_t tmem_cols;
 };
 
