@@ -217,6 +217,37 @@ class RoundBench:
         return self.res_host[:, 0].clone()
 
 
+def plain_ar_ms_per_token(cfg, weights, dev, rank, steps):
+    """Plain greedy decoding through the same library: one verify pass of a single-node tree + commit per token.
+
+    A second engine with a 16-row pass (the smallest GEMM row tile) on the same weights and a context of the same
+    length; every step commits exactly one token, so ms per step = ms per token.  Replayed from a CUDA graph.
+    """
+    ar_cfg = cfg.replace(tree_N=16, name=cfg.name + "-ar")
+    b = RoundBench(ar_cfg, dev, rank, weights=weights)
+    eng = b.eng
+
+    def step():
+        b.ar_tree.token[:, 0].copy_(eng.root)
+        eng.glance_verify_tree(tree=b.ar_tree)
+        eng.glance_accept_commit(tree=b.ar_tree)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    graph = eng.capture(step)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    graph.replay()
+    torch.cuda.synchronize()
+    start.record()
+    for _ in range(steps):
+        graph.replay()
+    stop.record()
+    torch.cuda.synchronize()
+    eng.check_device_status()
+    return start.elapsed_time(stop) / steps
+
+
 class OracleSample:
     """Times the CPU oracle (as it stands) on a bounded sample of one round and scales to the full depth.
 
@@ -295,6 +326,7 @@ def main():
     ap.add_argument("--no-lookahead", action="store_true",
                     help="random candidates instead of the look-ahead (profiling captures: fewer launches)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end arm (profiling captures)")
+    ap.add_argument("--no-ar", action="store_true", help="skip the plain greedy-decoding comparison arm")
     ap.add_argument("--no-graph", action="store_true", help="launch the round's kernels one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
     cfg = synth.CONFIGS[args.config]
@@ -463,6 +495,12 @@ def main():
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
     }
+    if not args.no_ar and world == 1 and cfg.batch == 1:
+        ar_ms = plain_ar_ms_per_token(cfg, (bench.tw, bench.hw), dev, rank, min(args.steps, 32))
+        line["plain_ar"] = {"value": 1e3 / ar_ms, "unit": UNIT, "ms_per_token": ar_ms,
+                            "speedup_of_speculative_rounds": value / (1e3 / ar_ms),
+                            "what": "greedy decoding through the same library: single-node 16-row verify pass + commit "
+                                    "per token, CUDA-graph replay, same weights and context length"}
     if not args.no_cpu_baseline and world == 1:
         sample = OracleSample(cfg, bench.tw, bench.hw)
         sample.round_seconds()                                   # first call pages the fp32 copies in
