@@ -129,6 +129,7 @@ class RoundBench:
         from paper_2609_00355_b200.binding import Engine, TreeBuffers
         self.cfg, self.dev = cfg, device
         self.no_lookahead = False
+        self.calibrated = False      # true token at rank r with the marginal's probability (budget sweeps)
         self.tw, self.hw = weights if weights is not None else synth.make_weights(cfg, device)
         self.stream = torch.cuda.Stream(device)      # the library's stream; also made torch's current stream
         torch.cuda.set_stream(self.stream)
@@ -181,8 +182,8 @@ class RoundBench:
     def make_candidates(self, Y):
         cfg = self.cfg
         for s in range(cfg.batch):
-            self.ids_host[s] = torch.from_numpy(
-                synth.controlled_candidates(list(Y[s]), self.p_ms[s], cfg.topk, cfg.L, cfg.vocab, self.rng))
+            gen = synth.calibrated_candidates if self.calibrated else synth.controlled_candidates
+            self.ids_host[s] = torch.from_numpy(gen(list(Y[s]), self.p_ms[s], cfg.topk, cfg.L, cfg.vocab, self.rng))
 
     def capture_round(self):
         """One CUDA graph for the four calls of a round (ragged lengths live in device memory)."""

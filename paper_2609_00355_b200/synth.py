@@ -175,6 +175,32 @@ def controlled_candidates(Y: List[int], p_m: float, k: int, L: int, vocab: int,
     return ids
 
 
+def calibrated_candidates(Y: List[int], p_m: float, k: int, L: int, vocab: int,
+                          rng: np.random.Generator) -> np.ndarray:
+    """Candidate ids[L][k] whose ranks are calibrated to the controlled marginals: the true token Y[j] sits at rank
+    r with probability q[r] (q[0] = p_m, q[r] = (1 - p_m) 2^-r) and is absent with the remaining mass, so that
+    sibling branches of a tree can be hit (budget sweeps); other candidates are distinct random ids != Y[j]."""
+    q = [p_m] + [(1.0 - p_m) * 2.0 ** (-r) for r in range(1, k)]
+    ids = np.zeros((L, k), dtype=np.int32)
+    for j in range(L):
+        y = int(Y[j])
+        u, r_hit, acc = rng.random(), -1, 0.0
+        for r in range(k):
+            acc += q[r]
+            if u < acc:
+                r_hit = r
+                break
+        others: List[int] = []
+        while len(others) < k:
+            c = int(rng.integers(0, vocab))
+            if c != y and c not in others:
+                others.append(c)
+        if r_hit >= 0:
+            others[r_hit] = y
+        ids[j] = np.array(others, dtype=np.int32)
+    return ids
+
+
 def random_topk(L: int, k: int, vocab: int, rng: np.random.Generator, ties: bool = False):
     """Random per-depth candidates: distinct ids and non-increasing fp32 log-probs (for tree-builder tests)."""
     ids = np.zeros((L, k), dtype=np.int32)

@@ -374,3 +374,14 @@ def test_rounds_batch3_two_row_blocks(harness):
     run.check_head_state()
     print("batch3 x 64 rows parity stats:", run.stats)
     assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_tiny_chain_k1(harness):
+    """k = 1: the candidate tree degenerates to the rank-0 chain (classic chain drafting through the same path)."""
+    cfg = synth.CONFIGS["tiny"].replace(topk=1, tree_N=4)
+    run = harness.ParityRun(cfg)
+    run.check_state()
+    for r in range(6):
+        run.round(p_m=0.8, check_draft=(r == 0))
+    print("chain parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
