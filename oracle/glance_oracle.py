@@ -35,6 +35,8 @@ random, chain and single-node trees; accepted length against brute-force members
 verify rows against chain_row; chain mask = causal; best-first = brute-force sort;
 attention against torch SDPA; top-k / lse against torch.topk / logsumexp; rotary
 relative-position identity; KV state after rounds = fresh prefill.
+sampling mode (Limitations section): Philox known-answer vectors, uniforms strictly inside (0,1), draw frequencies
+against the softmax, and tree rounds against plain ancestral sampling with the same noise field.
 draft_block (the reading of Section 3.2 stated above; the paper prints no worked example of the head):
 equality with decoder_layer under an all-ones mask, the identity-layer closed form (W_o = W_down = 0), the
 single-key closed form (B = 1, no context) written out in float64, invariance under a permutation of the
@@ -541,6 +543,105 @@ def spec_round(sh: Shape, tw: dict, hw: dict, st: SeqState, B: int, k: int, N: i
     top2 = torch.topk(logits, 2, dim=-1).values
     info.update(tree=tree, logits=logits, hidden=hidden, argmax=am, a=a, path=path, out=out, new_root=new_root,
                 margins=(top2[:, 0] - top2[:, 1]).numpy())
+    commit(sh, hw, st, path, hidden, out, new_root)
+    return info
+
+
+# ----------------------------------------------------------------------------------------------
+# sampling mode (Limitations: under sampling the walk draws each token from the verified row of its
+# node and descends while the draw is a child; every committed token is a draw from the target)
+# ----------------------------------------------------------------------------------------------
+# A draw from softmax(logits / T) is taken as argmax_v (logits[v] / T + g[v]) with g[v] i.i.d. standard Gumbel
+# (the Gumbel-max identity).  The noise is a fixed field g(seed, position of the token being drawn, v) from a
+# counter-based generator (Philox4x32-10), so that the token drawn at a position does not depend on which tree
+# row, round or decoding scheme asks for it: tree rounds then commit exactly the tokens that plain ancestral
+# sampling with the same field emits (sampled_ar_cachefree), which is what the sampling walk promises.
+
+_PHILOX_M0, _PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+_PHILOX_W0, _PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32(counter, key, rounds: int = 10) -> np.ndarray:
+    """Philox4x32 (Salmon et al., SC 2011).  counter: 4 arrays of uint32 (broadcastable), key: 2 uint32.
+    Returns uint32 [4, ...]."""
+    mask = np.uint64(0xFFFFFFFF)
+    c = [np.asarray(x, dtype=np.uint64) & mask for x in counter]
+    c = list(np.broadcast_arrays(*c))
+    k0, k1 = np.uint64(int(key[0]) & 0xFFFFFFFF), np.uint64(int(key[1]) & 0xFFFFFFFF)
+    for _ in range(rounds):
+        p0 = np.uint64(_PHILOX_M0) * c[0]
+        p1 = np.uint64(_PHILOX_M1) * c[2]
+        hi0, lo0 = p0 >> np.uint64(32), p0 & mask
+        hi1, lo1 = p1 >> np.uint64(32), p1 & mask
+        c = [(hi1 ^ c[1] ^ k0) & mask, lo1, (hi0 ^ c[3] ^ k1) & mask, lo0]
+        k0 = (k0 + np.uint64(_PHILOX_W0)) & mask
+        k1 = (k1 + np.uint64(_PHILOX_W1)) & mask
+    return np.stack(c).astype(np.uint32)
+
+
+def uniform_field(seed: int, position: int, V: int) -> np.ndarray:
+    """u[v] in (0,1), fp32 exact: vocabulary ids 4b..4b+3 take the four words of Philox(counter = (b, position, 0, 0),
+    key = (seed low, seed high)); u = ((word >> 9) + 0.5) * 2^-23."""
+    nb = (V + 3) // 4
+    words = philox4x32((np.arange(nb, dtype=np.uint64), np.uint64(position & 0xFFFFFFFF), np.uint64(0), np.uint64(0)),
+                       (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF))
+    flat = words.T.reshape(-1)[:V]                                   # id 4b+j <- word j of block b
+    return ((flat >> np.uint32(9)).astype(np.float32) + np.float32(0.5)) * np.float32(2.0 ** -23)
+
+
+def gumbel_field(seed: int, position: int, V: int) -> np.ndarray:
+    """Standard Gumbel noise g = -log(-log u) in fp32."""
+    u = uniform_field(seed, position, V)
+    return (-np.log(-np.log(u))).astype(np.float32)
+
+
+def perturbed_rows(logits: torch.Tensor, positions: Sequence[int], seed: int, inv_temperature: float = 1.0) -> np.ndarray:
+    """y[i][v] = logits[i][v] * inv_temperature + g(seed, positions[i], v), fp32.  positions[i] is the position of
+    the token that row i predicts (its own position + 1)."""
+    L = logits.numpy().astype(np.float32)
+    out = np.empty_like(L)
+    for i, pos in enumerate(positions):
+        out[i] = L[i] * np.float32(inv_temperature) + gumbel_field(seed, int(pos), L.shape[1])
+    return out
+
+
+def sample_rows(logits: torch.Tensor, positions: Sequence[int], seed: int, inv_temperature: float = 1.0):
+    """One draw per row from softmax(logits * inv_temperature): arg-max of the perturbed row, ties to the lowest id.
+    Returns (ids int32 [n], margins [n] = gap between the two largest perturbed values)."""
+    y = torch.from_numpy(perturbed_rows(logits, positions, seed, inv_temperature))
+    top2 = torch.topk(y, 2, dim=-1).values
+    return argmax_lowest(y), (top2[:, 0] - top2[:, 1]).numpy()
+
+
+def sampled_ar_cachefree(sh: Shape, tw: dict, ctx_embeds: torch.Tensor, first: int, n_new: int, seed: int):
+    """Plain ancestral sampling at temperature 1, one full causal forward per token, no cache: after the context and
+    the given first token (the pending root), token number k is drawn from the target's row with the noise field of
+    its own position.  Returns the n_new tokens after `first`."""
+    x = torch.cat([ctx_embeds, tw["embed"][first][None, :]], dim=0)
+    toks = []
+    for _ in range(n_new):
+        logits, _ = full_causal_forward(sh, tw, x)
+        t = int(sample_rows(logits[-1:], [x.shape[0]], seed)[0][0])
+        toks.append(t)
+        x = torch.cat([x, tw["embed"][t][None, :]], dim=0)
+    return toks
+
+
+def spec_round_sampled(sh: Shape, tw: dict, hw: dict, st: SeqState, B: int, k: int, N: int, seed: int,
+                       tree: Optional[Tree] = None):
+    """One round in sampling mode: as spec_round, but every row's decision is a draw from its verified row."""
+    info = {}
+    if tree is None:
+        dl = draft_block(sh, tw, hw, st, B)
+        ids, lp = topk_logprobs(dl, k)
+        tree = build_tree(st.root, ids, lp, N)
+        info.update(draft_logits=dl, ids=ids, lp=lp)
+    logits, hidden = verify_tree(sh, tw, st, tree)
+    positions = [st.P + int(d) + 1 for d in tree.depth]
+    draws, margins = sample_rows(logits, positions, seed)
+    a, path, out, new_root = walk(tree, draws)
+    info.update(tree=tree, logits=logits, hidden=hidden, argmax=draws, a=a, path=path, out=out, new_root=new_root,
+                margins=margins)
     commit(sh, hw, st, path, hidden, out, new_root)
     return info
 

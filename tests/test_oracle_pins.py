@@ -504,6 +504,78 @@ def test_draft_block_context_order_invariance(tiny):
     assert float((dl - dl3).abs().max()) > 1e-4 * float(dl.abs().max())
 
 
+# ------------------------------------------------------------------ sampling mode
+
+def test_philox_known_answers():
+    path = os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_known_answers.txt")
+    n = 0
+    for line in open(path):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        got = O.philox4x32(([w[0]], [w[1]], [w[2]], [w[3]]), (w[4], w[5]))[:, 0]
+        assert [int(x) for x in got] == w[6:10]
+        n += 1
+    assert n == 3
+
+
+def test_uniform_field_layout_and_range():
+    seed, pos, V = 0x1234567890ABCDEF, 777, 1003
+    u = O.uniform_field(seed, pos, V)
+    assert u.dtype == np.float32 and u.shape == (V,)
+    assert float(u.min()) > 0.0 and float(u.max()) < 1.0
+    # id 4b + j reads word j of the block whose counter is (b, position, 0, 0)
+    for v in (0, 1, 6, 1002):
+        w = O.philox4x32(([v // 4], [pos], [0], [0]), (seed & 0xFFFFFFFF, seed >> 32))[v % 4, 0]
+        assert u[v] == np.float32(((int(w) >> 9) + 0.5) * 2.0 ** -23)
+    # another position or seed gives another field
+    assert not np.array_equal(u, O.uniform_field(seed, pos + 1, V))
+    assert not np.array_equal(u, O.uniform_field(seed + 1, pos, V))
+
+
+def test_gumbel_max_draws_follow_the_softmax():
+    """Frequencies of arg-max(logits + g) over many positions against softmax(logits): chi-square, 7 degrees of
+    freedom, and the same at temperature 2 (inv_temperature 0.5)."""
+    logits = torch.tensor([[2.0, 1.0, 0.5, 0.0, -0.5, -1.0, 1.5, -3.0]])
+    n = 20000
+    for inv_t in (1.0, 0.5):
+        p = torch.softmax(logits[0] * inv_t, dim=0).numpy()
+        ids, _ = O.sample_rows(logits.repeat(n, 1), list(range(n)), seed=99, inv_temperature=inv_t)
+        cnt = np.bincount(ids, minlength=8)
+        chi2 = float(((cnt - n * p) ** 2 / (n * p)).sum())
+        assert chi2 < 24.3, (inv_t, chi2, cnt)          # P(chi2_7 > 24.3) = 0.001
+
+
+def test_sampled_rounds_equal_plain_ancestral_sampling(tiny):
+    """Sampling walk: tree rounds commit exactly the tokens that plain ancestral sampling (one cache-free forward
+    per token) draws with the same noise field, whatever the trees are."""
+    seed = 0xC0FFEE
+    st = _fresh(tiny)
+    first, P0 = st.root, st.P
+    rng = np.random.default_rng(17)
+    n_rounds = 6
+    ref = O.sampled_ar_cachefree(tiny.sh, tiny.tw, tiny.ctx, first, n_rounds * tiny.cfg.block_B, seed)
+    accepted = []
+    for r in range(n_rounds):
+        done = st.P - P0                      # tokens committed after the first root so far
+        Y = ref[done:done + tiny.cfg.L]
+        tree = None
+        if r % 2 == 1:                        # every other round: a random tree with the true draws planted
+            def pref(parent, depth):
+                return int(Y[depth - 1]) if rng.random() < 0.8 else None
+            tok, par, dep = synth.random_tree(8, tiny.cfg.L, tiny.cfg.vocab, rng, tokens_for=pref)
+            tok[0] = st.root
+            tree = O.tree_from_arrays(tok, par, dep, N=8)
+        info = O.spec_round_sampled(tiny.sh, tiny.tw, tiny.hw, st, tiny.cfg.block_B, tiny.cfg.topk, tiny.cfg.tree_N,
+                                    seed, tree=tree)
+        accepted.append(info["a"])
+        assert float(np.min(info["margins"][:info["tree"].n_nodes])) > 1e-4, "near-tie in a perturbed row: pick another seed"
+    committed = st.tokens + [st.root]
+    assert committed[0] == first
+    assert committed[1:] == ref[:len(committed) - 1]
+    assert sum(accepted) > 0
+
+
 def test_controlled_match_acceptance_statistics(tiny):
     """Measured mean accepted length under controlled per-depth match probability sits on Eq. 2."""
     rng = np.random.default_rng(21)
