@@ -130,6 +130,7 @@ class RoundBench:
         self.cfg, self.dev = cfg, device
         self.no_lookahead = False
         self.calibrated = False      # true token at rank r with the marginal's probability (budget sweeps)
+        self.sample_seed = None      # set: sampling mode at temperature 1 (draws instead of arg-max decisions)
         self.tw, self.hw = weights if weights is not None else synth.make_weights(cfg, device)
         self.stream = torch.cuda.Stream(device)      # the library's stream; also made torch's current stream
         torch.cuda.set_stream(self.stream)
@@ -173,7 +174,7 @@ class RoundBench:
         ys = []
         for _ in range(cfg.L):
             self.ar_tree.token[:, 0].copy_(eng.root)
-            eng.glance_verify_tree(tree=self.ar_tree)
+            self.verify(self.ar_tree)
             eng.glance_accept_commit(tree=self.ar_tree)
             ys.append(eng.root.clone())
         eng.restore_state(snap)
@@ -198,11 +199,17 @@ class RoundBench:
         else:
             self.round_calls()
 
+    def verify(self, tree=None):
+        if self.sample_seed is None:
+            self.eng.glance_verify_tree(tree=tree)
+        else:
+            self.eng.glance_verify_tree_sample(self.sample_seed, 1.0, tree=tree)
+
     def round_calls(self):
         eng = self.eng
         eng.glance_draft_block()
         eng.glance_build_tree(self.cand_ids, self.cand_lp)
-        eng.glance_verify_tree()
+        self.verify()
         eng.glance_accept_commit()
 
     def round_e2e(self):
@@ -327,6 +334,8 @@ def main():
     ap.add_argument("--no-lookahead", action="store_true",
                     help="random candidates instead of the look-ahead (profiling captures: fewer launches)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end arm (profiling captures)")
+    ap.add_argument("--sample-seed", type=int, default=None,
+                    help="run the rounds in sampling mode at temperature 1 with this seed (default: greedy)")
     ap.add_argument("--no-ar", action="store_true", help="skip the plain greedy-decoding comparison arm")
     ap.add_argument("--no-graph", action="store_true", help="launch the round's kernels one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
@@ -343,7 +352,8 @@ def main():
                           f"N={cfg.tree_N} p_m={cfg.p_m} batch {cfg.batch}",
               "l2": "inputs larger than L2: every round streams all weights (~15 GB at the 7B shape) and an untimed "
                     "look-ahead of L verify passes runs between timed rounds",
-              "replicas": world, "launch": "plain launches" if args.no_graph else "one CUDA graph per round"}
+              "replicas": world, "launch": "plain launches" if args.no_graph else "one CUDA graph per round",
+              "decisions": "greedy arg-max" if args.sample_seed is None else f"sampling, temperature 1, seed {args.sample_seed}"}
 
     if args.impl == "reference":
         if rank != 0:
@@ -382,6 +392,7 @@ def main():
     torch.manual_seed(0)
     bench = RoundBench(cfg, dev, rank)
     bench.no_lookahead = args.no_lookahead
+    bench.sample_seed = args.sample_seed
     eng = bench.eng
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 

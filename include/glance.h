@@ -147,6 +147,18 @@ int32_t glance_build_tree(glance_ctx *ctx, int32_t batch, const int32_t *root, c
 int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree,
                            int32_t *argmax, void *hidden, float *logits_dbg);
 
+/* Sampling mode (Limitations section: under sampling the walk draws each token from the verified row of its
+ * node and descends while the draw is a child).  Same pass as glance_verify_tree, but draws [batch][N] (device)
+ * holds one draw per row from softmax(row / temperature) instead of the arg-max; pass it to
+ * glance_accept_commit in place of argmax.  The draw is arg-max_v(row[v] / temperature + g(seed, p, v)) where p
+ * is the position of the token being drawn (seq_len + depth + 1) and g is standard Gumbel noise
+ * -log(-log u), u = ((w >> 9) + 0.5) 2^-23, w = word (v mod 4) of Philox4x32-10 with counter (v / 4, p, 0, 0)
+ * and key (seed low word, seed high word): the noise depends on the position, not on the row or the round, so
+ * the committed tokens equal plain ancestral sampling with the same field.  temperature > 0 (host value);
+ * ties to the lowest id; logits_dbg (if given) receives the unperturbed logits. */
+int32_t glance_verify_tree_sample(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, uint64_t seed,
+                                  float temperature, int32_t *draws, void *hidden, float *logits_dbg);
+
 /* Algorithm 1 lines 5-12 + commit.  Walks from the root along argmax while the token is a child
  * in the tree; then, per layer, moves cache row seq_len + path[d] to row seq_len + d (d = 1..a),
  * gathers hidden[path[0..a]] into feat, sets feat_count = a+1, seq_len += a+1, root = new root.

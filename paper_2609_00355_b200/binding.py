@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libglance.so")
 EXPORTS = [
     "glance_status_string", "glance_workspace_bytes", "glance_create", "glance_destroy", "glance_prefill",
     "glance_seq_truncate", "glance_draft_block", "glance_build_tree", "glance_verify_tree",
+    "glance_verify_tree_sample",
     "glance_accept_commit", "glance_commit_forced", "glance_poll_status", "glance_launch_count",
     "glance_debug_attention", "glance_debug_gemm", "glance_profile_enable", "glance_profile_read",
     "glance_topk_static", "glance_debug_trace",
@@ -82,6 +83,9 @@ def load_library() -> C.CDLL:
     lib.glance_build_tree.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Tree)]
     lib.glance_verify_tree.restype = C.c_int32
     lib.glance_verify_tree.argtypes = [C.c_void_p, C.POINTER(Seqs), C.POINTER(Tree), C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.glance_verify_tree_sample.restype = C.c_int32
+    lib.glance_verify_tree_sample.argtypes = [C.c_void_p, C.POINTER(Seqs), C.POINTER(Tree), C.c_uint64, C.c_float, C.c_void_p,
+                                              C.c_void_p, C.c_void_p]
     lib.glance_accept_commit.restype = C.c_int32
     lib.glance_accept_commit.argtypes = [C.c_void_p, C.POINTER(Seqs), C.POINTER(Tree), C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p]
@@ -255,6 +259,14 @@ class Engine:
         tree = tree or self.tree
         _check(self.lib.glance_verify_tree(self.ctx, C.byref(self.seqs), C.byref(tree.c), _ptr(self.argmax),
                                            _ptr(self.hidden), _ptr(logits_dbg)), "glance_verify_tree")
+
+    def glance_verify_tree_sample(self, seed: int, temperature: float = 1.0, tree: Optional[TreeBuffers] = None,
+                                  logits_dbg: Optional[torch.Tensor] = None):
+        """Sampling mode: self.argmax receives one draw per row instead of the arg-max."""
+        tree = tree or self.tree
+        _check(self.lib.glance_verify_tree_sample(self.ctx, C.byref(self.seqs), C.byref(tree.c), C.c_uint64(seed),
+                                                  C.c_float(temperature), _ptr(self.argmax), _ptr(self.hidden),
+                                                  _ptr(logits_dbg)), "glance_verify_tree_sample")
 
     def glance_accept_commit(self, tree: Optional[TreeBuffers] = None, argmax: Optional[torch.Tensor] = None):
         tree = tree or self.tree

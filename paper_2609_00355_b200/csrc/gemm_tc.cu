@@ -39,6 +39,24 @@ struct alignas(8) Barriers {
     int abort_flag;
 };
 
+// Philox4x32-10 (Salmon et al., SC 2011): the counter-based generator behind the sampling mode's noise field.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+        c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+        k.x += 0x9E3779B9u;
+        k.y += 0xBB67AE85u;
+    }
+    return c;
+}
+// standard Gumbel noise from one 32-bit word: u = ((w >> 9) + 0.5) 2^-23 lies strictly inside (0,1)
+__device__ __forceinline__ float gumbel_from_word(uint32_t w) {
+    const float u = ((float)(w >> 9) + 0.5f) * 1.1920928955078125e-07f;
+    return -logf(-logf(u));
+}
+
 // MODE 0: fp32 planes              MODE 1: SwiGLU (64 gate + 64 up rows per tile)   MODE 2: arg-max (+ optional logits)
 // MODE 3: split-K over a cluster, residual add + bf16 copy scaled by the next norm's gain + sum of squares
 // MODE 4: split-K over a cluster, rotary embedding + q / paged K,V write
@@ -323,6 +341,19 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                     }
                 }
                 if (MODE == 2) {
+                    if (a.sample_pos) {
+                        // sampling mode: a draw from softmax(row * inv_temperature) is the arg-max of the row plus
+                        // Gumbel noise; the noise of (token position, vocabulary id) is a fixed field, so the draw
+                        // for a position does not depend on which row or round asks for it.  Ids f..f+3 are the
+                        // four words of the block (f / 4, position of the predicted token).
+                        const uint32_t pos = (uint32_t)(a.sample_pos[rr] + 1);
+                        const uint4 w = philox4x32_10(make_uint4((uint32_t)(f >> 2), pos, 0u, 0u),
+                                                      make_uint2((uint32_t)a.sample_seed, (uint32_t)(a.sample_seed >> 32)));
+                        v.x = v.x * a.sample_inv_t + gumbel_from_word(w.x);
+                        v.y = v.y * a.sample_inv_t + gumbel_from_word(w.y);
+                        v.z = v.z * a.sample_inv_t + gumbel_from_word(w.z);
+                        v.w = v.w * a.sample_inv_t + gumbel_from_word(w.w);
+                    }
                     unsigned long long key = 0ull, k2;
                     if (f < a.Nout) key = pack_val_id(v.x, f);
                     if (f + 1 < a.Nout) { k2 = pack_val_id(v.y, f + 1); key = k2 > key ? k2 : key; }

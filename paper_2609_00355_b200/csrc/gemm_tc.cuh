@@ -21,6 +21,11 @@ struct TcGemmArgs {
     int32_t *argmax;
     int32_t *counter;
     int32_t *status;
+    // mode 2, sampling: sample_pos[r] = position of row r (the draw is for position + 1), or nullptr for the plain
+    // arg-max; values are scaled by sample_inv_t and perturbed by the Gumbel field of (sample_seed, position, id)
+    const int32_t *sample_pos;
+    unsigned long long sample_seed;
+    float sample_inv_t;
     // row scales (modes 0, 1, 2, 4): row r is multiplied by rsqrt(sum_i ssq[i*ssq_stride + r] / K + eps); nullptr = 1
     const float *ssq;
     int n_ssq, ssq_stride;

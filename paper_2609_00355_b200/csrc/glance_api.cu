@@ -121,6 +121,9 @@ bool config_ok(const glance_config *c) {
 }  // namespace
 
 struct glance_ctx {
+    bool sample_on = false;                 // the LM head of the pass in flight draws instead of taking the arg-max
+    unsigned long long sample_seed = 0;
+    float sample_inv_t = 1.f;
     glance_config cfg;
     Dims dims;
     Workspace ws;
@@ -342,6 +345,9 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
         TcGemmArgs g{};
         g.Nout = c.vocab; g.K = c.hidden; g.R = ps.R; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.argmax = argmax;
         g.x_lo_row = 0;      // logits only decide an arg-max / top-k: one term is enough
+        if (ctx->sample_on) {
+            g.sample_pos = ctx->ws.row_pos; g.sample_seed = ctx->sample_seed; g.sample_inv_t = ctx->sample_inv_t;
+        }
         with_row_scales(ctx, g);
         gemm(ctx, 2, ctx->lm_head, ctx->ws.xn, ctx->dims.Rmax, g);
     }
@@ -561,11 +567,11 @@ int32_t glance_build_tree(glance_ctx *ctx, int32_t batch, const int32_t *root, c
     return finish(ctx);
 }
 
-int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, int32_t *argmax,
-                           void *hidden, float *logits_dbg) {
+static int32_t verify_common(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, int32_t *decisions,
+                             void *hidden, float *logits_dbg) {
     int32_t rc = check_seqs(ctx, seqs);
     if (rc) return rc;
-    if (!tree || !tree->token || !tree->depth || !tree->anc || !argmax || !hidden) return GLANCE_E_INVALID_ARG;
+    if (!tree || !tree->token || !tree->depth || !tree->anc || !decisions || !hidden) return GLANCE_E_INVALID_ARG;
     const glance_config &c = ctx->cfg;
     Workspace &ws = ctx->ws;
     const int batch = seqs->batch, N = c.tree_N;
@@ -577,8 +583,26 @@ int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glanc
     vs.page_table = seqs->page_table; vs.out = rowout_of(ctx); vs.meta = meta_of(ctx); vs.status = ws.status;
     LAUNCH(ctx, KIND_SETUP, launch_setup_verify(vs, ctx->stream));
     PassInfo ps{batch * N, batch * N, batch, N, tree->anc, seqs, 0};
-    run_target(ctx, ps, (bf16 *)hidden, logits_dbg, argmax);
+    run_target(ctx, ps, (bf16 *)hidden, logits_dbg, decisions);
     return finish(ctx);
+}
+
+int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, int32_t *argmax,
+                           void *hidden, float *logits_dbg) {
+    if (!ctx) return GLANCE_E_INVALID_ARG;
+    ctx->sample_on = false;
+    return verify_common(ctx, seqs, tree, argmax, hidden, logits_dbg);
+}
+
+int32_t glance_verify_tree_sample(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, uint64_t seed,
+                                  float temperature, int32_t *draws, void *hidden, float *logits_dbg) {
+    if (!ctx || !(temperature > 0.f)) return GLANCE_E_INVALID_ARG;
+    ctx->sample_on = true;
+    ctx->sample_seed = seed;
+    ctx->sample_inv_t = 1.f / temperature;
+    const int32_t rc = verify_common(ctx, seqs, tree, draws, hidden, logits_dbg);
+    ctx->sample_on = false;
+    return rc;
 }
 
 static int32_t commit_common(glance_ctx *ctx, const glance_seqs *seqs, WalkCommit &wc, const void *hidden) {

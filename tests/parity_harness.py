@@ -111,17 +111,22 @@ class ParityRun:
                 close(V, st.hV[:n], f"head V seq {s}")
 
     # ---- oracle look-ahead: the greedy continuation after the pending root -------------------
-    def oracle_continuation(self, s: int, n: int):
+    def oracle_continuation(self, s: int, n: int, sample_seed=None):
         st = copy.deepcopy(self.states[s])
         Y = []
         for _ in range(n):
-            info = O.spec_round(self.sh, self.tw, self.hw, st, self.cfg.block_B, self.cfg.topk, 1,
-                                tree=O.chain_tree(st.root, [], 1))
+            if sample_seed is None:
+                info = O.spec_round(self.sh, self.tw, self.hw, st, self.cfg.block_B, self.cfg.topk, 1,
+                                    tree=O.chain_tree(st.root, [], 1))
+            else:
+                info = O.spec_round_sampled(self.sh, self.tw, self.hw, st, self.cfg.block_B, self.cfg.topk, 1,
+                                            sample_seed, tree=O.chain_tree(st.root, [], 1))
             Y.append(info["new_root"])
         return Y
 
     # ---- one teacher-forced round -------------------------------------------------------------
-    def round(self, p_m=None, check_draft=True):
+    def round(self, p_m=None, check_draft=True, sample_seed=None):
+        """sample_seed: run the round in sampling mode (temperature 1) with this seed instead of greedily."""
         cfg, eng, sh = self.cfg, self.eng, self.sh
         B, k, N, L, V = cfg.block_B, cfg.topk, cfg.tree_N, cfg.L, cfg.vocab
         dev = eng.device
@@ -153,7 +158,7 @@ class ParityRun:
         # (2) tree: either from the library's own draft output or from controlled-match candidates
         Ys = None
         if p_m is not None:
-            Ys = [self.oracle_continuation(s, L + 1) for s in range(self.batch)]
+            Ys = [self.oracle_continuation(s, L + 1, sample_seed) for s in range(self.batch)]
             lp_c = synth.controlled_marginals(p_m, k, L)
             ids_in = np.stack([synth.controlled_candidates(Ys[s][:L], p_m, k, L, V, self.rng) for s in range(self.batch)])
             lp_in = np.stack([lp_c] * self.batch)
@@ -171,7 +176,10 @@ class ParityRun:
         vlog = torch.zeros(self.batch, N, V, dtype=torch.float32, device=dev)
         pool_before = eng.kv_pool.clone()
         state_before = eng.snapshot_state()
-        eng.glance_verify_tree(logits_dbg=vlog)
+        if sample_seed is None:
+            eng.glance_verify_tree(logits_dbg=vlog)
+        else:
+            eng.glance_verify_tree_sample(sample_seed, 1.0, logits_dbg=vlog)
         am_g = eng.argmax.cpu().numpy()
         infos = []
         for s, st in enumerate(self.states):
@@ -181,16 +189,28 @@ class ParityRun:
             scale = float(ol[:n].abs().max())
             self.stats["max_rel_logit"] = max(self.stats["max_rel_logit"], close(vlog[s, :n], ol[:n], "verify logits", scale))
             close(eng.hidden[s, :n], oh[:n], "verify hidden")
-            oam = O.argmax_lowest(ol)
-            top2 = torch.topk(ol, 2, dim=-1).values
-            margin = (top2[:, 0] - top2[:, 1]).numpy()
+            if sample_seed is None:
+                oam = O.argmax_lowest(ol)
+                top2 = torch.topk(ol, 2, dim=-1).values
+                margin = (top2[:, 0] - top2[:, 1]).numpy()
+            else:
+                # one draw per row: arg-max of the row perturbed by the noise field of the predicted position
+                positions = [st.P + int(d) + 1 for d in trees[s].depth]
+                oam, margin = O.sample_rows(ol, positions, sample_seed)
             for i in range(n):
                 if margin[i] > MARGIN:
-                    assert am_g[s, i] == oam[i], f"argmax row {i} (margin {margin[i]:.3f})"
+                    assert am_g[s, i] == oam[i], f"decision row {i} (margin {margin[i]:.3f})"
                 elif am_g[s, i] != oam[i]:
                     self.stats["argmax_excused"] += 1
-            # the library's argmax is the argmax of its own fp32 logits, ties to the lowest id
-            assert np.array_equal(am_g[s], O.argmax_lowest(vlog[s].cpu()))
+            if sample_seed is None:
+                # the library's argmax is the argmax of its own fp32 logits, ties to the lowest id
+                assert np.array_equal(am_g[s], O.argmax_lowest(vlog[s].cpu()))
+            else:
+                # the library's draws are the arg-max of its own logits plus the same noise field (the two sides
+                # evaluate the logarithms of the Gumbel transform independently: near-ties are exempt)
+                own, own_margin = O.sample_rows(vlog[s].cpu(), positions, sample_seed)
+                for i in range(n):
+                    assert am_g[s, i] == own[i] or own_margin[i] < 1e-3, f"draw row {i} is not the perturbed arg-max"
             infos.append((ol, oh, oam))
         # tree K/V rows written at P + i
         for s, st in enumerate(self.states):

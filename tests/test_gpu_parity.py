@@ -385,3 +385,23 @@ def test_rounds_tiny_chain_k1(harness):
         run.round(p_m=0.8, check_draft=(r == 0))
     print("chain parity stats:", run.stats)
     assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_tiny_sampling_mode(harness):
+    """Sampling walk at temperature 1: every row's decision is a draw (Gumbel-max over the position-keyed noise
+    field); draws, walk, commit and state against the oracle's sampling rounds, with drafted and planted trees."""
+    run = harness.ParityRun(synth.CONFIGS["tiny"])
+    run.check_state()
+    for r in range(8):
+        run.round(p_m=(0.7 if r % 2 else None), check_draft=False, sample_seed=0xC0FFEE + 17)
+    run.check_head_state()
+    print("sampling parity stats:", run.stats)
+    assert run.stats["accepted"] > 0
+
+
+def test_rounds_small_sampling_mode(harness):
+    run = harness.ParityRun(synth.CONFIGS["small"])
+    for r in range(4):
+        run.round(p_m=0.6, check_draft=False, sample_seed=2024)
+    print("sampling parity stats (small):", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
