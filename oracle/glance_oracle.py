@@ -24,6 +24,9 @@ Readings of points the paper leaves open (each is restated in the design doc):
   * the one-layer head attends to [context features ; block] with one set of W_k/W_v;
     context features are the target's residual stream after the last layer, before the
     final norm, for committed positions only; the root enters as its embedding
+  * the multi-layer head (Section 3.2: five layers, keys/values from five kept target layers): head layer i is
+    one such layer with its own weights whose context keys/values are projections of the residual stream after
+    target layer taps[i]; the block rows flow through the head layers in order
   * q_j is the full-vocabulary softmax; candidates are restricted to per-slot top-k
   * ties: argmax/top-k prefer the lowest id; tree order is (score desc, depth asc,
     path key asc); node index = position in that order
@@ -37,6 +40,8 @@ attention against torch SDPA; top-k / lse against torch.topk / logsumexp; rotary
 relative-position identity; KV state after rounds = fresh prefill.
 sampling mode (Limitations section): Philox known-answer vectors, uniforms strictly inside (0,1), draw frequencies
 against the softmax, and tree rounds against plain ancestral sampling with the same noise field.
+multi-layer head: taps against truncated cache-free forwards, the stack against repeated decoder_layer calls,
+the one-tap case bit-identical to the one-layer head, head state after rounds = fresh prefill for every layer.
 draft_block (the reading of Section 3.2 stated above; the paper prints no worked example of the head):
 equality with decoder_layer under an all-ones mask, the identity-layer closed form (W_o = W_down = 0), the
 single-key closed form (B = 1, no context) written out in float64, invariance under a permutation of the
@@ -71,11 +76,17 @@ class Shape:
     vocab: int
     rms_eps: float = 1e-6
     rope_theta: float = 1e6
+    head_taps: Tuple[int, ...] = ()      # () = one head layer fed by the last target layer; else one tap per head layer
 
     @staticmethod
     def of(cfg) -> "Shape":
         return Shape(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn,
-                     cfg.vocab, cfg.rms_eps, cfg.rope_theta)
+                     cfg.vocab, cfg.rms_eps, cfg.rope_theta, tuple(getattr(cfg, "head_taps", ()) or ()))
+
+    @property
+    def taps(self) -> Tuple[int, ...]:
+        """Target layer (0-based) whose output feeds head layer i."""
+        return self.head_taps if self.head_taps else (self.n_layers - 1,)
 
 
 def widen(w):
@@ -399,15 +410,40 @@ class SeqState:
     V: List[torch.Tensor]
     hK: torch.Tensor             # head context keys [cap,Hkv,d]
     hV: torch.Tensor
-    feat: torch.Tensor           # [cap,H] target features of committed positions
+    feat: torch.Tensor           # [cap,H] target features of committed positions (tap of head layer 0)
     tokens: List[int] = field(default_factory=list)   # committed tokens after the context (for audits)
+    # head layers 1.. of a multi-layer head (Section 3.2: five layers, one tapped target layer each)
+    hK_more: List[torch.Tensor] = field(default_factory=list)
+    hV_more: List[torch.Tensor] = field(default_factory=list)
+    feat_more: List[torch.Tensor] = field(default_factory=list)
+
+
+def head_layer(hw: dict, i: int) -> dict:
+    """Weights of head layer i: layer 0 lives in the flat keys, layers 1.. in hw["more"]."""
+    return hw if i == 0 else hw["more"][i - 1]
 
 
 def head_context_kv(sh: Shape, hw: dict, feats: torch.Tensor, pos: torch.Tensor):
-    """K/V rows the head keeps for committed positions: projections of rms(feature) * g_ctx, keys rotated."""
+    """K/V rows a head layer keeps for committed positions: projections of rms(feature) * g_ctx, keys rotated.
+    `hw` is that layer's weight dict; `feats` the hidden states of the target layer it taps."""
     hn = rmsnorm(feats, hw["ctx_norm"], sh.rms_eps)
     _, k, v = split_qkv(sh, hn @ hw["wqkv"].T)
     return rope(k, pos, sh.rope_theta), v
+
+
+def _set_head_rows(sh: Shape, hw: dict, st: "SeqState", rows: torch.Tensor, tap_hidden: Sequence[torch.Tensor]) -> None:
+    """Store the tapped features of `rows` and fold them into every head layer's context K/V."""
+    for i, f in enumerate(tap_hidden):
+        feat = st.feat if i == 0 else st.feat_more[i - 1]
+        hK = st.hK if i == 0 else st.hK_more[i - 1]
+        hV = st.hV if i == 0 else st.hV_more[i - 1]
+        feat[rows] = f
+        hK[rows], hV[rows] = head_context_kv(sh, head_layer(hw, i), f, rows)
+
+
+def _taps_of(hidden: torch.Tensor) -> List[torch.Tensor]:
+    """hidden [n,H] (one tap) or [T,n,H] (one slice per head layer) -> list of [n,H]."""
+    return [hidden] if hidden.dim() == 2 else [hidden[i] for i in range(hidden.shape[0])]
 
 
 def prefill(sh: Shape, tw: dict, hw: dict, ctx_embeds: torch.Tensor, cap: int) -> SeqState:
@@ -417,19 +453,23 @@ def prefill(sh: Shape, tw: dict, hw: dict, ctx_embeds: torch.Tensor, cap: int) -
     mask = torch.tril(torch.ones(P, P, dtype=torch.bool))
     x = ctx_embeds.clone()
     Ks, Vs = [], []
-    for lw in tw["layers"]:
+    tapped = {}
+    for l, lw in enumerate(tw["layers"]):
         Kc = torch.zeros(cap, sh.n_kv_heads, sh.head_dim)
         Vc = torch.zeros(cap, sh.n_kv_heads, sh.head_dim)
         x = decoder_layer(sh, lw, x, pos, Kc, Vc, pos, mask)
         Ks.append(Kc); Vs.append(Vc)
+        if l in sh.taps:
+            tapped[l] = x
     logits = rmsnorm(x[-1:], tw["final_norm"], sh.rms_eps) @ tw["lm_head"].T
     root = int(argmax_lowest(logits)[0])
-    hK = torch.zeros(cap, sh.n_kv_heads, sh.head_dim)
-    hV = torch.zeros(cap, sh.n_kv_heads, sh.head_dim)
-    hK[:P], hV[:P] = head_context_kv(sh, hw, x, pos)
-    feat = torch.zeros(cap, sh.hidden)
-    feat[:P] = x
-    return SeqState(P, root, Ks, Vs, hK, hV, feat)
+    T = len(sh.taps)
+    zkv = lambda: torch.zeros(cap, sh.n_kv_heads, sh.head_dim)
+    st = SeqState(P, root, Ks, Vs, zkv(), zkv(), torch.zeros(cap, sh.hidden),
+                  hK_more=[zkv() for _ in range(T - 1)], hV_more=[zkv() for _ in range(T - 1)],
+                  feat_more=[torch.zeros(cap, sh.hidden) for _ in range(T - 1)])
+    _set_head_rows(sh, hw, st, pos, [tapped[t] for t in sh.taps])
+    return st
 
 
 def draft_block(sh: Shape, tw: dict, hw: dict, st: SeqState, B: int) -> torch.Tensor:
@@ -442,17 +482,22 @@ def draft_block(sh: Shape, tw: dict, hw: dict, st: SeqState, B: int) -> torch.Te
     X = hw["mask_embed"][None, :].repeat(B, 1)
     X[0] = tw["embed"][st.root]
     pos = torch.arange(P, P + B)
-    hn = rmsnorm(X, hw["ln1"], sh.rms_eps)
-    q, k, v = split_qkv(sh, hn @ hw["wqkv"].T)
-    q = rope(q, pos, sh.rope_theta)
-    k = rope(k, pos, sh.rope_theta)
-    K = torch.cat([st.hK[:P], k], dim=0)
-    V = torch.cat([st.hV[:P], v], dim=0)
     mask = torch.ones(B, P + B, dtype=torch.bool)
-    o = attention(q, K, V, mask)
-    X = X + o.reshape(B, -1) @ hw["wo"].T
-    h2 = rmsnorm(X, hw["ln2"], sh.rms_eps)
-    X = X + mlp(sh, h2, hw["wgu"], hw["wd"])
+    for i in range(len(sh.taps)):
+        # head layer i: context keys/values come from the target layer it taps, block rows from the layer below
+        lw = head_layer(hw, i)
+        hK = st.hK if i == 0 else st.hK_more[i - 1]
+        hV = st.hV if i == 0 else st.hV_more[i - 1]
+        hn = rmsnorm(X, lw["ln1"], sh.rms_eps)
+        q, k, v = split_qkv(sh, hn @ lw["wqkv"].T)
+        q = rope(q, pos, sh.rope_theta)
+        k = rope(k, pos, sh.rope_theta)
+        K = torch.cat([hK[:P], k], dim=0)
+        V = torch.cat([hV[:P], v], dim=0)
+        o = attention(q, K, V, mask)
+        X = X + o.reshape(B, -1) @ lw["wo"].T
+        h2 = rmsnorm(X, lw["ln2"], sh.rms_eps)
+        X = X + mlp(sh, h2, lw["wgu"], lw["wd"])
     return rmsnorm(X, hw["final_norm"], sh.rms_eps) @ tw["lm_head"].T
 
 
@@ -479,17 +524,23 @@ def verify_tree(sh: Shape, tw: dict, st: SeqState, tree: Tree, row_embeds: Optio
     """Algorithm 1 lines 3-4: the packed ancestor-masked target pass.
 
     Row i = node i at position P+depth[i]; K/V of node i written to cache row P+i;
-    returns (logits [N,V], hidden [N,H]) with hidden = pre-final-norm residual stream.
+    returns (logits [N,V], hidden [N,H]) with hidden = the residual stream after the tapped target layer (the last
+    one for the one-layer head: the pre-final-norm stream); [T,N,H] for a head of T layers.
     """
     P, N = st.P, tree.N
     x = tw["embed"][torch.as_tensor(tree.token, dtype=torch.long)].clone() if row_embeds is None else row_embeds.clone()
     pos = torch.as_tensor(P + tree.depth.astype(np.int64))
     rows = torch.arange(P, P + N)
     mask = visibility(tree, P)
+    tapped = {}
     for l, lw in enumerate(tw["layers"]):
         x = decoder_layer(sh, lw, x, pos, st.K[l], st.V[l], rows, mask)
+        if l in sh.taps:
+            tapped[l] = x
     logits = rmsnorm(x, tw["final_norm"], sh.rms_eps) @ tw["lm_head"].T
-    return logits, x
+    if len(sh.taps) == 1:
+        return logits, tapped[sh.taps[0]]
+    return logits, torch.stack([tapped[t] for t in sh.taps])     # [T,N,H], one slice per head layer
 
 
 def walk(tree: Tree, argmax: np.ndarray):
@@ -520,10 +571,9 @@ def commit(sh: Shape, hw: dict, st: SeqState, path: Sequence[int], hidden: torch
         for dd in range(1, a + 1):
             st.K[l][P + dd] = st.K[l][P + path[dd]].clone()
             st.V[l][P + dd] = st.V[l][P + path[dd]].clone()
-    f = hidden[torch.as_tensor(list(path), dtype=torch.long)]
+    idx = torch.as_tensor(list(path), dtype=torch.long)
     pos = torch.arange(P, P + a + 1)
-    st.feat[P:P + a + 1] = f
-    st.hK[P:P + a + 1], st.hV[P:P + a + 1] = head_context_kv(sh, hw, f, pos)
+    _set_head_rows(sh, hw, st, pos, [h[idx] for h in _taps_of(hidden)])
     st.tokens.extend([st.root] + [int(t) for t in out])
     st.P = P + a + 1
     st.root = int(new_root)

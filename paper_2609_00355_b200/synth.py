@@ -47,6 +47,13 @@ class RoundConfig:
     page_size: int = 64
     rms_eps: float = 1e-6
     rope_theta: float = 1e6
+    # () = one head layer fed by the last target layer; otherwise head layer i reads the hidden states after
+    # target layer head_taps[i] (0-based), one tap per head layer (Section 3.2: five layers, five kept target layers)
+    head_taps: tuple = ()
+
+    @property
+    def head_layers(self) -> int:
+        return max(1, len(self.head_taps))
 
     @property
     def L(self) -> int:
@@ -84,7 +91,8 @@ def make_weights(cfg: RoundConfig, device="cpu", seed: int = 0):
     target: embed [V,H], lm_head [V,H], final_norm [H], layers: list of dicts with
             ln1 [H], wqkv [(Hq+2Hkv)d, H], wo [H, Hq d], ln2 [H], wgu [2F, H], wd [H, F]
     head:   mask_embed [H], ctx_norm [H], ln1, wqkv, wo, ln2, wgu, wd, final_norm
-            (embed and lm_head are shared with the target)
+            (embed and lm_head are shared with the target); with cfg.head_taps of T > 1 entries also
+            more: list of T-1 dicts {ctx_norm, ln1, wqkv, wo, ln2, wgu, wd} for head layers 1..T-1
     """
     gen = torch.Generator(device=device)
     gen.manual_seed(seed)
@@ -118,6 +126,20 @@ def make_weights(cfg: RoundConfig, device="cpu", seed: int = 0):
         "wd": _normal_bf16((H, F), std, gen, device),
         "final_norm": ones(),
     }
+    # head layers 1.. (drawn after everything else, so a one-layer head keeps its bits)
+    more = []
+    for _ in range(cfg.head_layers - 1):
+        more.append({
+            "ctx_norm": ones(),
+            "ln1": ones(),
+            "wqkv": _normal_bf16((qkv_out, H), std, gen, device),
+            "wo": _normal_bf16((H, cfg.n_q_heads * d), std, gen, device),
+            "ln2": ones(),
+            "wgu": _normal_bf16((2 * F, H), std, gen, device),
+            "wd": _normal_bf16((H, F), std, gen, device),
+        })
+    if more:
+        head["more"] = more
     return target, head
 
 

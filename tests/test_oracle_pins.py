@@ -504,6 +504,83 @@ def test_draft_block_context_order_invariance(tiny):
     assert float((dl - dl3).abs().max()) > 1e-4 * float(dl.abs().max())
 
 
+# ------------------------------------------------------------------ multi-layer, multi-tap head
+
+@pytest.fixture(scope="module")
+def tiny2():
+    """The tiny configuration with a two-layer head: head layer 0 taps target layer 0, head layer 1 taps layer 1."""
+    torch.manual_seed(0)
+    cfg = synth.CONFIGS["tiny"].replace(head_taps=(0, 1))
+    tw_b, hw_b = synth.make_weights(cfg)
+    img, ids = synth.make_context(cfg)
+    t = Tiny()
+    t.cfg, t.sh = cfg, O.Shape.of(cfg)
+    t.tw, t.hw = O.widen(tw_b), O.widen(hw_b)
+    t.ctx = O.context_embeddings(t.tw, img, ids.numpy())
+    t.n_new = 40
+    t.Y, t.margins = O.greedy_ar_cachefree(t.sh, t.tw, t.ctx, t.n_new)
+    t.cap = cfg.ctx + t.n_new + cfg.tree_N + 64
+    return t
+
+
+def test_head_taps_are_the_named_target_layers(tiny2):
+    """The features a head layer reads are the residual stream after the target layer it taps: equal to the output
+    of a cache-free causal forward through the target truncated after that layer."""
+    st = _fresh(tiny2)
+    P = st.P
+    for i, t in enumerate(tiny2.sh.taps):
+        sh_t = O.Shape(t + 1, *[getattr(tiny2.sh, f) for f in ("hidden", "n_q_heads", "n_kv_heads", "head_dim", "ffn", "vocab")])
+        tw_t = dict(tiny2.tw, layers=tiny2.tw["layers"][:t + 1])
+        _, feats = O.full_causal_forward(sh_t, tw_t, tiny2.ctx)
+        got = st.feat if i == 0 else st.feat_more[i - 1]
+        assert float((got[:P] - feats).abs().max()) <= 1e-5 * float(feats.abs().max())
+    assert not torch.equal(st.feat[:P], st.feat_more[0][:P])
+
+
+def test_multilayer_head_is_a_stack_of_unmasked_decoder_layers(tiny2):
+    """Each head layer is one decoder layer over the block rows whose context keys/values are that layer's own
+    projections of its tap: the block pushed through decoder_layer once per head layer gives the same logits."""
+    st = _fresh(tiny2)
+    sh, B, P = tiny2.sh, tiny2.cfg.block_B, st.P
+    dl = O.draft_block(sh, tiny2.tw, tiny2.hw, st, B)
+    X = tiny2.hw["mask_embed"][None, :].repeat(B, 1)
+    X[0] = tiny2.tw["embed"][st.root]
+    pos = torch.arange(P, P + B)
+    for i in range(2):
+        lw = O.head_layer(tiny2.hw, i)
+        Kc = (st.hK if i == 0 else st.hK_more[i - 1]).clone()
+        Vc = (st.hV if i == 0 else st.hV_more[i - 1]).clone()
+        X = O.decoder_layer(sh, {k: lw[k] for k in ("ln1", "wqkv", "wo", "ln2", "wgu", "wd")}, X, pos, Kc, Vc, pos,
+                            torch.ones(B, P + B, dtype=torch.bool))
+    ref = O.rmsnorm(X, tiny2.hw["final_norm"], sh.rms_eps) @ tiny2.tw["lm_head"].T
+    assert float((dl - ref).abs().max()) <= 1e-5 * float(ref.abs().max())
+    # the second layer matters, and so does which tap feeds it
+    one = O.draft_block(O.Shape.of(tiny2.cfg.replace(head_taps=(0,))), tiny2.tw, tiny2.hw, st, B)
+    assert float((dl - one).abs().max()) > 1e-3 * float(dl.abs().max())
+
+
+def test_explicit_last_layer_tap_is_the_one_layer_head(tiny):
+    """head_taps = (n_layers - 1,) spelled out is the default one-layer head, bit for bit."""
+    cfg = tiny.cfg.replace(head_taps=(tiny.cfg.n_layers - 1,))
+    sh = O.Shape.of(cfg)
+    st_a, st_b = _fresh(tiny), O.prefill(sh, tiny.tw, tiny.hw, tiny.ctx, tiny.cap)
+    assert torch.equal(st_a.hK, st_b.hK) and torch.equal(st_a.feat, st_b.feat)
+    assert torch.equal(O.draft_block(tiny.sh, tiny.tw, tiny.hw, st_a, cfg.block_B),
+                       O.draft_block(sh, tiny.tw, tiny.hw, st_b, cfg.block_B))
+
+
+def test_multilayer_head_rounds_lossless_and_state_equals_fresh_prefill(tiny2):
+    """Rounds with the two-layer head stay lossless (Theorem 1), and the lazily appended head state of BOTH layers
+    (features, keys, values of the committed positions) equals what a fresh prefill of the same tokens builds."""
+    st, acc = _run_rounds(tiny2, lambda st, Y: None, 6)
+    x = torch.cat([tiny2.ctx, tiny2.tw["embed"][torch.tensor(st.tokens)]], dim=0)
+    ref = O.prefill(tiny2.sh, tiny2.tw, tiny2.hw, x, tiny2.cap)
+    assert ref.P == st.P and ref.root == st.root
+    for a, b in ((st.hK, ref.hK), (st.hV, ref.hV), (st.feat, ref.feat), (st.hK_more[0], ref.hK_more[0]),
+                 (st.hV_more[0], ref.hV_more[0]), (st.feat_more[0], ref.feat_more[0])):
+        assert float((a[:st.P] - b[:st.P]).abs().max()) < 1e-4 * max(1.0, float(b[:st.P].abs().max()))
+
+
 # ------------------------------------------------------------------ sampling mode
 
 def test_philox_known_answers():
