@@ -57,7 +57,7 @@ def round_algorithmic_bytes(cfg) -> float:
     P = cfg.ctx
     kv_layer = 2.0 * P * cfg.n_kv_heads * d * 2
     target = cfg.n_layers * (layer + kv_layer + 2.0 * cfg.tree_N * cfg.n_kv_heads * d * 2) + 2.0 * V * H
-    head = layer + kv_layer + 2.0 * V * H
+    head = getattr(cfg, "head_layers", 1) * (layer + kv_layer) + 2.0 * V * H
     return target + head
 
 
@@ -334,6 +334,8 @@ def main():
     ap.add_argument("--no-lookahead", action="store_true",
                     help="random candidates instead of the look-ahead (profiling captures: fewer launches)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the end-to-end arm (profiling captures)")
+    ap.add_argument("--head-taps", type=int, nargs="+", default=None,
+                    help="multi-layer block head: one tapped target layer (0-based) per head layer, e.g. 1 7 14 21 27")
     ap.add_argument("--sample-seed", type=int, default=None,
                     help="run the rounds in sampling mode at temperature 1 with this seed (default: greedy)")
     ap.add_argument("--no-ar", action="store_true", help="skip the plain greedy-decoding comparison arm")
@@ -342,6 +344,8 @@ def main():
     cfg = synth.CONFIGS[args.config]
     if args.layers > 0:
         cfg = cfg.replace(n_layers=args.layers, name=f"{cfg.name}-{args.layers}layers")
+    if args.head_taps:
+        cfg = cfg.replace(head_taps=tuple(args.head_taps), name=f"{cfg.name}-head{len(args.head_taps)}")
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -353,6 +357,7 @@ def main():
               "l2": "inputs larger than L2: every round streams all weights (~15 GB at the 7B shape) and an untimed "
                     "look-ahead of L verify passes runs between timed rounds",
               "replicas": world, "launch": "plain launches" if args.no_graph else "one CUDA graph per round",
+              "head": "one layer on the last target layer" if not cfg.head_taps else f"{len(cfg.head_taps)} layers tapping target layers {list(cfg.head_taps)}",
               "decisions": "greedy arg-max" if args.sample_seed is None else f"sampling, temperature 1, seed {args.sample_seed}"}
 
     if args.impl == "reference":

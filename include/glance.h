@@ -46,10 +46,17 @@ typedef struct glance_ctx glance_ctx;
 /* Model and round shape.  Supported: head_dim in {64, 128}; hidden, ffn multiples of 64;
  * 2 <= block_B <= 16; 1 <= topk <= 16; 2 <= tree_N <= 128 (tree_N counts the root row: the
  * paper's budget is tree_N - 1); page_size = 64; n_q_heads a multiple of n_kv_heads. */
+#define GLANCE_MAX_HEAD_LAYERS 8
 typedef struct {
     int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
     float rms_eps, rope_theta;
     int32_t block_B, topk, tree_N, page_size, max_batch, max_pages_per_seq;
+    /* Block head depth (Section 3.2: five layers whose keys/values are the target's hidden states at five kept
+     * layers).  head_layers 0 or 1: one head layer fed by the last target layer (head_taps ignored).  Otherwise
+     * head layer i takes its context keys/values from the residual stream after target layer head_taps[i]
+     * (0-based, distinct, < n_layers); head_layers <= GLANCE_MAX_HEAD_LAYERS. */
+    int32_t head_layers;
+    int32_t head_taps[GLANCE_MAX_HEAD_LAYERS];
 } glance_config;
 
 /* Target decoder weights (device, bf16).  embed [V,H], lm_head [V,H], final_norm [H].
@@ -65,7 +72,11 @@ typedef struct {
  * mask_embed [H] fills the masked block slots; ctx_norm [H] normalises the target features that
  * form the head's context keys/values. */
 typedef struct {
-    const void *mask_embed, *ctx_norm, *ln1, *wqkv, *wo, *ln2, *wgu, *wd, *final_norm;
+    const void *ctx_norm, *ln1, *wqkv, *wo, *ln2, *wgu, *wd;
+} glance_head_layer;
+typedef struct {
+    const void *mask_embed, *ctx_norm, *ln1, *wqkv, *wo, *ln2, *wgu, *wd, *final_norm;   /* head layer 0 */
+    const glance_head_layer *more;   /* HOST array of head_layers - 1 entries (head layers 1..), or NULL */
 } glance_head_weights;
 
 /* Sequence state; every pointer is caller-owned device memory.
@@ -80,8 +91,9 @@ typedef struct {
     int32_t *root;             /* [batch] pending root token b; updated by commit */
     const int32_t *page_table; /* [batch][max_pages_per_seq] */
     void *kv_pool;             /* target: [n_layers][n_pages][2][Hkv][page_size][d] bf16 */
-    void *head_kv_pool;        /* head:   [n_pages][2][Hkv][page_size][d] bf16 */
-    void *feat;                /* [batch][block_B][H] bf16: target features of the rows committed last */
+    void *head_kv_pool;        /* head:   [head_layers][n_pages][2][Hkv][page_size][d] bf16 */
+    void *feat;                /* [head_layers][batch][block_B][H] bf16: tapped target features of the rows
+                                  committed last (slice i = the tap of head layer i) */
     int32_t *feat_count;       /* [batch] valid rows in feat (a+1 of the last round, 0 after prefill) */
 } glance_seqs;
 
@@ -142,7 +154,8 @@ int32_t glance_build_tree(glance_ctx *ctx, int32_t batch, const int32_t *root, c
  * seq_len + depth[i]; attends to all committed positions and to tree rows j with anc[i] bit j;
  * writes K/V of node i at cache row seq_len + i in every layer.
  * Outputs (device): argmax [batch][N] (ties to the lowest id, taken on fp32 accumulators);
- * hidden [batch][N][H] bf16 = residual stream after the last layer, before the final norm;
+ * hidden [head_layers][batch][N][H] bf16: slice i = residual stream after the target layer that head layer i
+ * taps (one slice, the stream after the last layer and before the final norm, for the one-layer head);
  * logits_dbg [batch][N][V] fp32 or NULL. */
 int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree,
                            int32_t *argmax, void *hidden, float *logits_dbg);
@@ -161,7 +174,7 @@ int32_t glance_verify_tree_sample(glance_ctx *ctx, const glance_seqs *seqs, cons
 
 /* Algorithm 1 lines 5-12 + commit.  Walks from the root along argmax while the token is a child
  * in the tree; then, per layer, moves cache row seq_len + path[d] to row seq_len + d (d = 1..a),
- * gathers hidden[path[0..a]] into feat, sets feat_count = a+1, seq_len += a+1, root = new root.
+ * gathers hidden[path[0..a]] into feat (every tap slice), sets feat_count = a+1, seq_len += a+1, root = new root.
  * Outputs (device): accept_len [batch] = a; path [batch][block_B] node indices (path[0] = 0);
  * out_tokens [batch][block_B]: the a accepted tokens followed by the new root. */
 int32_t glance_accept_commit(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree,

@@ -31,7 +31,8 @@ class GlanceError(RuntimeError):
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "hidden", "n_q_heads", "n_kv_heads", "head_dim", "ffn", "vocab")] + \
                [("rms_eps", C.c_float), ("rope_theta", C.c_float)] + \
-               [(n, C.c_int32) for n in ("block_B", "topk", "tree_N", "page_size", "max_batch", "max_pages_per_seq")]
+               [(n, C.c_int32) for n in ("block_B", "topk", "tree_N", "page_size", "max_batch", "max_pages_per_seq")] + \
+               [("head_layers", C.c_int32), ("head_taps", C.c_int32 * 8)]
 
 
 class TargetWeights(C.Structure):
@@ -39,8 +40,13 @@ class TargetWeights(C.Structure):
                [(n, C.POINTER(C.c_void_p)) for n in ("ln1", "wqkv", "wo", "ln2", "wgu", "wd")]
 
 
+class HeadLayer(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("ctx_norm", "ln1", "wqkv", "wo", "ln2", "wgu", "wd")]
+
+
 class HeadWeights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in ("mask_embed", "ctx_norm", "ln1", "wqkv", "wo", "ln2", "wgu", "wd", "final_norm")]
+    _fields_ = [(n, C.c_void_p) for n in ("mask_embed", "ctx_norm", "ln1", "wqkv", "wo", "ln2", "wgu", "wd", "final_norm")] + \
+               [("more", C.POINTER(HeadLayer))]
 
 
 class Seqs(C.Structure):
@@ -127,9 +133,10 @@ def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
 
 
 def make_config(cfg, max_batch: int, max_pages_per_seq: int) -> Config:
+    taps = tuple(getattr(cfg, "head_taps", ()) or ())
     return Config(cfg.n_layers, cfg.hidden, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn, cfg.vocab,
                   cfg.rms_eps, cfg.rope_theta, cfg.block_B, cfg.topk, cfg.tree_N, cfg.page_size, max_batch,
-                  max_pages_per_seq)
+                  max_pages_per_seq, len(taps), (C.c_int32 * 8)(*taps))
 
 
 def glance_topk_static(logits: torch.Tensor, k: int, topk_ids: torch.Tensor, topk_lp: torch.Tensor) -> int:
@@ -187,7 +194,13 @@ class Engine:
         self._arrs = {k: arr(k) for k in ("ln1", "wqkv", "wo", "ln2", "wgu", "wd")}
         self.tw = TargetWeights(_ptr(target["embed"]), _ptr(target["lm_head"]), _ptr(target["final_norm"]),
                                 *[C.cast(self._arrs[k], C.POINTER(C.c_void_p)) for k in ("ln1", "wqkv", "wo", "ln2", "wgu", "wd")])
-        self.hw = HeadWeights(*[_ptr(head[k]) for k in ("mask_embed", "ctx_norm", "ln1", "wqkv", "wo", "ln2", "wgu", "wd", "final_norm")])
+        more = head.get("more", [])
+        self._more = (HeadLayer * max(1, len(more)))(*[HeadLayer(*[_ptr(lw[k]) for k in ("ctx_norm", "ln1", "wqkv", "wo", "ln2", "wgu", "wd")])
+                                                        for lw in more])
+        self.hw = HeadWeights(*[_ptr(head[k]) for k in ("mask_embed", "ctx_norm", "ln1", "wqkv", "wo", "ln2", "wgu", "wd", "final_norm")],
+                              C.cast(self._more, C.POINTER(HeadLayer)) if more else None)
+        self.head_layers = 1 + len(more)
+        assert self.head_layers == max(1, len(getattr(cfg, "head_taps", ()) or ())), "one head weight set per tap"
         nbytes = self.lib.glance_workspace_bytes(C.byref(self.ccfg))
         if nbytes == 0:
             raise GlanceError("configuration not supported by the library")
@@ -197,16 +210,20 @@ class Engine:
         self.seq_len = torch.zeros(batch, **i32)
         self.root = torch.zeros(batch, **i32)
         self.feat_count = torch.zeros(batch, **i32)
-        self.feat = torch.zeros(batch, cfg.block_B, cfg.hidden, dtype=torch.bfloat16, device=dev)
+        T = self.head_layers
+        # one slice per head layer (= per tapped target layer); .feat / .hidden / .head_kv_pool are slice 0
+        self.feat_all = torch.zeros(T, batch, cfg.block_B, cfg.hidden, dtype=torch.bfloat16, device=dev)
+        self.feat = self.feat_all[0]
         # page tables: a fixed random permutation of the pool so that logical and physical order differ
         g = torch.Generator().manual_seed(1234)
         perm = torch.randperm(self.n_pages, generator=g).to(torch.int32)
         self.page_table = perm.reshape(batch, self.pages_per_seq).contiguous().to(dev)
         kv_shape = (cfg.n_layers, self.n_pages, 2, cfg.n_kv_heads, page, cfg.head_dim)
         self.kv_pool = torch.zeros(kv_shape, dtype=torch.bfloat16, device=dev)
-        self.head_kv_pool = torch.zeros(kv_shape[1:], dtype=torch.bfloat16, device=dev)
+        self.head_kv_all = torch.zeros((T,) + kv_shape[1:], dtype=torch.bfloat16, device=dev)
+        self.head_kv_pool = self.head_kv_all[0]
         self.seqs = Seqs(batch, self.n_pages, _ptr(self.seq_len), _ptr(self.root), _ptr(self.page_table),
-                         _ptr(self.kv_pool), _ptr(self.head_kv_pool), _ptr(self.feat), _ptr(self.feat_count))
+                         _ptr(self.kv_pool), _ptr(self.head_kv_all), _ptr(self.feat_all), _ptr(self.feat_count))
         ctx = C.c_void_p()
         sp = stream.cuda_stream if stream is not None else torch.cuda.current_stream(dev).cuda_stream
         self._stream_ptr = sp
@@ -219,7 +236,8 @@ class Engine:
         self.topk_lp = torch.zeros(batch, Lh, k, dtype=torch.float32, device=dev)
         self.tree = TreeBuffers(batch, N, dev)
         self.argmax = torch.zeros(batch, N, **i32)
-        self.hidden = torch.zeros(batch, N, cfg.hidden, dtype=torch.bfloat16, device=dev)
+        self.hidden_all = torch.zeros(T, batch, N, cfg.hidden, dtype=torch.bfloat16, device=dev)
+        self.hidden = self.hidden_all[0]
         self.accept_len = torch.zeros(batch, **i32)
         self.path = torch.zeros(batch, B, **i32)
         self.out_tokens = torch.zeros(batch, B, **i32)
@@ -258,25 +276,25 @@ class Engine:
     def glance_verify_tree(self, tree: Optional[TreeBuffers] = None, logits_dbg: Optional[torch.Tensor] = None):
         tree = tree or self.tree
         _check(self.lib.glance_verify_tree(self.ctx, C.byref(self.seqs), C.byref(tree.c), _ptr(self.argmax),
-                                           _ptr(self.hidden), _ptr(logits_dbg)), "glance_verify_tree")
+                                           _ptr(self.hidden_all), _ptr(logits_dbg)), "glance_verify_tree")
 
     def glance_verify_tree_sample(self, seed: int, temperature: float = 1.0, tree: Optional[TreeBuffers] = None,
                                   logits_dbg: Optional[torch.Tensor] = None):
         """Sampling mode: self.argmax receives one draw per row instead of the arg-max."""
         tree = tree or self.tree
         _check(self.lib.glance_verify_tree_sample(self.ctx, C.byref(self.seqs), C.byref(tree.c), C.c_uint64(seed),
-                                                  C.c_float(temperature), _ptr(self.argmax), _ptr(self.hidden),
+                                                  C.c_float(temperature), _ptr(self.argmax), _ptr(self.hidden_all),
                                                   _ptr(logits_dbg)), "glance_verify_tree_sample")
 
     def glance_accept_commit(self, tree: Optional[TreeBuffers] = None, argmax: Optional[torch.Tensor] = None):
         tree = tree or self.tree
         _check(self.lib.glance_accept_commit(self.ctx, C.byref(self.seqs), C.byref(tree.c),
-                                             _ptr(self.argmax if argmax is None else argmax), _ptr(self.hidden),
+                                             _ptr(self.argmax if argmax is None else argmax), _ptr(self.hidden_all),
                                              _ptr(self.accept_len), _ptr(self.path), _ptr(self.out_tokens)),
                "glance_accept_commit")
 
     def glance_commit_forced(self, path: torch.Tensor, path_len: torch.Tensor, new_root: torch.Tensor):
-        _check(self.lib.glance_commit_forced(self.ctx, C.byref(self.seqs), _ptr(self.hidden), _ptr(path), _ptr(path_len),
+        _check(self.lib.glance_commit_forced(self.ctx, C.byref(self.seqs), _ptr(self.hidden_all), _ptr(path), _ptr(path_len),
                                              _ptr(new_root)), "glance_commit_forced")
 
     def glance_poll_status(self) -> int:
@@ -344,17 +362,17 @@ class Engine:
         return g
 
     def snapshot_state(self):
-        return (self.seq_len.clone(), self.root.clone(), self.feat.clone(), self.feat_count.clone())
+        return (self.seq_len.clone(), self.root.clone(), self.feat_all.clone(), self.feat_count.clone())
 
     def restore_state(self, snap):
-        self.seq_len.copy_(snap[0]); self.root.copy_(snap[1]); self.feat.copy_(snap[2]); self.feat_count.copy_(snap[3])
+        self.seq_len.copy_(snap[0]); self.root.copy_(snap[1]); self.feat_all.copy_(snap[2]); self.feat_count.copy_(snap[3])
 
     def gather_kv(self, seq: int, layer: int, length: int):
         """Logical K,V rows [length, Hkv, d] of one sequence and layer, read back through the page table (tests)."""
         return _gather(self.kv_pool[layer], self.page_table[seq], length, self.cfg.page_size)
 
-    def gather_head_kv(self, seq: int, length: int):
-        return _gather(self.head_kv_pool, self.page_table[seq], length, self.cfg.page_size)
+    def gather_head_kv(self, seq: int, length: int, head_layer: int = 0):
+        return _gather(self.head_kv_all[head_layer], self.page_table[seq], length, self.cfg.page_size)
 
 
 def _gather(pool_layer: torch.Tensor, page_table: torch.Tensor, length: int, page: int):

@@ -42,7 +42,7 @@ struct Workspace {
     float *rope_cos, *rope_sin;
     double *inv_freq;      // [d/2]
     uint64_t *chain_anc;   // [N][W] prefill chain mask
-    bf16 *hidden_tmp;      // [N][H] prefill hidden
+    bf16 *hidden_tmp;      // [head layers][N][H] prefill: tapped hidden states of the chunk
     int32_t *argmax_tmp;   // [N]
     int32_t *status;
     unsigned long long *am_keys;   // [Rlog] packed arg-max keys, zero between launches
@@ -93,7 +93,7 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.rope_sin = (float *)take(R * (c.head_dim / 2) * 4);
     w.inv_freq = (double *)take((size_t)(c.head_dim / 2) * 8);
     w.chain_anc = (uint64_t *)take((size_t)c.tree_N * d.W * 8);
-    w.hidden_tmp = (bf16 *)take((size_t)c.tree_N * H * 2);
+    w.hidden_tmp = (bf16 *)take((size_t)(c.head_layers > 1 ? c.head_layers : 1) * c.tree_N * H * 2);
     w.argmax_tmp = (int32_t *)take((size_t)c.tree_N * 4);
     w.status = (int32_t *)take(256);
     w.am_keys = (unsigned long long *)take((size_t)d.Rlog * 8);
@@ -115,8 +115,18 @@ bool config_ok(const glance_config *c) {
     if (c->tree_N < 1 || c->tree_N > kMaxTreeN) return false;
     if (c->page_size != kPage || c->max_batch < 1 || c->max_batch > 64 || c->max_pages_per_seq < 1) return false;
     if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
+    if (c->head_layers < 0 || c->head_layers > GLANCE_MAX_HEAD_LAYERS) return false;
+    for (int i = 0; i < c->head_layers && c->head_layers > 1; ++i) {
+        if (c->head_taps[i] < 0 || c->head_taps[i] >= c->n_layers) return false;
+        for (int j = 0; j < i; ++j)
+            if (c->head_taps[j] == c->head_taps[i]) return false;
+    }
     return true;
 }
+
+// head depth and the target layer each head layer taps
+int head_depth(const glance_config &c) { return c.head_layers > 1 ? c.head_layers : 1; }
+int head_tap(const glance_config &c, int i) { return c.head_layers > 1 ? c.head_taps[i] : c.n_layers - 1; }
 
 }  // namespace
 
@@ -131,6 +141,7 @@ struct glance_ctx {
     const bf16 *embed, *lm_head, *final_norm;
     std::vector<const bf16 *> ln1, wqkv, wo, ln2, wgu, wd;
     glance_head_weights head;
+    std::vector<glance_head_layer> head_layer;   // all head layers, layer 0 first
     int64_t launches;
     // optional per-launch timing (event pairs created when profiling is first enabled)
     bool profiling = false;
@@ -332,6 +343,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
 }
 
 // all target layers (+ LM head with fused arg-max) over rows prepared by a setup kernel
+// `hidden_out` [head layers][ps.R][H]: slice i receives the residual stream after the target layer head layer i taps
 void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *logits, int32_t *argmax) {
     const glance_config &c = ctx->cfg;
     const KvGeom geom = geom_of(ctx, ps.seqs);
@@ -339,7 +351,10 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
         LayerW w{ctx->ln2[l], ctx->wqkv[l], ctx->wo[l], ctx->wgu[l], ctx->wd[l]};
         const bool last = (l + 1 == c.n_layers);
         bf16 *pool_layer = (bf16 *)ps.seqs->kv_pool + (size_t)l * geom.layer_stride();
-        run_layer(ctx, w, pool_layer, ps, last ? ctx->final_norm : ctx->ln1[l + 1], last ? hidden_out : nullptr);
+        bf16 *tap_out = nullptr;
+        for (int i = 0; i < head_depth(c) && hidden_out; ++i)
+            if (head_tap(c, i) == l) tap_out = hidden_out + (size_t)i * ps.R * c.hidden;
+        run_layer(ctx, w, pool_layer, ps, last ? ctx->final_norm : ctx->ln1[l + 1], tap_out);
     }
     if (argmax) {   // logits are stored only on request
         TcGemmArgs g{};
@@ -432,6 +447,15 @@ int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, 
         ctx->wd.push_back((const bf16 *)t->wd[l]);
     }
     ctx->head = *h;
+    ctx->head_layer.push_back(glance_head_layer{h->ctx_norm, h->ln1, h->wqkv, h->wo, h->ln2, h->wgu, h->wd});
+    for (int i = 1; i < head_depth(*cfg); ++i) {
+        const glance_head_layer *m = h->more ? &h->more[i - 1] : nullptr;
+        if (!m || !m->ctx_norm || !m->ln1 || !m->wqkv || !m->wo || !m->ln2 || !m->wgu || !m->wd) {
+            delete ctx;
+            return GLANCE_E_INVALID_ARG;
+        }
+        ctx->head_layer.push_back(*m);
+    }
     ctx->launches = 0;
     // rotary frequencies theta^(-2i/d) in double, uploaded once
     ctx->inv_freq_host.resize(cfg->head_dim / 2);
@@ -487,19 +511,24 @@ int32_t glance_prefill(glance_ctx *ctx, const glance_seqs *seqs, int32_t seq, co
         LAUNCH(ctx, KIND_SETUP, launch_setup_verify(vs, st));
         PassInfo ps{N, N, 1, N, ws.chain_anc, seqs, seq};
         run_target(ctx, ps, ws.hidden_tmp, nullptr, last ? ws.argmax_tmp : nullptr);
-        // head context K/V of the new positions (Section 3.2: keys and values are the target's hidden states)
-        DraftSetup ds{};
-        ds.batch = 1; ds.B = c.block_B; ds.FR = N; ds.d = c.head_dim; ds.theta = c.rope_theta;
-        ds.seq_len = seqs->seq_len + seq; ds.root = seqs->root + seq; ds.feat = ws.hidden_tmp; ds.feat_count = nullptr;
-        ds.count_const = n; ds.n_block = 0; ds.embed = ctx->embed; ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
-        ds.gain_block = (const bf16 *)ctx->head.ln1; ds.gain_feat = (const bf16 *)ctx->head.ctx_norm;
-        ds.vocab = c.vocab; ds.capacity = c.max_pages_per_seq * kPage; ds.geom = tg; ds.page_table = pt;
-        ds.out = rowout_of(ctx); ds.meta = meta_of(ctx); ds.status = ws.status;
-        LAUNCH(ctx, KIND_SETUP, launch_setup_draft(ds, st));
-        LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
-                  (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
-        PassInfo hp{N, 0, 1, N, nullptr, seqs, seq};
-        run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, hp, nullptr, nullptr);
+        // head context K/V of the new positions (Section 3.2: keys and values are the target's hidden states): every
+        // head layer projects the hidden states of the target layer it taps with its own weights into its own pool
+        for (int i = 0; i < head_depth(c); ++i) {
+            const glance_head_layer &hl = ctx->head_layer[i];
+            DraftSetup ds{};
+            ds.batch = 1; ds.B = c.block_B; ds.FR = N; ds.d = c.head_dim; ds.theta = c.rope_theta;
+            ds.seq_len = seqs->seq_len + seq; ds.root = seqs->root + seq;
+            ds.feat = ws.hidden_tmp + (size_t)i * N * c.hidden; ds.feat_count = nullptr;
+            ds.count_const = n; ds.n_block = 0; ds.embed = ctx->embed; ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
+            ds.gain_block = (const bf16 *)hl.ln1; ds.gain_feat = (const bf16 *)hl.ctx_norm;
+            ds.vocab = c.vocab; ds.capacity = c.max_pages_per_seq * kPage; ds.geom = tg; ds.page_table = pt;
+            ds.out = rowout_of(ctx); ds.meta = meta_of(ctx); ds.status = ws.status;
+            LAUNCH(ctx, KIND_SETUP, launch_setup_draft(ds, st));
+            LayerW hw{(const bf16 *)hl.ln2, (const bf16 *)hl.wqkv, (const bf16 *)hl.wo, (const bf16 *)hl.wgu,
+                      (const bf16 *)hl.wd};
+            PassInfo hp{N, 0, 1, N, nullptr, seqs, seq};
+            run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool + (size_t)i * tg.layer_stride(), hp, nullptr, nullptr);
+        }
         LAUNCH(ctx, KIND_CONTROL, launch_prefill_advance(seqs->seq_len + seq, seqs->root + seq, seqs->feat_count + seq,
                                                          last ? ws.argmax_tmp : nullptr, n, st));
     }
@@ -525,20 +554,28 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
     cudaStream_t st = ctx->stream;
     const int batch = seqs->batch, B = c.block_B;
     const int R1 = batch * B, R = 2 * R1;
-    DraftSetup ds{};
-    ds.batch = batch; ds.B = B; ds.FR = B; ds.d = c.head_dim; ds.theta = c.rope_theta;
-    ds.seq_len = seqs->seq_len; ds.root = seqs->root; ds.feat = (const bf16 *)seqs->feat;
-    ds.feat_count = seqs->feat_count; ds.count_const = 0; ds.n_block = B; ds.embed = ctx->embed;
-    ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
-    // block rows use the head's input norm, feature rows the context norm
-    ds.gain_block = (const bf16 *)ctx->head.ln1; ds.gain_feat = (const bf16 *)ctx->head.ctx_norm; ds.vocab = c.vocab;
-    ds.capacity = c.max_pages_per_seq * kPage; ds.geom = geom_of(ctx, seqs); ds.page_table = seqs->page_table;
-    ds.out = rowout_of(ctx); ds.meta = meta_of(ctx); ds.status = ws.status;
-    LAUNCH(ctx, KIND_SETUP, launch_setup_draft(ds, st));
-    LayerW hw{(const bf16 *)ctx->head.ln2, (const bf16 *)ctx->head.wqkv, (const bf16 *)ctx->head.wo,
-              (const bf16 *)ctx->head.wgu, (const bf16 *)ctx->head.wd};
-    PassInfo ps{R, R1, batch, B, nullptr, seqs, 0};
-    run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool, ps, (const bf16 *)ctx->head.final_norm, nullptr);
+    const KvGeom hgeom = geom_of(ctx, seqs);
+    const int HL = head_depth(c);
+    for (int i = 0; i < HL; ++i) {
+        // head layer i: block rows (from the embeddings, or from the layer below) and the feature rows of the
+        // positions committed last, taken from the target layer this head layer taps
+        const glance_head_layer &hl = ctx->head_layer[i];
+        DraftSetup ds{};
+        ds.batch = batch; ds.B = B; ds.FR = B; ds.d = c.head_dim; ds.theta = c.rope_theta;
+        ds.seq_len = seqs->seq_len; ds.root = seqs->root;
+        ds.feat = (const bf16 *)seqs->feat + (size_t)i * batch * B * c.hidden;
+        ds.feat_count = seqs->feat_count; ds.count_const = 0; ds.n_block = B; ds.features_only = i > 0 ? 1 : 0;
+        ds.embed = ctx->embed; ds.mask_embed = (const bf16 *)ctx->head.mask_embed;
+        // block rows use the head layer's input norm, feature rows its context norm
+        ds.gain_block = (const bf16 *)hl.ln1; ds.gain_feat = (const bf16 *)hl.ctx_norm; ds.vocab = c.vocab;
+        ds.capacity = c.max_pages_per_seq * kPage; ds.geom = hgeom; ds.page_table = seqs->page_table;
+        ds.out = rowout_of(ctx); ds.meta = meta_of(ctx); ds.status = ws.status;
+        LAUNCH(ctx, KIND_SETUP, launch_setup_draft(ds, st));
+        LayerW hw{(const bf16 *)hl.ln2, (const bf16 *)hl.wqkv, (const bf16 *)hl.wo, (const bf16 *)hl.wgu, (const bf16 *)hl.wd};
+        PassInfo ps{R, R1, batch, B, nullptr, seqs, 0};
+        const bf16 *next_gain = i + 1 < HL ? (const bf16 *)ctx->head_layer[i + 1].ln1 : (const bf16 *)ctx->head.final_norm;
+        run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool + (size_t)i * hgeom.layer_stride(), ps, next_gain, nullptr);
+    }
     float *logits = logits_dbg ? logits_dbg : ws.logits;
     {
         TcGemmArgs g{};
@@ -611,6 +648,7 @@ static int32_t commit_common(glance_ctx *ctx, const glance_seqs *seqs, WalkCommi
     wc.hidden = (const bf16 *)hidden; wc.kv_pool = (bf16 *)seqs->kv_pool; wc.geom = geom_of(ctx, seqs);
     wc.page_table = seqs->page_table; wc.seq_len = seqs->seq_len; wc.root = seqs->root;
     wc.feat_count = seqs->feat_count; wc.feat = (bf16 *)seqs->feat; wc.counters = ctx->ws.walk_ctr;
+    wc.n_taps = head_depth(c);
     wc.status = ctx->ws.status;
     LAUNCH(ctx, KIND_CONTROL, launch_walk_commit(wc, ctx->stream));
     return finish(ctx);

@@ -49,6 +49,7 @@ struct DraftSetup {
     const int32_t *feat_count;  // [batch] or nullptr (then count_const rows, appended at seq_len)
     int count_const;
     int n_block;                // B (round) or 0 (prefill: only feature rows)
+    int features_only;          // 1: leave the block rows alone (head layers 1..: their inputs come from the layer below)
     const bf16 *embed, *mask_embed;
     const bf16 *gain_block, *gain_feat;   // head input norm / context norm
     int vocab;
@@ -76,12 +77,13 @@ struct WalkCommit {
     const int32_t *token, *parent, *n_nodes;   // tree (walk mode) or nullptr
     const int32_t *argmax;                      // [batch][N] (walk mode)
     const int32_t *forced_path, *forced_len, *forced_root;   // forced mode (argmax == nullptr)
-    const bf16 *hidden;                         // [batch][N][H]
+    const bf16 *hidden;                         // [n_taps][batch][N][H]
+    int n_taps;                                 // head layers = tapped target layers
     bf16 *kv_pool;
     KvGeom geom;
     const int32_t *page_table;
     int32_t *seq_len, *root, *feat_count;
-    bf16 *feat;                                 // [batch][B][H]
+    bf16 *feat;                                 // [n_taps][batch][B][H]
     int32_t *accept_len, *path, *out_tokens;    // outputs (may be nullptr in forced mode)
     int32_t *counters;                          // [batch], zero between calls
     int32_t *status;

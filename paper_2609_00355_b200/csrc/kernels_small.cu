@@ -143,8 +143,8 @@ void launch_setup_verify(const VerifySetup &p, cudaStream_t st) {
 // embedding, position P + j.  Feature rows: target features of the positions committed last, whose K/V
 // become head context at positions P - count .. P - 1 (or P .. P+count-1 while prefilling).
 __global__ void __launch_bounds__(128) setup_draft_kernel(DraftSetup p) {
-    const int r = blockIdx.x;
     const int R1 = p.batch * p.n_block;
+    const int r = blockIdx.x + (p.features_only ? R1 : 0);
     const bf16 *src = nullptr;
     int s, pos, slot;
     if (r < R1) {
@@ -189,7 +189,7 @@ __global__ void __launch_bounds__(128) setup_draft_kernel(DraftSetup p) {
 }
 
 void launch_setup_draft(const DraftSetup &p, cudaStream_t st) {
-    const int R = p.batch * p.n_block + p.batch * p.FR;
+    const int R = (p.features_only ? 0 : p.batch * p.n_block) + p.batch * p.FR;
     setup_draft_kernel<<<R, 128, 0, st>>>(p);
 }
 

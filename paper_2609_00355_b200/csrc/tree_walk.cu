@@ -253,10 +253,14 @@ __global__ void __launch_bounds__(256) walk_commit_kernel(WalkCommit p) {
     if (threadIdx.x == 0) sh_last = (atomicAdd(&p.counters[s], 1) == (int)gridDim.y - 1);
     __syncthreads();
     if (!sh_last) return;
-    for (int i = 0; i <= a; ++i) {
-        const bf16 *src = p.hidden + ((size_t)s * p.N + sh_path[i]) * p.H;
-        bf16 *dst = p.feat + ((size_t)s * p.B + i) * p.H;
-        for (int c = threadIdx.x; c < p.H; c += blockDim.x) dst[c] = src[c];
+    for (int tap = 0; tap < p.n_taps; ++tap) {
+        const bf16 *hid = p.hidden + (size_t)tap * p.batch * p.N * p.H;
+        bf16 *ft = p.feat + (size_t)tap * p.batch * p.B * p.H;
+        for (int i = 0; i <= a; ++i) {
+            const bf16 *src = hid + ((size_t)s * p.N + sh_path[i]) * p.H;
+            bf16 *dst = ft + ((size_t)s * p.B + i) * p.H;
+            for (int c = threadIdx.x; c < p.H; c += blockDim.x) dst[c] = src[c];
+        }
     }
     if (threadIdx.x == 0) {
         if (p.accept_len) p.accept_len[s] = a;

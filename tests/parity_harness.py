@@ -106,9 +106,10 @@ class ParityRun:
         for s, st in enumerate(self.states):
             n = st.P - int(self.eng.feat_count[s])
             if n > 0:
-                K, V = self.eng.gather_head_kv(s, n)
-                close(K, st.hK[:n], f"head K seq {s}")
-                close(V, st.hV[:n], f"head V seq {s}")
+                for i in range(self.eng.head_layers):
+                    K, V = self.eng.gather_head_kv(s, n, i)
+                    close(K, (st.hK if i == 0 else st.hK_more[i - 1])[:n], f"head layer {i} K seq {s}")
+                    close(V, (st.hV if i == 0 else st.hV_more[i - 1])[:n], f"head layer {i} V seq {s}")
 
     # ---- oracle look-ahead: the greedy continuation after the pending root -------------------
     def oracle_continuation(self, s: int, n: int, sample_seed=None):
@@ -188,7 +189,8 @@ class ParityRun:
             n = trees[s].n_nodes
             scale = float(ol[:n].abs().max())
             self.stats["max_rel_logit"] = max(self.stats["max_rel_logit"], close(vlog[s, :n], ol[:n], "verify logits", scale))
-            close(eng.hidden[s, :n], oh[:n], "verify hidden")
+            for i, oh_i in enumerate([oh] if oh.dim() == 2 else list(oh)):       # one slice per tapped layer
+                close(eng.hidden_all[i, s, :n], oh_i[:n], f"verify hidden, tap {i}")
             if sample_seed is None:
                 oam = O.argmax_lowest(ol)
                 top2 = torch.topk(ol, 2, dim=-1).values
@@ -231,7 +233,8 @@ class ParityRun:
             assert out_g[s, a] == new_root and int(eng.root[s]) == new_root
             assert int(eng.seq_len[s]) == st.P + a + 1 and int(eng.feat_count[s]) == a + 1
             self._check_compaction(s, st.P, path, pool_verified)
-            assert torch.equal(eng.feat[s, :a + 1], eng.hidden[s, torch.tensor(path, device=dev)])
+            for i in range(eng.head_layers):
+                assert torch.equal(eng.feat_all[i, s, :a + 1], eng.hidden_all[i, s, torch.tensor(path, device=dev)])
             oa, opath, oout, oroot = O.walk(trees[s], infos[s][2])
             if (a, path, new_root) != (oa, opath, oroot):
                 need_force = True

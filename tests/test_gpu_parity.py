@@ -405,3 +405,30 @@ def test_rounds_small_sampling_mode(harness):
         run.round(p_m=0.6, check_draft=False, sample_seed=2024)
     print("sampling parity stats (small):", run.stats)
     assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_two_layer_head_two_taps(harness):
+    """Multi-layer block head (Section 3.2): two head layers, the first fed by target layer 0 and the second by
+    target layer 1.  Draft logits, tapped hidden states, per-layer head context K/V and the rounds against the
+    oracle."""
+    cfg = synth.CONFIGS["tiny"].replace(head_taps=(0, 1))
+    run = harness.ParityRun(cfg)
+    run.check_state()
+    run.check_head_state()
+    for r in range(6):
+        run.round(p_m=(0.7 if r % 2 else None), check_draft=True)
+    run.check_head_state()
+    print("two-layer head parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_small_three_layer_head(harness):
+    """Three head layers tapping target layers 1, 4 and 7 of the 8-layer small configuration."""
+    cfg = synth.CONFIGS["small"].replace(head_taps=(1, 4, 7))
+    run = harness.ParityRun(cfg)
+    run.check_head_state()
+    for r in range(4):
+        run.round(p_m=0.6, check_draft=(r < 2))
+    run.check_head_state()
+    print("three-layer head parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
