@@ -700,6 +700,15 @@ def spec_round_sampled(sh: Shape, tw: dict, hw: dict, st: SeqState, B: int, k: i
 # acceptance statistics (Eq. 1, Eq. 2)
 # ----------------------------------------------------------------------------------------------
 
+def root_entropy(logits_row: torch.Tensor) -> float:
+    """Section 4: the target's next-token entropy at the round root, H = -sum_v p_v log p_v in nats, p = softmax of
+    the root row's logits; computed as lse - sum_v p_v * logit_v in float64."""
+    x = logits_row.double()
+    lse = torch.logsumexp(x, dim=-1)
+    p = torch.exp(x - lse)
+    return float(lse - (p * x).sum())
+
+
 def expected_accept(p_m: float, L: int) -> float:
     """Eq. 2: E[a | p_m] = sum_{l=1..L} p_m^l."""
     return float(sum(p_m ** l for l in range(1, L + 1)))

@@ -653,6 +653,24 @@ def test_sampled_rounds_equal_plain_ancestral_sampling(tiny):
     assert sum(accepted) > 0
 
 
+def test_root_entropy_closed_forms():
+    """Entropy of the root row (Section 4) against closed forms: uniform, two-level and shifted distributions."""
+    V = 1000
+    assert abs(O.root_entropy(torch.zeros(V)) - math.log(V)) < 1e-9
+    assert abs(O.root_entropy(torch.full((V,), 3.7)) - math.log(V)) < 1e-9          # a constant shift changes nothing
+    # one token with probability q, the rest uniform: H = -q log q - (1-q) log((1-q)/(V-1))
+    for q in (0.5, 0.9, 0.999):
+        x = torch.zeros(V, dtype=torch.float64)
+        x[17] = math.log(q / ((1 - q) / (V - 1)))
+        ref = -q * math.log(q) - (1 - q) * math.log((1 - q) / (V - 1))
+        assert abs(O.root_entropy(x) - ref) < 1e-9
+    # a dominant logit: H -> 0; and H never exceeds log V
+    x = torch.randn(V, generator=torch.Generator().manual_seed(1))
+    assert 0.0 < O.root_entropy(x) < math.log(V)
+    x[3] = 80.0
+    assert O.root_entropy(x) < 1e-20 + 1e-12
+
+
 def test_controlled_match_acceptance_statistics(tiny):
     """Measured mean accepted length under controlled per-depth match probability sits on Eq. 2."""
     rng = np.random.default_rng(21)
