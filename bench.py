@@ -137,6 +137,9 @@ class RoundBench:
         self.eng = Engine(cfg, self.tw, self.hw, batch=cfg.batch, stream=self.stream)
         self.graph = None
         eng = self.eng
+        # round log for the entropy law: every verify pass leaves the root entropy of each sequence here
+        self.root_entropy = torch.zeros(cfg.batch, dtype=torch.float32, device=device)
+        eng.glance_log_root_entropy(self.root_entropy)
         lens = [cfg.ctx] * cfg.batch
         if cfg.batch > 1:
             lens = synth.batch_context_lengths(cfg)
@@ -408,6 +411,7 @@ def main():
 
     # ---- device-resident arm -------------------------------------------------------------------
     round_ms, wall_ms, committed = [], [], 0
+    ent_log = []
     sampler = ClockSampler(local_rank)
     for step in range(warmup + args.steps):
         Y = bench.lookahead()
@@ -430,6 +434,7 @@ def main():
             round_ms.append(start.elapsed_time(stop))
             wall_ms.append(1e3 * (w1 - w0))
             committed += int(eng.accept_len.sum().item()) + cfg.batch
+            ent_log.append(float(bench.root_entropy.mean().item()))
     barrier()
     eng.check_device_status()
     # ---- per-kernel pass: the same rounds again with every launch bracketed by CUDA events (the events add
@@ -493,6 +498,8 @@ def main():
         "round_us": {"mean": 1e3 * ms_per_step, "median": 1e3 * statistics.median(round_ms),
                      "host_wall_mean": 1e3 * sum(wall_ms) / len(wall_ms)},
         "tau": committed / (args.steps * cfg.batch * world), "tau_expected": expected_tau,
+        "root_entropy_nats": {"mean": sum(ent_log) / max(len(ent_log), 1), "log_vocab": math.log(cfg.vocab),
+                              "note": "logged by the verify pass of every timed round (random-init target: near log V)"},
         "round_hbm": {"algorithmic_gb": round_bytes / 1e9, "achieved_gbs": round_bytes / (ms_per_step * 1e-3) / 1e9,
                       "frac_of_measured_peak": round_bytes / (ms_per_step * 1e-3) / 1e9 / peak},
         "roofline": {"bound": "hbm", "kernel": "weight-streaming GEMM (all projections, MLP, LM head)",

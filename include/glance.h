@@ -172,6 +172,12 @@ int32_t glance_verify_tree(glance_ctx *ctx, const glance_seqs *seqs, const glanc
 int32_t glance_verify_tree_sample(glance_ctx *ctx, const glance_seqs *seqs, const glance_tree *tree, uint64_t seed,
                                   float temperature, int32_t *draws, void *hidden, float *logits_dbg);
 
+/* Round log for the entropy law (Section 4: the target's next-token entropy H at the round root).  While
+ * `entropy` (device, [max_batch] floats) is set, every verify pass -- greedy or sampling -- also writes, for each
+ * sequence s, H[s] = -sum_v p_v log p_v in nats with p = softmax of the root row's logits (node 0, temperature 1,
+ * no noise), computed from per-tile statistics inside the LM-head epilogue.  NULL switches it off.  Host call. */
+int32_t glance_log_root_entropy(glance_ctx *ctx, float *entropy);
+
 /* Algorithm 1 lines 5-12 + commit.  Walks from the root along argmax while the token is a child
  * in the tree; then, per layer, moves cache row seq_len + path[d] to row seq_len + d (d = 1..a),
  * gathers hidden[path[0..a]] into feat (every tap slice), sets feat_count = a+1, seq_len += a+1, root = new root.

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libglance.so")
 EXPORTS = [
     "glance_status_string", "glance_workspace_bytes", "glance_create", "glance_destroy", "glance_prefill",
     "glance_seq_truncate", "glance_draft_block", "glance_build_tree", "glance_verify_tree",
-    "glance_verify_tree_sample",
+    "glance_verify_tree_sample", "glance_log_root_entropy",
     "glance_accept_commit", "glance_commit_forced", "glance_poll_status", "glance_launch_count",
     "glance_debug_attention", "glance_debug_gemm", "glance_profile_enable", "glance_profile_read",
     "glance_topk_static", "glance_debug_trace",
@@ -89,6 +89,8 @@ def load_library() -> C.CDLL:
     lib.glance_build_tree.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(Tree)]
     lib.glance_verify_tree.restype = C.c_int32
     lib.glance_verify_tree.argtypes = [C.c_void_p, C.POINTER(Seqs), C.POINTER(Tree), C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.glance_log_root_entropy.restype = C.c_int32
+    lib.glance_log_root_entropy.argtypes = [C.c_void_p, C.c_void_p]
     lib.glance_verify_tree_sample.restype = C.c_int32
     lib.glance_verify_tree_sample.argtypes = [C.c_void_p, C.POINTER(Seqs), C.POINTER(Tree), C.c_uint64, C.c_float, C.c_void_p,
                                               C.c_void_p, C.c_void_p]
@@ -285,6 +287,11 @@ class Engine:
         _check(self.lib.glance_verify_tree_sample(self.ctx, C.byref(self.seqs), C.byref(tree.c), C.c_uint64(seed),
                                                   C.c_float(temperature), _ptr(self.argmax), _ptr(self.hidden_all),
                                                   _ptr(logits_dbg)), "glance_verify_tree_sample")
+
+    def glance_log_root_entropy(self, entropy: Optional[torch.Tensor]):
+        """entropy: float32 CUDA tensor [batch] that every later verify pass fills, or None to stop logging."""
+        self._entropy_keep = entropy
+        _check(self.lib.glance_log_root_entropy(self.ctx, _ptr(entropy)), "glance_log_root_entropy")
 
     def glance_accept_commit(self, tree: Optional[TreeBuffers] = None, argmax: Optional[torch.Tensor] = None):
         tree = tree or self.tree

@@ -341,6 +341,26 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                     }
                 }
                 if (MODE == 2) {
+                    if (a.ent_out && rr % a.ent_N == 0) {
+                        // root row of a sequence: this tile's share of the soft-max statistics behind the entropy
+                        float m = -INFINITY;
+                        if (f < a.Nout) m = v.x;
+                        if (f + 1 < a.Nout) m = fmaxf(m, v.y);
+                        if (f + 2 < a.Nout) m = fmaxf(m, v.z);
+                        if (f + 3 < a.Nout) m = fmaxf(m, v.w);
+                        m = warp_max(m);
+                        float l = 0.f, t = 0.f, e;
+                        if (f < a.Nout) { e = __expf(v.x - m); l += e; t += e * v.x; }
+                        if (f + 1 < a.Nout) { e = __expf(v.y - m); l += e; t += e * v.y; }
+                        if (f + 2 < a.Nout) { e = __expf(v.z - m); l += e; t += e * v.z; }
+                        if (f + 3 < a.Nout) { e = __expf(v.w - m); l += e; t += e * v.w; }
+                        l = warp_sum(l);
+                        t = warp_sum(t);
+                        if (lane == 0) {
+                            float *dst = a.ent_part + ((size_t)tile_idx * a.ent_batch + rr / a.ent_N) * 3;
+                            dst[0] = m; dst[1] = l; dst[2] = t;
+                        }
+                    }
                     if (a.sample_pos) {
                         // sampling mode: a draw from softmax(row * inv_temperature) is the arg-max of the row plus
                         // Gumbel noise; the noise of (token position, vocabulary id) is a fixed field, so the draw
@@ -491,6 +511,48 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                 a.keys[r] = 0ull;
             }
             if (threadIdx.x == 0) *a.counter = 0;
+            if (a.ent_out) {
+                // entropy of every root row from the per-tile statistics: H = (M + log L) - T / L, merged in a fixed order
+                __shared__ float red_m[NTHR / 32], red_l[NTHR / 32], red_t[NTHR / 32];
+                const int tiles = (a.Nout + BM - 1) / BM;
+                const int wid = threadIdx.x >> 5, ln = threadIdx.x & 31;
+                for (int sq = 0; sq < a.ent_batch && sq * a.ent_N < a.R; ++sq) {
+                    float M = -INFINITY, L = 0.f, T = 0.f;
+                    for (int tl = threadIdx.x; tl < tiles; tl += blockDim.x) {
+                        const float *src = a.ent_part + ((size_t)tl * a.ent_batch + sq) * 3;
+                        const float m = __ldcg(src), l = __ldcg(src + 1), t = __ldcg(src + 2);
+                        const float nm = fmaxf(M, m);
+                        const float c0 = (M == -INFINITY) ? 0.f : __expf(M - nm), c1 = __expf(m - nm);
+                        L = L * c0 + l * c1;
+                        T = T * c0 + t * c1;
+                        M = nm;
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        const float m = __shfl_xor_sync(0xffffffffu, M, o), l = __shfl_xor_sync(0xffffffffu, L, o);
+                        const float t = __shfl_xor_sync(0xffffffffu, T, o);
+                        const float nm = fmaxf(M, m);
+                        const float c0 = (M == -INFINITY) ? 0.f : __expf(M - nm), c1 = (m == -INFINITY) ? 0.f : __expf(m - nm);
+                        L = L * c0 + l * c1;
+                        T = T * c0 + t * c1;
+                        M = nm;
+                    }
+                    if (ln == 0) { red_m[wid] = M; red_l[wid] = L; red_t[wid] = T; }
+                    __syncthreads();
+                    if (threadIdx.x == 0) {
+                        float gm = -INFINITY;
+                        for (int w = 0; w < NTHR / 32; ++w) gm = fmaxf(gm, red_m[w]);
+                        float gl = 0.f, gt = 0.f;
+                        for (int w = 0; w < NTHR / 32; ++w) {
+                            const float c = (red_m[w] == -INFINITY) ? 0.f : __expf(red_m[w] - gm);
+                            gl += red_l[w] * c;
+                            gt += red_t[w] * c;
+                        }
+                        a.ent_out[sq] = (gm + logf(gl)) - gt / gl;
+                    }
+                    __syncthreads();
+                }
+            }
         }
     }
 }

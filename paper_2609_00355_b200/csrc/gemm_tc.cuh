@@ -26,6 +26,11 @@ struct TcGemmArgs {
     const int32_t *sample_pos;
     unsigned long long sample_seed;
     float sample_inv_t;
+    // mode 2, root-entropy log: rows r with r % ent_N == 0 are round roots; every tile leaves (max, sum exp, sum exp *
+    // logit) of its 128 features in ent_part [tiles][ent_batch][3] and the last CTA writes the entropy (nats) of
+    // sequence r / ent_N to ent_out; ent_out == nullptr: off
+    float *ent_part, *ent_out;
+    int ent_N, ent_batch;
     // row scales (modes 0, 1, 2, 4): row r is multiplied by rsqrt(sum_i ssq[i*ssq_stride + r] / K + eps); nullptr = 1
     const float *ssq;
     int n_ssq, ssq_stride;

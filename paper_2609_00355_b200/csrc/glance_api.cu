@@ -47,6 +47,7 @@ struct Workspace {
     int32_t *status;
     unsigned long long *am_keys;   // [Rlog] packed arg-max keys, zero between launches
     int32_t *am_counter;
+    float *ent_part;       // [vocab tiles][max_batch][3] soft-max statistics of the root rows (entropy log)
     unsigned long long *topk_cand; // [batch*L][warps][k]
     float *topk_ml;                // [batch*L][warps][2]
     size_t total;
@@ -98,6 +99,7 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.status = (int32_t *)take(256);
     w.am_keys = (unsigned long long *)take((size_t)d.Rlog * 8);
     w.am_counter = (int32_t *)take(256);
+    w.ent_part = (float *)take((size_t)((c.vocab + 127) / 128) * c.max_batch * 3 * 4);
     const size_t trows = (size_t)c.max_batch * (c.block_B - 1) * topk_warps(c.vocab);
     w.topk_cand = (unsigned long long *)take(trows * c.topk * 8);
     w.topk_ml = (float *)take(trows * 2 * 4);
@@ -131,6 +133,8 @@ int head_tap(const glance_config &c, int i) { return c.head_layers > 1 ? c.head_
 }  // namespace
 
 struct glance_ctx {
+    float *ent_out = nullptr;               // device [max_batch]: root entropy written by every verify pass, or off
+    bool ent_on = false;                    // the pass in flight is a verify pass (roots are rows s * N)
     bool sample_on = false;                 // the LM head of the pass in flight draws instead of taking the arg-max
     unsigned long long sample_seed = 0;
     float sample_inv_t = 1.f;
@@ -362,6 +366,9 @@ void run_target(glance_ctx *ctx, const PassInfo &ps, bf16 *hidden_out, float *lo
         g.x_lo_row = 0;      // logits only decide an arg-max / top-k: one term is enough
         if (ctx->sample_on) {
             g.sample_pos = ctx->ws.row_pos; g.sample_seed = ctx->sample_seed; g.sample_inv_t = ctx->sample_inv_t;
+        }
+        if (ctx->ent_on && ctx->ent_out) {
+            g.ent_out = ctx->ent_out; g.ent_part = ctx->ws.ent_part; g.ent_N = ps.T; g.ent_batch = ps.batch;
         }
         with_row_scales(ctx, g);
         gemm(ctx, 2, ctx->lm_head, ctx->ws.xn, ctx->dims.Rmax, g);
@@ -620,7 +627,9 @@ static int32_t verify_common(glance_ctx *ctx, const glance_seqs *seqs, const gla
     vs.page_table = seqs->page_table; vs.out = rowout_of(ctx); vs.meta = meta_of(ctx); vs.status = ws.status;
     LAUNCH(ctx, KIND_SETUP, launch_setup_verify(vs, ctx->stream));
     PassInfo ps{batch * N, batch * N, batch, N, tree->anc, seqs, 0};
+    ctx->ent_on = true;
     run_target(ctx, ps, (bf16 *)hidden, logits_dbg, decisions);
+    ctx->ent_on = false;
     return finish(ctx);
 }
 
@@ -675,6 +684,12 @@ int32_t glance_commit_forced(glance_ctx *ctx, const glance_seqs *seqs, const voi
     WalkCommit wc{};
     wc.forced_path = path; wc.forced_len = path_len; wc.forced_root = new_root;
     return commit_common(ctx, seqs, wc, hidden);
+}
+
+int32_t glance_log_root_entropy(glance_ctx *ctx, float *entropy) {
+    if (!ctx) return GLANCE_E_INVALID_ARG;
+    ctx->ent_out = entropy;
+    return GLANCE_OK;
 }
 
 int32_t glance_poll_status(glance_ctx *ctx, int32_t *device_status) {

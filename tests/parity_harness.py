@@ -87,6 +87,9 @@ class ParityRun:
                 self.eng.glance_seq_truncate(s, st.P, st.root)
                 self.stats["forced"] += 1
         self.rng = np.random.default_rng(7)
+        # round log: root entropy of every verify pass
+        self.entropy = torch.zeros(batch, dtype=torch.float32, device=dev)
+        self.eng.glance_log_root_entropy(self.entropy)
 
     # ---- state comparison -------------------------------------------------------------------
     def check_state(self, check_root=True):
@@ -182,6 +185,7 @@ class ParityRun:
         else:
             eng.glance_verify_tree_sample(sample_seed, 1.0, logits_dbg=vlog)
         am_g = eng.argmax.cpu().numpy()
+        ent_g = self.entropy.cpu().numpy()
         infos = []
         for s, st in enumerate(self.states):
             assert roots[s] == st.root
@@ -191,6 +195,10 @@ class ParityRun:
             self.stats["max_rel_logit"] = max(self.stats["max_rel_logit"], close(vlog[s, :n], ol[:n], "verify logits", scale))
             for i, oh_i in enumerate([oh] if oh.dim() == 2 else list(oh)):       # one slice per tapped layer
                 close(eng.hidden_all[i, s, :n], oh_i[:n], f"verify hidden, tap {i}")
+            # root entropy (Section 4): exact on the library's own logits, within the logit tolerance of the oracle's
+            own_H = O.root_entropy(vlog[s, 0].cpu())
+            assert abs(float(ent_g[s]) - own_H) <= 1e-3 * max(1.0, own_H), f"root entropy {ent_g[s]} vs {own_H} on own logits"
+            assert abs(float(ent_g[s]) - O.root_entropy(ol[0])) <= 4 * REL_TOL * scale, "root entropy against the oracle"
             if sample_seed is None:
                 oam = O.argmax_lowest(ol)
                 top2 = torch.topk(ol, 2, dim=-1).values
