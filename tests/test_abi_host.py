@@ -51,6 +51,17 @@ def test_workspace_sizing_and_shape_validation(lib):
     assert lib.glance_workspace_bytes(C.byref(bad)) == 0
     bad = binding.make_config(synth.CONFIGS["tiny"].replace(page_size=32), 1, 8)
     assert lib.glance_workspace_bytes(C.byref(bad)) == 0
+    # multi-layer head: taps must be distinct target layers; deeper heads need more workspace
+    one = lib.glance_workspace_bytes(C.byref(binding.make_config(synth.CONFIGS["tiny"], 1, 8)))
+    two = lib.glance_workspace_bytes(C.byref(binding.make_config(synth.CONFIGS["tiny"].replace(head_taps=(0, 1)), 1, 8)))
+    assert two > one > 0
+    for taps in ((0, 0), (0, 2), (-1, 1)):
+        bad = binding.make_config(synth.CONFIGS["tiny"].replace(head_taps=taps), 1, 8)
+        assert lib.glance_workspace_bytes(C.byref(bad)) == 0
+    nine = binding.make_config(synth.CONFIGS["small"].replace(head_taps=(0, 1, 2, 3, 4, 5, 6, 7)), 1, 8)
+    assert lib.glance_workspace_bytes(C.byref(nine)) > 0
+    nine.head_layers = 9
+    assert lib.glance_workspace_bytes(C.byref(nine)) == 0
 
 
 def test_null_arguments_are_rejected_on_the_host(lib):
@@ -60,6 +71,8 @@ def test_null_arguments_are_rejected_on_the_host(lib):
     assert lib.glance_destroy(None) == -1
     assert lib.glance_poll_status(None, None) == -1
     assert lib.glance_build_tree(None, 1, None, None, None, None) == -1
+    assert lib.glance_log_root_entropy(None, None) == -1
+    assert lib.glance_verify_tree_sample(None, None, None, C.c_uint64(1), C.c_float(1.0), None, None, None) == -1
     assert lib.glance_launch_count(None) == 0
 
 
