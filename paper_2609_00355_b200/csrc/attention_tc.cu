@@ -27,6 +27,7 @@ using namespace tc;
 
 constexpr int QT = 128;          // packed query rows per CTA (UMMA M)
 constexpr int KT = kPage;        // keys per tile (UMMA N of S, K of P V)
+constexpr int KS = 3;             // K page ring (one deeper than V's: the next scores are issued a tile ahead)
 constexpr int MAX_SPLITS = 8;     // the splits of a tile form one thread-block cluster
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 
@@ -44,7 +45,7 @@ struct Smem {
     static constexpr int Q_BYTES = SLABS * QT * 128;     // 32 KB at d = 128
     static constexpr int KV_BYTES = SLABS * KT * 128;    // one K or V page: 16 KB at d = 128
     static constexpr int P_BYTES = QT * 128;             // 128 rows x 64 keys bf16
-    static constexpr int OPER_BYTES = Q_BYTES + 4 * KV_BYTES + 2 * P_BYTES;   // P is double-buffered;   // operand buffers (and merge staging)
+    static constexpr int OPER_BYTES = Q_BYTES + (KS + 2) * KV_BYTES + 2 * P_BYTES;   // P is double-buffered;   // operand buffers (and merge staging)
     static constexpr int ROWF = D + 4;                   // floats per merged row: O, m, l, padding
     // split merge: rows received from the cluster's CTAs (each owner gets <= ceil(QT/S) rows from each of S CTAs)
     static constexpr int RECV_BYTES = (QT + MAX_SPLITS) * ROWF * 4;
@@ -53,7 +54,7 @@ struct Smem {
 };
 
 struct alignas(8) AttnBars {
-    uint64_t q_ready, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], merge;
+    uint64_t q_ready, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], merge;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -65,8 +66,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     unsigned char *sQ = smem;
-    unsigned char *sK = sQ + Smem<D>::Q_BYTES;                       // 2 stages
-    unsigned char *sV = sK + 2 * Smem<D>::KV_BYTES;                  // 2 stages
+    unsigned char *sK = sQ + Smem<D>::Q_BYTES;                       // KS stages
+    unsigned char *sV = sK + KS * Smem<D>::KV_BYTES;                 // 2 stages
     unsigned char *sP = sV + 2 * Smem<D>::KV_BYTES;
     __shared__ AttnBars bars;
     __shared__ float red[2][4][QT];                       // cross-column-group exchange of row maxima / sums
@@ -83,9 +84,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 
     if (threadIdx.x == 0) {
         mbar_init(&bars.q_ready, NSOFT);
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < KS; ++b) {
             mbar_init(&bars.k_full[b], 1);
             mbar_init(&bars.k_empty[b], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
             mbar_init(&bars.v_full[b], 1);
             mbar_init(&bars.v_empty[b], 1);
             mbar_init(&bars.s_full[b], 1);
@@ -140,14 +143,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kv) : "memory");
             bool waited = false;
-            int issued = 0;
-            for (int i = 0; i < nt; ++i) {
-                const int st = i & 1;
-                const uint32_t ph = (uint32_t)((i >> 1) & 1);
+            // Rows written by this pass lie in [P - block_B, P + T): the head's refreshed context rows and the new
+            // tree / block rows.  Pages entirely below that are committed context that no kernel of the pass writes,
+            // so they may be fetched before the dependency wait.
+            auto page_rows = [&](int i, int &krow, int &vrow) {
                 const int t = t_begin + i;
-                // rows written by this pass lie in [P - block_B, P + T): the head's refreshed context rows and
-                // the new tree / block rows
-                if (!waited && (i >= 2 || (t + 1) * KT > P - kMaxBlock)) {
+                if (!waited && (t + 1) * KT > P - kMaxBlock) {
                     pdl_wait();
                     waited = true;
                 }
@@ -156,30 +157,51 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     page = 0;
                     set_status(p.status, GLANCE_E_BOUNDS);
                 }
-                const int krow = ((page * 2 + 0) * p.geom.n_kv_heads + kvh) * KT;
-                const int vrow = ((page * 2 + 1) * p.geom.n_kv_heads + kvh) * KT;
-                if (!mbar_wait(&bars.k_empty[st], ph ^ 1u, abort_flag, p.status)) break;
+                krow = ((page * 2 + 0) * p.geom.n_kv_heads + kvh) * KT;
+                vrow = ((page * 2 + 1) * p.geom.n_kv_heads + kvh) * KT;
+            };
+            int issued_k = 0, issued_v = 0;
+            auto issue_k = [&](int i) -> bool {
+                int krow, vrow;
+                page_rows(i, krow, vrow);
+                const int st = i % KS;
+                if (!mbar_wait(&bars.k_empty[st], ((uint32_t)(i / KS) & 1u) ^ 1u, abort_flag, p.status)) return false;
                 mbar_expect_tx(&bars.k_full[st], (uint32_t)Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int sl = 0; sl < SLABS; ++sl)
                     tma_load_2d(sK + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.k_full[st], sl * 64, krow);
-                if (!mbar_wait(&bars.v_empty[st], ph ^ 1u, abort_flag, p.status)) { issued = -(i + 1); break; }
+                issued_k = i + 1;
+                return true;
+            };
+            auto issue_v = [&](int i) -> bool {
+                int krow, vrow;
+                page_rows(i, krow, vrow);
+                const int st = i & 1;
+                if (!mbar_wait(&bars.v_empty[st], ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_flag, p.status)) return false;
                 mbar_expect_tx(&bars.v_full[st], (uint32_t)Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int sl = 0; sl < SLABS; ++sl)
                     tma_load_2d(sV + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.v_full[st], sl * 64, vrow);
-                issued = i + 1;
+                issued_v = i + 1;
+                return true;
+            };
+            // K pages run KS - 1 tiles ahead of V pages: the scores of tile i + 1 are issued before P V of tile i,
+            // and a V slot only frees when P V of two tiles back has finished
+            bool pok = true;
+            for (int i = 0; i < KS - 1 && i < nt && pok; ++i) pok = issue_k(i);
+            for (int i = 0; i < nt && pok; ++i) {
+                if (i + KS - 1 < nt) pok = issue_k(i + KS - 1);
+                pok = pok && issue_v(i);
             }
             if (!waited) pdl_wait();
             if (*abort_flag) {
                 // copies already issued must land before the CTA may exit
-                const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
-                for (int i = max(0, nk - 2); i < nk; ++i) {
+                for (int i = max(0, issued_k - KS); i < issued_k; ++i) {
                     const uint64_t t0 = global_ns();
-                    while (!mbar_try_wait(&bars.k_full[i & 1], (uint32_t)(i >> 1) & 1u))
+                    while (!mbar_try_wait(&bars.k_full[i % KS], (uint32_t)(i / KS) & 1u))
                         if (global_ns() - t0 > kWaitLimitNs) break;
                 }
-                for (int i = max(0, nv - 2); i < nv; ++i) {
+                for (int i = max(0, issued_v - 2); i < issued_v; ++i) {
                     const uint64_t t0 = global_ns();
                     while (!mbar_try_wait(&bars.v_full[i & 1], (uint32_t)(i >> 1) & 1u))
                         if (global_ns() - t0 > kWaitLimitNs) break;
@@ -194,17 +216,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             const uint32_t idesc_s = umma_idesc(KT);              // M 128, N 64 keys
             const uint32_t idesc_o = umma_idesc_bmn(D);           // M 128, N d, B = V is MN-major
             auto issue_s = [&](int i) -> bool {
-                const int st = i & 1;
-                if (!mbar_wait(&bars.k_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) return false;
+                const int st = i & 1, ks_slot = i % KS;   // S buffer in TMEM / K page slot in shared memory
+                if (!mbar_wait(&bars.k_full[ks_slot], (uint32_t)(i / KS) & 1u, abort_flag, p.status)) return false;
                 tc_fence_after();
-                const uint32_t kbase = smem_u32(sK + st * Smem<D>::KV_BYTES);
+                const uint32_t kbase = smem_u32(sK + ks_slot * Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const int sl = ks >> 2, kk = ks & 3;
                     umma_f16(tmem_S + (uint32_t)(st * 64), umma_desc(smem_u32(sQ) + sl * QT * 128) + (uint64_t)(kk * 2),
                              umma_desc(kbase + sl * KT * 128) + (uint64_t)(kk * 2), idesc_s, ks > 0 ? 1u : 0u);
                 }
-                umma_commit(&bars.k_empty[st]);           // K page free once these MMAs have read it
+                umma_commit(&bars.k_empty[ks_slot]);      // K page free once these MMAs have read it
                 umma_commit(&bars.s_full[st]);
                 return true;
             };
@@ -300,7 +322,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             float mt = -INFINITY;
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-                float v = sc[j] * sl2;
+                float v = sc[j];                          // raw score: the scale is folded into the exponent below
                 if (need_mask) {
                     const int key = key0 + cg * 16 + j;
                     bool vis = key < P;
@@ -314,7 +336,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 sc[j] = v;
                 mt = fmaxf(mt, v);
             }
-            // row maximum of the tile across the four column groups
+            // row maximum of the tile across the four column groups (in scaled log2 units: sl2 > 0 keeps the order)
+            mt *= sl2;
             red[i & 1][cg][row] = mt;
             asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");   // only the four warps of this lane quarter share rows
             if (*abort_flag) break;                       // a quarter that leaves stops arriving at p_full: every wait is bounded
@@ -362,8 +385,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     const float a = sc[c * 8 + 2 * j], b = sc[c * 8 + 2 * j + 1];
-                    const float pa = ex2_approx(a - m_sub);
-                    const float pb = ex2_approx(b - m_sub);
+                    const float pa = ex2_approx(fmaf(a, sl2, -m_sub));
+                    const float pb = ex2_approx(fmaf(b, sl2, -m_sub));
                     rs += pa + pb;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
                     w[j] = *reinterpret_cast<uint32_t *>(&h2);
