@@ -125,7 +125,8 @@ def to_device(w, dev):
 class RoundBench:
     """Drives rounds of the library at controlled p_m.  All method arithmetic runs in the CUDA library."""
 
-    def __init__(self, cfg, device, rank=0, weights=None):
+    def __init__(self, cfg, device, rank=0, weights=None, max_new=None):
+        """max_new: tokens the sequences may grow by over the engine's life (default: cfg.rounds full blocks)."""
         from paper_2609_00355_b200.binding import Engine, TreeBuffers
         self.cfg, self.dev = cfg, device
         self.no_lookahead = False
@@ -134,7 +135,11 @@ class RoundBench:
         self.tw, self.hw = weights if weights is not None else synth.make_weights(cfg, device)
         self.stream = torch.cuda.Stream(device)      # the library's stream; also made torch's current stream
         torch.cuda.set_stream(self.stream)
-        self.eng = Engine(cfg, self.tw, self.hw, batch=cfg.batch, stream=self.stream)
+        max_len = None
+        if max_new is not None:
+            longest = max(synth.batch_context_lengths(cfg)) if cfg.batch > 1 else cfg.ctx
+            max_len = longest + max_new + 2 * cfg.tree_N + cfg.page_size
+        self.eng = Engine(cfg, self.tw, self.hw, batch=cfg.batch, stream=self.stream, max_len=max_len)
         self.graph = None
         eng = self.eng
         # round log for the entropy law: every verify pass leaves the root entropy of each sequence here
@@ -398,7 +403,9 @@ def main():
         dist_mod.init_process_group("nccl", device_id=dev)
         dist = dist_mod
     torch.manual_seed(0)
-    bench = RoundBench(cfg, dev, rank)
+    # every timed, profiled and end-to-end round may commit a whole block
+    rounds_total = 2 * (warmup + args.steps) + min(args.steps, 16) + 2
+    bench = RoundBench(cfg, dev, rank, max_new=max(rounds_total, cfg.rounds) * cfg.block_B)
     bench.no_lookahead = args.no_lookahead
     bench.sample_seed = args.sample_seed
     eng = bench.eng
