@@ -432,3 +432,70 @@ def test_rounds_small_three_layer_head(harness):
     run.check_head_state()
     print("three-layer head parity stats:", run.stats)
     assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_graph_replay_equals_plain_launches(harness):
+    """One CUDA graph captured from a round serves every later round (all ragged quantities live in device memory):
+    an engine replaying the graph and an engine making the four calls stay bit-identical over rounds with different
+    trees and accept lengths."""
+    from paper_2609_00355_b200.binding import Engine
+    cfg = synth.CONFIGS["small"].replace(rounds=16)
+    tw, hw = synth.make_weights(cfg, "cuda")
+    img, ids = synth.make_context(cfg, "cuda")
+    stream = torch.cuda.Stream()
+    engines = []
+    for use_stream in (None, stream):
+        eng = Engine(cfg, tw, hw, batch=1, stream=use_stream)
+        eng.prefill_context(0, img, ids)
+        engines.append(eng)
+    plain, graphed = engines
+    L, k = cfg.L, cfg.topk
+    cand_ids = torch.zeros(1, L, k, dtype=torch.int32, device="cuda")
+    cand_lp = torch.from_numpy(synth.controlled_marginals(0.6, k, L))[None].cuda()
+    rng = np.random.default_rng(5)
+
+    def calls(eng):
+        eng.glance_draft_block()
+        eng.glance_build_tree(cand_ids, cand_lp)
+        eng.glance_verify_tree()
+        eng.glance_accept_commit()
+
+    graph = None
+    accepts = []
+    for r in range(10):
+        # plant the plain engine's true continuation so that accept lengths vary: look ahead with single-node trees
+        snap = plain.snapshot_state()
+        one = harness.TreeBuffers(1, cfg.tree_N, torch.device("cuda"))
+        for i in range(cfg.tree_N):                 # every row sees itself only (tree_N <= 63 here)
+            one.anc[0, i, 0] = 1 << i
+        Y = []
+        for _ in range(L):
+            one.token[:, 0].copy_(plain.root)
+            plain.glance_verify_tree(tree=one)
+            plain.glance_accept_commit(tree=one)
+            Y.append(int(plain.root[0]))
+        plain.restore_state(snap)
+        cand_ids.copy_(torch.from_numpy(synth.controlled_candidates(Y, 0.6, k, L, cfg.vocab, rng))[None])
+        calls(plain)
+        with torch.cuda.stream(stream):
+            if r == 0:
+                calls(graphed)                      # first round plain: sets up attributes and descriptors
+            else:
+                if graph is None:
+                    snap_g = graphed.snapshot_state()
+                    graph = graphed.capture(lambda: calls(graphed))
+                    graphed.restore_state(snap_g)
+                graph.replay()
+        torch.cuda.synchronize()
+        plain.check_device_status()
+        graphed.check_device_status()
+        accepts.append(int(plain.accept_len[0]))
+        assert torch.equal(plain.seq_len, graphed.seq_len) and torch.equal(plain.root, graphed.root)
+        assert torch.equal(plain.accept_len, graphed.accept_len) and torch.equal(plain.out_tokens, graphed.out_tokens)
+        assert torch.equal(plain.topk_ids, graphed.topk_ids) and torch.equal(plain.topk_lp, graphed.topk_lp)
+        P = int(plain.seq_len[0])
+        for l in (0, cfg.n_layers - 1):
+            Ka, Va = plain.gather_kv(0, l, P)
+            Kb, Vb = graphed.gather_kv(0, l, P)
+            assert torch.equal(Ka, Kb) and torch.equal(Va, Vb)
+    assert len(set(accepts)) > 1, accepts
