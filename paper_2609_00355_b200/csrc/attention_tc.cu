@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     unsigned char *sP = sV + 2 * Smem<D>::KV_BYTES;
     __shared__ AttnBars bars;
     __shared__ float red[2][4][QT];                       // cross-column-group exchange of row maxima / sums
+    __shared__ int quit[2][4];                            // per lane quarter: leave the tile loop (decided by one thread)
 
     unsigned long long *trace = (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? p.trace : nullptr;
     if (trace && threadIdx.x == 0) trace[0] = global_ns();
@@ -339,8 +340,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             // row maximum of the tile across the four column groups (in scaled log2 units: sl2 > 0 keeps the order)
             mt *= sl2;
             red[i & 1][cg][row] = mt;
+            // Leaving the loop must be decided once per quarter: its four warps meet at the barrier below every tile,
+            // and the abort flag can change between two warps' reads.  One thread samples it before the barrier.
+            if (cg == 0 && lane == 0) quit[i & 1][q] = *abort_flag;
             asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");   // only the four warps of this lane quarter share rows
-            if (*abort_flag) break;                       // a quarter that leaves stops arriving at p_full: every wait is bounded
+            if (quit[i & 1][q]) break;                    // a quarter that leaves stops arriving at p_full: every wait is bounded
             mt = fmaxf(fmaxf(red[i & 1][0][row], red[i & 1][1][row]), fmaxf(red[i & 1][2][row], red[i & 1][3][row]));
             if (i > 1) {
                 // this tile's P buffer was read by the second MMA of tile i-2
