@@ -103,3 +103,67 @@ def test_verify_pass_7b_full_depth():
     for i in range(n):
         if margin[i] > H.MARGIN:
             assert am[i] == int(oam[i]), f"node {i}: arg-max differs at margin {margin[i]:.3g}"
+
+
+def test_draft_pass_7b_full_vocabulary():
+    """The draft pass at the benchmark's widths and full vocabulary (head layer 3584 / 18944, LM head over 152064
+    ids, top-8 of every block slot) against the oracle, on a seeded synthetic head context of 1536 positions.
+    The target is cut to one layer: the draft pass does not run it."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_00355_b200.binding import Engine
+    from tests import parity_harness as H
+
+    cfg = synth.CONFIGS["7b"].replace(n_layers=1)
+    dev = torch.device("cuda:0")
+    tw, hw = synth.make_weights(cfg, dev)
+    eng = Engine(cfg, tw, hw, batch=1)
+    P, B, k = cfg.ctx, cfg.block_B, cfg.topk
+    g = torch.Generator(device=dev).manual_seed(23)
+    page = cfg.page_size
+    pos = torch.arange(P, device=dev)
+    pages = eng.page_table[0].long()[pos // page]
+    hK = (torch.randn(P, cfg.n_kv_heads, cfg.head_dim, generator=g, device=dev) * 0.5).to(torch.bfloat16)
+    hV = (torch.randn(P, cfg.n_kv_heads, cfg.head_dim, generator=g, device=dev) * 0.5).to(torch.bfloat16)
+    eng.head_kv_all[0, pages, 0, :, pos % page, :] = hK
+    eng.head_kv_all[0, pages, 1, :, pos % page, :] = hV
+    eng.seq_len[0] = P
+    eng.root[0] = 4321
+    eng.feat_count[0] = 0                      # nothing pending: the context above is complete
+    dlog = torch.zeros(1, B, cfg.vocab, dtype=torch.float32, device=dev)
+    eng.glance_draft_block(logits_dbg=dlog)
+    eng.check_device_status()
+    torch.cuda.synchronize()
+
+    sh = O.Shape.of(cfg)
+    otw = {"embed": tw["embed"].cpu().float(), "lm_head": tw["lm_head"].cpu().float()}
+    ohw = O.widen(hw)
+    cap = P + B + 8
+    st = O.SeqState(P, 4321, [], [], torch.zeros(cap, cfg.n_kv_heads, cfg.head_dim),
+                    torch.zeros(cap, cfg.n_kv_heads, cfg.head_dim), torch.zeros(1))
+    st.hK[:P], st.hV[:P] = hK.cpu().float(), hV.cpu().float()
+    ol = O.draft_block(sh, otw, ohw, st, B)
+    scale = float(ol[1:].abs().max())
+    err = float((dlog[0, 1:].cpu() - ol[1:]).abs().max())
+    assert err <= H.REL_TOL * scale, f"draft logits: max-abs error {err:.4g} > {H.REL_TOL} x {scale:.4g}"
+    # top-k ids and log-probabilities wherever the oracle's neighbouring gaps are clear
+    oid, olp = O.topk_logprobs(ol, k)
+    ids_g, lp_g = eng.topk_ids[0].cpu().numpy(), eng.topk_lp[0].cpu().numpy()
+    srt = torch.sort(ol, dim=-1, descending=True).values.numpy()
+    checked = 0
+    for j in range(cfg.L):
+        for r in range(k):
+            gap_hi = srt[j + 1][r - 1] - srt[j + 1][r] if r > 0 else np.inf
+            gap_lo = srt[j + 1][r] - srt[j + 1][r + 1]
+            if gap_hi > H.MARGIN and gap_lo > H.MARGIN:
+                assert ids_g[j, r] == oid[j, r], f"top-k id offset {j + 1} rank {r}"
+                assert abs(lp_g[j, r] - olp[j, r]) <= H.REL_TOL * scale
+                checked += 1
+    assert checked > 0
+    # the library's (ids, lp) are exactly the top-k and log-softmax of its own logits
+    own = dlog[0, 1:].cpu()
+    lse = torch.logsumexp(own.double(), dim=-1)
+    top = torch.topk(own, k, dim=-1)
+    assert np.array_equal(np.sort(ids_g, axis=1), np.sort(top.indices.numpy(), axis=1))
+    got = torch.gather(own.double(), 1, torch.from_numpy(ids_g).long()) - lse[:, None]
+    assert float((got - torch.from_numpy(lp_g).double()).abs().max()) < 1e-3
