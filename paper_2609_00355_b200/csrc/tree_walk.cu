@@ -174,11 +174,20 @@ __global__ void __launch_bounds__(256) walk_commit_kernel(WalkCommit p) {
     const int P = p.seq_len[s];
     const int L = p.B - 1;
 
+    // the walk's three small arrays are fetched once, coalesced, instead of one dependent global load per step
+    __shared__ int sh_am[kMaxTreeN], sh_tok[kMaxTreeN], sh_par[kMaxTreeN];
+    if (p.argmax) {
+        for (int i = threadIdx.x; i < p.N; i += blockDim.x) {
+            sh_am[i] = p.argmax[(size_t)s * p.N + i];
+            sh_tok[i] = p.token[(size_t)s * p.N + i];
+            sh_par[i] = p.parent[(size_t)s * p.N + i];
+        }
+    }
+    __syncthreads();
     if (threadIdx.x < 32) {
         const int lane = threadIdx.x;
         if (p.argmax) {
-            const int32_t *am = p.argmax + (size_t)s * p.N;
-            const int32_t *tok = p.token + (size_t)s * p.N, *par = p.parent + (size_t)s * p.N;
+            const int *am = sh_am, *tok = sh_tok, *par = sh_par;
             int nn = p.n_nodes[s];
             nn = nn < 1 ? 1 : (nn > p.N ? p.N : nn);
             int v = 0, a = 0, t = am[0];
@@ -247,21 +256,27 @@ __global__ void __launch_bounds__(256) walk_commit_kernel(WalkCommit p) {
         __syncthreads();
     }
 
+    // features of the accepted path (every tap slice): hidden[path[i]] -> feat[i], in 16-byte pieces shared out over
+    // all blocks of the sequence (nothing reads feat before the next draft pass)
+    {
+        const int CH = p.H >> 3;                        // H is a multiple of 64
+        const int per_tap = (a + 1) * CH;
+        const int total = p.n_taps * per_tap;
+        for (int it = blockIdx.y * blockDim.x + threadIdx.x; it < total; it += gridDim.y * blockDim.x) {
+            const int tap = it / per_tap, rem = it - tap * per_tap;
+            const int i = rem / CH, c = rem - i * CH;
+            const int4 *src = reinterpret_cast<const int4 *>(p.hidden + ((size_t)tap * p.batch * p.N + (size_t)s * p.N + sh_path[i]) * p.H) + c;
+            int4 *dst = reinterpret_cast<int4 *>(p.feat + ((size_t)tap * p.batch * p.B + (size_t)s * p.B + i) * p.H) + c;
+            *dst = *src;
+        }
+    }
+
     // last block of the sequence publishes the outcome
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) sh_last = (atomicAdd(&p.counters[s], 1) == (int)gridDim.y - 1);
     __syncthreads();
     if (!sh_last) return;
-    for (int tap = 0; tap < p.n_taps; ++tap) {
-        const bf16 *hid = p.hidden + (size_t)tap * p.batch * p.N * p.H;
-        bf16 *ft = p.feat + (size_t)tap * p.batch * p.B * p.H;
-        for (int i = 0; i <= a; ++i) {
-            const bf16 *src = hid + ((size_t)s * p.N + sh_path[i]) * p.H;
-            bf16 *dst = ft + ((size_t)s * p.B + i) * p.H;
-            for (int c = threadIdx.x; c < p.H; c += blockDim.x) dst[c] = src[c];
-        }
-    }
     if (threadIdx.x == 0) {
         if (p.accept_len) p.accept_len[s] = a;
         for (int d = 0; d < p.B; ++d) {
