@@ -499,3 +499,17 @@ def test_graph_replay_equals_plain_launches(harness):
             Kb, Vb = graphed.gather_kv(0, l, P)
             assert torch.equal(Ka, Kb) and torch.equal(Va, Vb)
     assert len(set(accepts)) > 1, accepts
+
+
+@pytest.mark.parametrize("block_B,topk,tree_N", [(2, 16, 2), (2, 1, 2), (16, 16, 128), (3, 2, 7), (16, 2, 33)])
+def test_rounds_extreme_block_topk_budget(harness, block_B, topk, tree_N):
+    """Corners of the supported shapes: the shortest block (L = 1), the widest top-k, the smallest and the largest
+    verify budget, budgets that the candidate trie cannot fill (n_nodes < N) and budgets that are not multiples of
+    the GEMM row granularity."""
+    cfg = synth.CONFIGS["tiny"].replace(block_B=block_B, topk=topk, tree_N=tree_N, rounds=8)
+    run = harness.ParityRun(cfg)
+    run.check_state()
+    for r in range(3):
+        run.round(p_m=(0.7 if r else None), check_draft=(r == 0))
+    run.check_head_state()
+    assert run.stats["max_rel_logit"] <= 2e-2
