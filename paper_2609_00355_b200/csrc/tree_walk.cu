@@ -23,16 +23,17 @@ __device__ __forceinline__ bool cand_before(const Cand &a, const Cand &b) {
     return a.key < b.key;
 }
 
-// Everything the loop touches lives in shared memory (candidate tables, node arrays, ancestor masks): an
-// iteration is a handful of shared-memory accesses and one warp reduction; the tree is written out once at the end.
+// The frontier lives in registers, entry e in slot e / 32 of lane e % 32; every lane follows the whole loop
+// redundantly (counts, the popped entry, the two new entries), so that a pop needs one hardware warp max over the
+// 32-bit score images, a handful of shuffles and no barrier: the only shared-memory traffic is the candidate
+// tables (read-only) and the node arrays (each written and later re-read by the same lane).
+// An entry is (sk, t, meta, ps): sk = order-preserving image of the score, t = tie word ((15 - depth) << 60 |
+// complemented 60-bit path key), meta = depth | rank << 4 | parent << 8, ps = the parent's score (a next-rank
+// sibling's score is one fp32 add from it).  Larger (sk, t) is popped first.
+constexpr int kFrSlots = (kMaxTreeN + 4 + 31) / 32;      // 5 slots cover a frontier of N + 1 <= 129 entries
+
 __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, const int32_t *root, const int32_t *ids,
                                                         const float *lp, glance_tree out) {
-    constexpr int CAP = kMaxTreeN + 4;
-    __shared__ float f_score[CAP];
-    __shared__ int f_depth[CAP], f_rank[CAP], f_parent[CAP];
-    __shared__ unsigned long long f_key[CAP];
-    __shared__ uint32_t f_sk[CAP];                   // order-preserving image of f_score
-    __shared__ unsigned long long f_t[CAP];          // tie word: (15 - depth) << 60 | ~key
     __shared__ float n_score[kMaxTreeN];
     __shared__ int n_token[kMaxTreeN], n_parent[kMaxTreeN], n_depth[kMaxTreeN], n_rank[kMaxTreeN];
     __shared__ unsigned long long n_anc[kMaxTreeN * 2];
@@ -49,36 +50,49 @@ __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, con
     const int32_t root_tok = root[s];
     __syncwarp();
 
+    // five slots as named scalars (arrays, even with unrolled compile-time indices, ended up in local memory)
+    static_assert(kFrSlots == 5, "the slot macros below spell out five slots");
+    uint32_t sk0 = 0u, sk1 = 0u, sk2 = 0u, sk3 = 0u, sk4 = 0u, me0 = 0u, me1 = 0u, me2 = 0u, me3 = 0u, me4 = 0u;
+    unsigned long long tw0 = 0ull, tw1 = 0ull, tw2 = 0ull, tw3 = 0ull, tw4 = 0ull;
+    float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f, ps4 = 0.f;
+    const bool deep = N > 94;                            // the frontier (<= N + 1 entries) reaches slots 3 and 4
+#define GLANCE_SLOTS(OP) OP(0, sk0, tw0, me0, ps0) OP(1, sk1, tw1, me1, ps1) OP(2, sk2, tw2, me2, ps2) \
+    if (deep) { OP(3, sk3, tw3, me3, ps3) OP(4, sk4, tw4, me4, ps4) }
+#define GLANCE_PUT_OP(u, sk, tw, me, ps) if (pmine && pslot == u) { sk = psk; tw = ptw; me = pmeta; ps = pps; }
+#define GLANCE_PUT(e_, sk_, t_, meta_, ps_)                                     \
+    do {                                                                        \
+        const int pe = (e_);                                                    \
+        const bool pmine = (pe & 31) == lane;                                   \
+        const int pslot = pe >> 5;                                              \
+        const uint32_t psk = (sk_), pmeta = (meta_);                            \
+        const unsigned long long ptw = (t_);                                    \
+        const float pps = (ps_);                                                \
+        GLANCE_SLOTS(GLANCE_PUT_OP)                                             \
+    } while (0)
     auto tie_word = [](int depth, unsigned long long key) {
         return ((unsigned long long)(15 - depth) << 60) | (~key & 0x0fffffffffffffffull);
     };
-    int nc = 1, fc = 0;                                  // node / frontier counts: the same in every lane
-    if (L >= 1 && N > 1) fc = 1;
     if (lane == 0) {
         n_token[0] = root_tok; n_parent[0] = -1; n_depth[0] = 0; n_rank[0] = 0; n_score[0] = 0.f;
-        if (fc) {
-            const float sc0 = __fadd_rn(0.f, s_lp[0]);
-            f_score[0] = sc0; f_sk[0] = float_key(sc0);
-            f_depth[0] = 1; f_rank[0] = 0; f_parent[0] = 0; f_key[0] = 0ull; f_t[0] = tie_word(1, 0ull);
-        }
     }
     if (lane < W) n_anc[lane] = (lane == 0) ? 1ull : 0ull;
-    __syncwarp();
+    int nc = 1, fc = 0;                                  // node / frontier counts: the same in every lane
+    if (L >= 1 && N > 1) {
+        GLANCE_PUT(0, float_key(__fadd_rn(0.f, s_lp[0])), tie_word(1, 0ull), 1u, 0.f);
+        fc = 1;
+    }
 
-    // The order (score desc, depth asc, key asc) as integers: a 32-bit order-preserving image of the score and a
-    // 64-bit tie word (15 - depth in the top four bits, the complemented 60-bit path key below); larger wins.
     while (fc > 0 && nc < N) {
-        uint32_t bsk = 0;
+        // this lane's best entry
+        uint32_t bsk = 0u;
         unsigned long long bt = 0ull;
-        int bi = -1;
-        for (int e = lane; e < fc; e += 32) {
-            const uint32_t sk = f_sk[e];
-            const unsigned long long t = f_t[e];
-            if (bi < 0 || sk > bsk || (sk == bsk && t > bt)) { bsk = sk; bt = t; bi = e; }
-        }
+        int bu = -1;
+#define GLANCE_BEST_OP(u, sk, tw, me, ps) \
+        if (u * 32 + lane < fc && (bu < 0 || sk > bsk || (sk == bsk && tw > bt))) { bsk = sk; bt = tw; bu = u; }
+        GLANCE_SLOTS(GLANCE_BEST_OP)
         // warp arg-best: hardware max over the score image, then (rarely) over the halves of the tie word
-        const uint32_t m1 = __reduce_max_sync(0xffffffffu, bi >= 0 ? bsk : 0u);
-        uint32_t live = __ballot_sync(0xffffffffu, bi >= 0 && bsk == m1);
+        const uint32_t m1 = __reduce_max_sync(0xffffffffu, bu >= 0 ? bsk : 0u);
+        uint32_t live = __ballot_sync(0xffffffffu, bu >= 0 && bsk == m1);
         if (__popc(live) > 1) {
             const bool in = (live >> lane) & 1u;
             const uint32_t m2 = __reduce_max_sync(0xffffffffu, in ? (uint32_t)(bt >> 32) : 0u);
@@ -89,51 +103,60 @@ __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, con
                 live = __ballot_sync(0xffffffffu, in2 && (uint32_t)bt == m3);
             }
         }
-        // (score, depth, key) identifies a candidate uniquely: exactly one lane is left
-        bi = __shfl_sync(0xffffffffu, bi, __ffs(live) - 1);
-        const int i = nc;
-        const int dpt = f_depth[bi], rk = f_rank[bi], par = f_parent[bi];
-        const float sc = f_score[bi];
-        const unsigned long long key = f_key[bi];
-        // the popped entry is replaced by the last one; the child and the next sibling are appended
-        const int last = fc - 1;
-        const bool has_child = dpt < L, has_sib = rk + 1 < k;
-        float mv_score = 0.f; int mv_depth = 0, mv_rank = 0, mv_parent = 0; unsigned long long mv_key = 0ull, mv_t = 0ull;
-        uint32_t mv_sk = 0u;
-        if (lane == 3 && bi != last) {
-            mv_score = f_score[last]; mv_depth = f_depth[last]; mv_rank = f_rank[last];
-            mv_parent = f_parent[last]; mv_key = f_key[last]; mv_sk = f_sk[last]; mv_t = f_t[last];
-        }
-        unsigned long long aw = 0ull;
-        if (lane < W) {
-            aw = n_anc[par * W + lane];
-            if ((i >> 6) == lane) aw |= 1ull << (i & 63);
-        }
-        const float par_score = n_score[par];
-        __syncwarp();                                    // all reads of the old frontier are done
-        if (lane < W) n_anc[i * W + lane] = aw;
+        // (score, depth, key) identifies a candidate uniquely: exactly one lane is left; everybody takes its entry
+        const int wl = __ffs(live) - 1;
+        uint32_t bmeta = 0u;
+        float bps = 0.f;
+#define GLANCE_META_OP(u, sk, tw, me, ps) if (bu == u) { bmeta = me; bps = ps; }
+        GLANCE_SLOTS(GLANCE_META_OP)
+        bu = __shfl_sync(0xffffffffu, bu, wl);
+        bsk = __shfl_sync(0xffffffffu, bsk, wl);
+        bt = __shfl_sync(0xffffffffu, bt, wl);
+        bmeta = __shfl_sync(0xffffffffu, bmeta, wl);
+        bps = __shfl_sync(0xffffffffu, bps, wl);
+        const int dpt = bmeta & 15, rk = (bmeta >> 4) & 15, par = (int)(bmeta >> 8);
+        const float sc = key_float(bsk);
+        const unsigned long long key = ~bt & 0x0fffffffffffffffull;
+        const int i = nc++;
         if (lane == 0) {
             n_token[i] = s_id[(dpt - 1) * k + rk];
             n_parent[i] = par; n_depth[i] = dpt; n_rank[i] = rk; n_score[i] = sc;
-        } else if (lane == 1 && has_child) {
-            const float cs = __fadd_rn(sc, s_lp[dpt * k + 0]);
-            f_score[last] = cs; f_sk[last] = float_key(cs);
-            f_depth[last] = dpt + 1; f_rank[last] = 0; f_parent[last] = i; f_key[last] = key; f_t[last] = tie_word(dpt + 1, key);
-        } else if (lane == 2 && has_sib) {
-            const int at = last + (has_child ? 1 : 0);
-            const float ss = __fadd_rn(par_score, s_lp[(dpt - 1) * k + rk + 1]);
-            const unsigned long long sk2 = key + (1ull << (4 * (15 - dpt)));
-            f_score[at] = ss; f_sk[at] = float_key(ss);
-            f_depth[at] = dpt; f_rank[at] = rk + 1; f_parent[at] = par;
-            f_key[at] = sk2; f_t[at] = tie_word(dpt, sk2);
-        } else if (lane == 3 && bi != last) {
-            f_score[bi] = mv_score; f_depth[bi] = mv_depth; f_rank[bi] = mv_rank; f_parent[bi] = mv_parent; f_key[bi] = mv_key;
-            f_sk[bi] = mv_sk; f_t[bi] = mv_t;
         }
-        nc = nc + 1;
-        fc = last + (has_child ? 1 : 0) + (has_sib ? 1 : 0);
-        __syncwarp();
+        if (lane < W) {                                  // lane w owns word w of every node's mask
+            unsigned long long aw = n_anc[par * W + lane];
+            if ((i >> 6) == lane) aw |= 1ull << (i & 63);
+            n_anc[i * W + lane] = aw;
+        }
+        // the popped slot takes the last entry; the child and the next sibling are appended
+        const int bi = bu * 32 + wl, last = fc - 1;
+        if (bi != last) {
+            uint32_t lsk = 0u, lmeta = 0u;
+            unsigned long long lt = 0ull;
+            float lps = 0.f;
+#define GLANCE_LAST_OP(u, sk, tw, me, ps) if ((last >> 5) == u) { lsk = sk; lt = tw; lmeta = me; lps = ps; }
+            GLANCE_SLOTS(GLANCE_LAST_OP)
+            lsk = __shfl_sync(0xffffffffu, lsk, last & 31);
+            lt = __shfl_sync(0xffffffffu, lt, last & 31);
+            lmeta = __shfl_sync(0xffffffffu, lmeta, last & 31);
+            lps = __shfl_sync(0xffffffffu, lps, last & 31);
+            GLANCE_PUT(bi, lsk, lt, lmeta, lps);
+        }
+        fc = last;
+        if (dpt < L) {
+            GLANCE_PUT(fc, float_key(__fadd_rn(sc, s_lp[dpt * k])), tie_word(dpt + 1, key), (uint32_t)(dpt + 1) | ((uint32_t)i << 8), sc);
+            ++fc;
+        }
+        if (rk + 1 < k) {
+            GLANCE_PUT(fc, float_key(__fadd_rn(bps, s_lp[(dpt - 1) * k + rk + 1])), tie_word(dpt, key + (1ull << (4 * (15 - dpt)))), (uint32_t)dpt | ((uint32_t)(rk + 1) << 4) | ((uint32_t)par << 8), bps);
+            ++fc;
+        }
     }
+#undef GLANCE_SLOTS
+#undef GLANCE_PUT_OP
+#undef GLANCE_PUT
+#undef GLANCE_BEST_OP
+#undef GLANCE_META_OP
+#undef GLANCE_LAST_OP
     __syncwarp();
     if (lane == 0) out.n_nodes[s] = nc;
     int32_t *token = out.token + (size_t)s * N, *parent = out.parent + (size_t)s * N;
