@@ -194,105 +194,194 @@ void launch_setup_draft(const DraftSetup &p, cudaStream_t st) {
 }
 
 // ------------------------------------------------------------------------------------------
-// block-wide max of packed (value desc, id asc) keys
-// ------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long *sh) {
-    v = warp_max_u64(v);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
-    __syncthreads();
-    unsigned long long r = 0;
-    const int nw = blockDim.x >> 5;
-    for (int w = 0; w < nw; ++w) r = sh[w] > r ? sh[w] : r;
-    return r;
-}
-
-// ------------------------------------------------------------------------------------------
 // per-offset top-k and log-softmax (Assumption 1: marginals q_j over the full vocabulary), two stages.
 // Stage 1: every warp owns 1024 consecutive vocabulary entries held in registers and emits its k best
-// packed (value, id) keys plus its max and sum of exponentials.  Stage 2: one block per (sequence,
-// offset) merges the warps' candidates with k rounds of a block-wide max and combines the partial
-// log-sum-exp terms in a fixed order.  Keys are unique, so the result does not depend on timing.
+// packed (value, id) keys (sorted) plus its max and sum of exponentials.  Stage 2: one warp per (sequence,
+// offset) merges the warps' candidates and combines the partial log-sum-exp terms in a fixed order.  Both
+// stages first find a threshold that the k best are known to reach (the k-th largest of the lane maxima / of
+// the lists' heads), collect the few keys at or above it and rank only those.  Keys are unique, so the result
+// does not depend on timing.
 // ------------------------------------------------------------------------------------------
 constexpr int kTopkWarpSpan = 1024;
 
 __global__ void __launch_bounds__(128) topk_stage1_kernel(const float *logits, int B, int V, int k, int n_warps,
                                                           unsigned long long *cand, float *ml) {
+    constexpr int CAP = 64;                              // candidates a warp may collect before it falls back
+    __shared__ unsigned long long lists[4][CAP];
     const int L = B - 1;
     const int row = blockIdx.y;                         // (s, j-1)
     const int s = row / L, j = row % L + 1;
-    const int gw = blockIdx.x * 4 + (threadIdx.x >> 5);
+    const int wib = threadIdx.x >> 5;
+    const int gw = blockIdx.x * 4 + wib;
     const int lane = threadIdx.x & 31;
     if (gw >= n_warps) return;
     const float *src = logits + ((size_t)s * B + j) * V;
     const int base = gw * kTopkWarpSpan;
-    unsigned long long key[32];
+    float val[32];
     float m = -INFINITY;
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
         const int c = base + i * 32 + lane;
-        const float v = c < V ? src[c] : -INFINITY;
-        key[i] = c < V ? pack_val_id(v, c) : 0ull;
-        m = fmaxf(m, v);
+        val[i] = c < V ? src[c] : -INFINITY;
+        m = fmaxf(m, val[i]);
     }
+    const float lane_max = m;
     m = warp_max(m);
     float sum = 0.f;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        const int c = base + i * 32 + lane;
-        if (c < V) sum += expf(unpack_val(key[i]) - m);
-    }
+    for (int i = 0; i < 32; ++i) sum += expf(val[i] - m);        // entries beyond V are -inf: they add exactly 0
     sum = warp_sum(sum);
     if (lane == 0) {
         ml[((size_t)row * n_warps + gw) * 2] = m;
         ml[((size_t)row * n_warps + gw) * 2 + 1] = sum;
     }
+    unsigned long long *out = cand + ((size_t)row * n_warps + gw) * k;
+    // Threshold: the k-th largest of the 32 lane maxima.  At least k values of the span are >= it, so every one of
+    // the span's k best is; usually only a few more are.  (k <= 16 <= 32 lanes.)
+    uint32_t cur = float_key(lane_max), thr = 0u;
+    for (int t = 0; t < k; ++t) {
+        thr = __reduce_max_sync(0xffffffffu, cur);
+        const uint32_t holders = __ballot_sync(0xffffffffu, cur == thr);
+        if (lane == __ffs(holders) - 1) cur = 0u;          // one holder leaves per round (0 sorts below every real value)
+    }
+    const float T = thr ? key_float(thr) : -INFINITY;    // fewer than k lanes hold anything: take everything
+    // collect the packed keys of all values >= T
+    unsigned long long *list = lists[wib];
+    int count = 0;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const int c = base + i * 32 + lane;
+        const bool hit = c < V && val[i] >= T;
+        const uint32_t hits = __ballot_sync(0xffffffffu, hit);
+        if (hits) {
+            const int at = count + __popc(hits & ((1u << lane) - 1u));
+            if (hit && at < CAP) list[at] = pack_val_id(val[i], c);
+            count += __popc(hits);
+        }
+    }
+    __syncwarp();
+    if (count <= CAP) {
+        // the k best of the few candidates (k rounds of a warp max over at most two keys per lane)
+        unsigned long long c0 = lane < count ? list[lane] : 0ull, c1 = lane + 32 < count ? list[lane + 32] : 0ull;
+        unsigned long long prev = ~0ull;
+        for (int t = 0; t < k; ++t) {
+            unsigned long long best = 0ull;
+            if (c0 < prev && c0 > best) best = c0;
+            if (c1 < prev && c1 > best) best = c1;
+            best = warp_max_u64(best);
+            if (lane == 0) out[t] = best;
+            prev = best;
+        }
+        return;
+    }
+    // many equal values at the threshold (ties): exact selection over the whole span
     unsigned long long prev = ~0ull;
     for (int t = 0; t < k; ++t) {
         unsigned long long best = 0ull;
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-            if (key[i] < prev && key[i] > best) best = key[i];
+        for (int i = 0; i < 32; ++i) {
+            const int c = base + i * 32 + lane;
+            const unsigned long long key = c < V ? pack_val_id(val[i], c) : 0ull;
+            if (key < prev && key > best) best = key;
+        }
         best = warp_max_u64(best);
-        if (lane == 0) cand[((size_t)row * n_warps + gw) * k + t] = best;
+        if (lane == 0) out[t] = best;
         prev = best;
     }
 }
 
-__global__ void __launch_bounds__(256) topk_stage2_kernel(int k, int n_warps, const unsigned long long *cand,
-                                                          const float *ml, int32_t *ids, float *lp) {
-    __shared__ unsigned long long sh[16];
-    __shared__ float shf[16];
-    const int row = blockIdx.x;
+// Stage 2: one warp per (sequence, offset).  The stage-1 lists are sorted, so the k-th largest of their heads is a
+// threshold that all of the row's k best keys reach; the few keys at or above it are collected and ranked.
+__global__ void __launch_bounds__(32) topk_stage2_kernel(int k, int n_warps, const unsigned long long *cand,
+                                                         const float *ml, int32_t *ids, float *lp) {
+    constexpr int CAP = 64;
+    __shared__ unsigned long long list[CAP];
+    const int row = blockIdx.x, lane = threadIdx.x;
     const float *rml = ml + (size_t)row * n_warps * 2;
-    float M = -INFINITY;
-    for (int w = threadIdx.x; w < n_warps; w += blockDim.x) M = fmaxf(M, rml[2 * w]);
-    M = warp_max(M);
-    if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = M;
-    __syncthreads();
-    M = shf[0];
-    for (int w = 1; w < 8; ++w) M = fmaxf(M, shf[w]);
-    __syncthreads();
-    // fixed-order sum: thread t adds warps t, t+256, ...; partial sums are then added in warp/lane order
-    float sum = 0.f;
-    for (int w = threadIdx.x; w < n_warps; w += blockDim.x) sum += rml[2 * w + 1] * expf(rml[2 * w] - M);
-    sum = warp_sum(sum);
-    if ((threadIdx.x & 31) == 0) shf[threadIdx.x >> 5] = sum;
-    __syncthreads();
-    sum = 0.f;
-    for (int w = 0; w < 8; ++w) sum += shf[w];
-    const float lse = M + logf(sum);
     const unsigned long long *rc = cand + (size_t)row * n_warps * k;
+    // log-sum-exp over the spans, fixed order: lane l adds spans l, l + 32, ...; lanes are then summed by shuffles
+    float M = -INFINITY;
+    for (int w = lane; w < n_warps; w += 32) M = fmaxf(M, rml[2 * w]);
+    M = warp_max(M);
+    float sum = 0.f;
+    for (int w = lane; w < n_warps; w += 32) sum += rml[2 * w + 1] * expf(rml[2 * w] - M);
+    sum = warp_sum(sum);
+    const float lse = M + logf(sum);
+    // threshold = k-th largest head (heads are unique keys); up to 8 heads per lane are held in registers
+    unsigned long long thr = ~0ull;
+    if (n_warps <= 256) {
+        unsigned long long h0 = 0, h1 = 0, h2 = 0, h3 = 0, h4 = 0, h5 = 0, h6 = 0, h7 = 0;
+        if (lane < n_warps) h0 = rc[(size_t)lane * k];
+        if (lane + 32 < n_warps) h1 = rc[(size_t)(lane + 32) * k];
+        if (lane + 64 < n_warps) h2 = rc[(size_t)(lane + 64) * k];
+        if (lane + 96 < n_warps) h3 = rc[(size_t)(lane + 96) * k];
+        if (lane + 128 < n_warps) h4 = rc[(size_t)(lane + 128) * k];
+        if (lane + 160 < n_warps) h5 = rc[(size_t)(lane + 160) * k];
+        if (lane + 192 < n_warps) h6 = rc[(size_t)(lane + 192) * k];
+        if (lane + 224 < n_warps) h7 = rc[(size_t)(lane + 224) * k];
+        for (int t = 0; t < k; ++t) {
+            unsigned long long best = 0ull;
+#define GLANCE_HEAD(h) if (h < thr && h > best) best = h;
+            GLANCE_HEAD(h0) GLANCE_HEAD(h1) GLANCE_HEAD(h2) GLANCE_HEAD(h3) GLANCE_HEAD(h4) GLANCE_HEAD(h5) GLANCE_HEAD(h6) GLANCE_HEAD(h7)
+#undef GLANCE_HEAD
+            thr = warp_max_u64(best);
+        }
+    } else {
+        for (int t = 0; t < k; ++t) {
+            unsigned long long best = 0ull;
+            for (int w = lane; w < n_warps; w += 32) {
+                const unsigned long long h = rc[(size_t)w * k];
+                if (h < thr && h > best) best = h;
+            }
+            thr = warp_max_u64(best);
+        }
+    }
+    // every key >= thr (thr == 0: fewer than k spans hold anything -- then every non-empty key qualifies)
     const int n = n_warps * k;
+    int count = 0;
+    for (int c0 = 0; c0 < n; c0 += 128) {
+        unsigned long long key4[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {                    // four independent loads in flight
+            const int c = c0 + u * 32 + lane;
+            key4[u] = c < n ? rc[c] : 0ull;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const bool hit = key4[u] != 0ull && key4[u] >= thr;
+            const uint32_t hits = __ballot_sync(0xffffffffu, hit);
+            if (hits) {
+                const int at = count + __popc(hits & ((1u << lane) - 1u));
+                if (hit && at < CAP) list[at] = key4[u];
+                count += __popc(hits);
+            }
+        }
+    }
+    __syncwarp();
     unsigned long long prev = ~0ull;
-    for (int t = 0; t < k; ++t) {
+    if (count <= CAP) {
+        const unsigned long long a0 = lane < count ? list[lane] : 0ull, a1 = lane + 32 < count ? list[lane + 32] : 0ull;
+        for (int t = 0; t < k; ++t) {
+            unsigned long long best = 0ull;
+            if (a0 < prev && a0 > best) best = a0;
+            if (a1 < prev && a1 > best) best = a1;
+            best = warp_max_u64(best);
+            if (lane == 0) {
+                ids[(size_t)row * k + t] = unpack_id(best);
+                lp[(size_t)row * k + t] = unpack_val(best) - lse;
+            }
+            prev = best;
+        }
+        return;
+    }
+    for (int t = 0; t < k; ++t) {                        // (not reached with unique keys; kept for safety)
         unsigned long long best = 0ull;
-        for (int c = threadIdx.x; c < n; c += blockDim.x) {
+        for (int c = lane; c < n; c += 32) {
             const unsigned long long key = rc[c];
             if (key < prev && key > best) best = key;
         }
-        best = block_max_u64(best, sh);
-        if (threadIdx.x == 0) {
+        best = warp_max_u64(best);
+        if (lane == 0) {
             ids[(size_t)row * k + t] = unpack_id(best);
             lp[(size_t)row * k + t] = unpack_val(best) - lse;
         }
@@ -308,7 +397,7 @@ void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *i
     const int rows = batch * (B - 1), nw = topk_warps(V);
     dim3 g1((nw + 3) / 4, rows);
     topk_stage1_kernel<<<g1, 128, 0, st>>>(logits, B, V, k, nw, cand, ml);
-    topk_stage2_kernel<<<rows, 256, 0, st>>>(k, nw, cand, ml, ids, lp);
+    topk_stage2_kernel<<<rows, 32, 0, st>>>(k, nw, cand, ml, ids, lp);
 }
 
 __global__ void prefill_advance_kernel(int32_t *seq_len, int32_t *root, int32_t *feat_count, const int32_t *argmax,
