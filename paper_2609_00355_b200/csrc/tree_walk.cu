@@ -27,6 +27,8 @@ __device__ __forceinline__ bool cand_before(const Cand &a, const Cand &b) {
 // redundantly (counts, the popped entry, the two new entries), so that a pop needs one hardware warp max over the
 // 32-bit score images, a handful of shuffles and no barrier: the only shared-memory traffic is the candidate
 // tables (read-only) and the node arrays (each written and later re-read by the same lane).
+// A pop replaces the entry by its child in place and appends its next sibling, so the frontier never exceeds N
+// entries and nothing is moved.
 // An entry is (sk, t, meta, ps): sk = order-preserving image of the score, t = tie word ((15 - depth) << 60 |
 // complemented 60-bit path key), meta = depth | rank << 4 | parent << 8, ps = the parent's score (a next-rank
 // sibling's score is one fp32 add from it).  Larger (sk, t) is popped first.
@@ -82,7 +84,8 @@ __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, con
         fc = 1;
     }
 
-    while (fc > 0 && nc < N) {
+    int live = fc;                                       // entries that are not empty slots
+    while (live > 0 && nc < N) {
         // this lane's best entry
         uint32_t bsk = 0u;
         unsigned long long bt = 0ull;
@@ -127,28 +130,19 @@ __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, con
             if ((i >> 6) == lane) aw |= 1ull << (i & 63);
             n_anc[i * W + lane] = aw;
         }
-        // the popped slot takes the last entry; the child and the next sibling are appended
-        const int bi = bu * 32 + wl, last = fc - 1;
-        if (bi != last) {
-            uint32_t lsk = 0u, lmeta = 0u;
-            unsigned long long lt = 0ull;
-            float lps = 0.f;
-#define GLANCE_LAST_OP(u, sk, tw, me, ps) if ((last >> 5) == u) { lsk = sk; lt = tw; lmeta = me; lps = ps; }
-            GLANCE_SLOTS(GLANCE_LAST_OP)
-            lsk = __shfl_sync(0xffffffffu, lsk, last & 31);
-            lt = __shfl_sync(0xffffffffu, lt, last & 31);
-            lmeta = __shfl_sync(0xffffffffu, lmeta, last & 31);
-            lps = __shfl_sync(0xffffffffu, lps, last & 31);
-            GLANCE_PUT(bi, lsk, lt, lmeta, lps);
-        }
-        fc = last;
+        // the child takes the popped entry's slot (or the slot goes empty: key 0 loses against every real entry); the
+        // next sibling is appended -- the frontier grows by at most one entry per pop and nothing has to be moved
+        const int bi = bu * 32 + wl;
         if (dpt < L) {
-            GLANCE_PUT(fc, float_key(__fadd_rn(sc, s_lp[dpt * k])), tie_word(dpt + 1, key), (uint32_t)(dpt + 1) | ((uint32_t)i << 8), sc);
-            ++fc;
+            GLANCE_PUT(bi, float_key(__fadd_rn(sc, s_lp[dpt * k])), tie_word(dpt + 1, key), (uint32_t)(dpt + 1) | ((uint32_t)i << 8), sc);
+        } else {
+            GLANCE_PUT(bi, 0u, 0ull, 0u, 0.f);
+            --live;
         }
         if (rk + 1 < k) {
             GLANCE_PUT(fc, float_key(__fadd_rn(bps, s_lp[(dpt - 1) * k + rk + 1])), tie_word(dpt, key + (1ull << (4 * (15 - dpt)))), (uint32_t)dpt | ((uint32_t)(rk + 1) << 4) | ((uint32_t)par << 8), bps);
             ++fc;
+            ++live;
         }
     }
 #undef GLANCE_SLOTS
@@ -156,7 +150,6 @@ __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, con
 #undef GLANCE_PUT
 #undef GLANCE_BEST_OP
 #undef GLANCE_META_OP
-#undef GLANCE_LAST_OP
     __syncwarp();
     if (lane == 0) out.n_nodes[s] = nc;
     int32_t *token = out.token + (size_t)s * N, *parent = out.parent + (size_t)s * N;
