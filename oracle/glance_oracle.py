@@ -18,7 +18,7 @@ Two groups of functions:
  (II) the round step by step, in the order of Algorithm 1
       prefill -> draft_block -> topk_logprobs -> build_tree -> verify_tree -> walk -> commit
 
-Readings of points the paper leaves open (each is restated in the design doc):
+Readings of points the paper leaves open:
   * the verify pass has N rows including the root; the paper's budget is N-1
   * horizon L = B-1; block slot 0 holds the root, slot j predicts offset j (no shift)
   * the one-layer head attends to [context features ; block] with one set of W_k/W_v;
