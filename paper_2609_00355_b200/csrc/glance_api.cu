@@ -17,15 +17,17 @@ namespace {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // split-K factor of a weight-streaming GEMM: as many CTAs as fit one wave at two CTAs per SM (one CTA per SM
-// keeps too few weight bytes in flight to cover the HBM latency), at least 8 k-tiles per split
+// keeps too few weight bytes in flight to cover the HBM latency), at least 7 k-tiles per split
 // The splits of one tile form a thread-block cluster (<= 8 CTAs) that reduces them through shared memory.
 int choose_split(int Nout, int K, int rows) {
     const int tiles = (Nout + 127) / 128;
     const int ktiles = K / 64;
     (void)rows;
     int s = (2 * 148) / tiles;
-    s = std::min(s, std::max(1, ktiles / 8));
-    return std::max(1, std::min(s, 8));
+    s = std::min(s, std::max(1, ktiles / 7));
+    s = std::max(1, std::min(s, 8));
+    if (s == 8 && tiles > 33) s = 7;                   // at most 33 clusters of eight are resident at two CTAs per SM
+    return s;
 }
 
 struct Workspace {
