@@ -500,17 +500,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             constexpr int SEG = D / 4;                    // 4-float segments per row
             for (int item = tsm; item < my_rows * SEG; item += NSOFT) {
                 const int lr = item / SEG, c0 = (item % SEG) * 4;
+                const float *rp0 = rows + (size_t)lr * ROWF;
+                const size_t sstride = (size_t)RPC * ROWF;      // floats between the same row of consecutive splits
+                // all loads first (the values of up to MAX_SPLITS splits), then the arithmetic
+                float ms[MAX_SPLITS], ls[MAX_SPLITS];
+                float4 vs[MAX_SPLITS];
                 float M = -INFINITY;
-                for (int sp = 0; sp < p.S; ++sp) M = fmaxf(M, rows[(size_t)(sp * RPC + lr) * ROWF + D]);
+#pragma unroll
+                for (int sp = 0; sp < MAX_SPLITS; ++sp) {
+                    ms[sp] = -INFINITY; ls[sp] = 0.f; vs[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (sp < p.S) {
+                        const float *rp = rp0 + sp * sstride;
+                        ms[sp] = rp[D];
+                        ls[sp] = rp[D + 1];
+                        vs[sp] = *reinterpret_cast<const float4 *>(rp + c0);
+                        M = fmaxf(M, ms[sp]);
+                    }
+                }
                 float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                 float den = 0.f;
-                for (int sp = 0; sp < p.S; ++sp) {        // split order: bit-reproducible
-                    const float *rp = rows + (size_t)(sp * RPC + lr) * ROWF;
-                    const float ms = rp[D];
-                    const float w = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
-                    den += w * rp[D + 1];
-                    const float4 v = *reinterpret_cast<const float4 *>(rp + c0);
-                    acc.x += w * v.x; acc.y += w * v.y; acc.z += w * v.z; acc.w += w * v.w;
+#pragma unroll
+                for (int sp = 0; sp < MAX_SPLITS; ++sp) {  // split order: bit-reproducible
+                    const float w = ex2_approx(ms[sp] - M);    // 2^-inf = 0 for an empty split
+                    den += w * ls[sp];
+                    acc.x += w * vs[sp].x; acc.y += w * vs[sp].y; acc.z += w * vs[sp].z; acc.w += w * vs[sp].w;
                 }
                 const float inv = 1.f / den;
                 const int prr = qt * QT + row_lo + lr;
