@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        mbar_init(&bars.q_ready, NSOFT);
+        mbar_init(&bars.q_ready, NSOFT / 32);            // one arrival per softmax warp
         for (int b = 0; b < KS; ++b) {
             mbar_init(&bars.k_full[b], 1);
             mbar_init(&bars.k_empty[b], 1);
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             mbar_init(&bars.s_full[b], 1);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&bars.p_full[b], NSOFT);
+            mbar_init(&bars.p_full[b], NSOFT / 32);
             mbar_init(&bars.o_done[b], 1);
         }
         mbar_init(&bars.merge, 1);
@@ -277,7 +277,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         asm volatile("cp.async.commit_group;" ::);
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         fence_async_smem();
-        mbar_arrive(&bars.q_ready);
+        __syncwarp();                                     // every lane's rows are written and fenced: one arrival per warp
+        if (lane == 0) mbar_arrive(&bars.q_ready);
         if (trace && threadIdx.x == 64) trace[3] = global_ns();
 
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
@@ -400,7 +401,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             l_run += rs;
             fence_async_smem();
             tc_fence_before();
-            mbar_arrive(&bars.p_full[st]);                // always arrive: the MMA issuer counts 512 arrivals
+            __syncwarp();                                 // 512 single arrivals would serialise on the barrier word
+            if (lane == 0) mbar_arrive(&bars.p_full[st]);  // always arrive: the MMA issuer counts one arrival per warp
             if (trace && threadIdx.x == 64 && i == 0) trace[5] = global_ns();
         }
         if (trace && threadIdx.x == 64) trace[6] = global_ns();
