@@ -36,7 +36,9 @@ __device__ __forceinline__ float ex2_approx(float x) {   // 2^x, hardware approx
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-constexpr int NSOFT = 512;       // softmax / epilogue threads (16 warps)
+constexpr int NCG = 4;           // column groups: threads per query row (a row's 64 scores and d outputs are split over them)
+constexpr int KPT = KT / NCG;    // keys per thread and tile
+constexpr int NSOFT = 128 * NCG; // softmax / epilogue threads
 constexpr int NTHREADS = 64 + NSOFT;
 
 template <int D>
@@ -70,7 +72,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     unsigned char *sV = sK + KS * Smem<D>::KV_BYTES;                 // 2 stages
     unsigned char *sP = sV + 2 * Smem<D>::KV_BYTES;
     __shared__ AttnBars bars;
-    __shared__ float red[2][4][QT];                       // cross-column-group exchange of row maxima / sums
+    __shared__ float red[2][NCG][QT];                       // cross-column-group exchange of row maxima / sums
     __shared__ int quit[2][4];                            // per lane quarter: leave the tile loop (decided by one thread)
 
     unsigned long long *trace = (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? p.trace : nullptr;
@@ -253,7 +255,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         // 16 warps: warp (q, cg) serves the TMEM lane quarter q (32 query rows) and the column group cg;
         // a row's 64 scores are split over four threads (16 keys each), its d output columns likewise.
         const int q = warp & 3;                           // TMEM lane quarter this warp may access
-        const int cg = (warp - 2) >> 2;                   // column group 0..3
+        const int cg = (warp - 2) >> 2;                   // column group 0..NCG-1
         const int row = q * 32 + lane;
         const int tsm = threadIdx.x - 64;                 // 0..511
         int pr = qt * QT + row;
@@ -283,7 +285,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;
-        constexpr int OC = D / 4;                         // output columns per thread
+        constexpr int OC = D / NCG;                       // output columns per thread
         float m_ref = -INFINITY, l_run = 0.f;             // l_run: this thread's share of the row sum
         bool ok = true;
         for (int i = 0; i < nt; ++i) {
@@ -307,26 +309,27 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are warp-collective
             if (trace && threadIdx.x == 64 && i == 0) trace[4] = global_ns();
             tc_fence_after();
-            float sc[16];
-            {
+            float sc[KPT];
+#pragma unroll
+            for (int c = 0; c < KPT; c += 16) {
                 uint32_t v[16];
                 if (ok) {
-                    tmem_ld16(tmem_S + lane_addr + (uint32_t)(st * 64 + cg * 16), v);
+                    tmem_ld16(tmem_S + lane_addr + (uint32_t)(st * 64 + cg * KPT + c), v);
                     tmem_ld_wait();
                 } else {
 #pragma unroll
                     for (int j = 0; j < 16; ++j) v[j] = 0u;
                 }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) sc[j] = __uint_as_float(v[j]);
+                for (int j = 0; j < 16; ++j) sc[c + j] = __uint_as_float(v[j]);
             }
             const bool need_mask = key0 + KT > P;
             float mt = -INFINITY;
 #pragma unroll
-            for (int j = 0; j < 16; ++j) {
+            for (int j = 0; j < KPT; ++j) {
                 float v = sc[j];                          // raw score: the scale is folded into the exponent below
                 if (need_mask) {
-                    const int key = key0 + cg * 16 + j;
+                    const int key = key0 + cg * KPT + j;
                     bool vis = key < P;
                     if (!vis && key < n_keys) {
                         const int b = key - P;
@@ -344,9 +347,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             // Leaving the loop must be decided once per quarter: its four warps meet at the barrier below every tile,
             // and the abort flag can change between two warps' reads.  One thread samples it before the barrier.
             if (cg == 0 && lane == 0) quit[i & 1][q] = *abort_flag;
-            asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");   // only the four warps of this lane quarter share rows
+            asm volatile("bar.sync %0, %1;" ::"r"(2 + q), "n"(32 * NCG) : "memory");   // only the warps of this lane quarter share rows
             if (quit[i & 1][q]) break;                    // a quarter that leaves stops arriving at p_full: every wait is bounded
-            mt = fmaxf(fmaxf(red[i & 1][0][row], red[i & 1][1][row]), fmaxf(red[i & 1][2][row], red[i & 1][3][row]));
+            mt = red[i & 1][0][row];
+#pragma unroll
+            for (int c = 1; c < NCG; ++c) mt = fmaxf(mt, red[i & 1][c][row]);
             if (i > 1) {
                 // this tile's P buffer was read by the second MMA of tile i-2
                 ok = ok && mbar_wait(&bars.o_done[st], (uint32_t)((i - 2) >> 1) & 1u, abort_flag, p.status);
@@ -385,7 +390,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             unsigned char *prow = sP + st * Smem<D>::P_BYTES + row * 128;
             const float m_sub = (m_ref == -INFINITY) ? 0.f : m_ref;   // a fully masked row keeps -inf - 0 = -inf -> 2^-inf = 0
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < KPT / 8; ++c) {
                 uint32_t w[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
@@ -396,7 +401,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
                     w[j] = *reinterpret_cast<uint32_t *>(&h2);
                 }
-                *reinterpret_cast<uint4 *>(prow + (((cg * 2 + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4 *>(prow + (((cg * (KPT / 8) + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
             }
             l_run += rs;
             fence_async_smem();
@@ -412,10 +417,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             tc_fence_after();
         }
         // row sums across the four column groups (fixed order)
-        asm volatile("bar.sync 1, 512;" ::: "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
         red[0][cg][row] = l_run;
-        asm volatile("bar.sync 1, 512;" ::: "memory");
-        const float l_row = ((red[0][0][row] + red[0][1][row]) + red[0][2][row]) + red[0][3][row];
+        asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
+        float l_row = red[0][0][row];
+#pragma unroll
+        for (int c = 1; c < NCG; ++c) l_row += red[0][c][row];
         ok = ok && (*abort_flag == 0);
         // ---------------- epilogue ----------------
         if (p.S == 1 && ok) {
@@ -448,7 +455,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         // asynchronous shared-to-shared copy per owner ships that owner's band into the owner's receive region
         // and counts its bytes on the owner's merge barrier; the owner combines the S bands in split order.
         constexpr int ROWF = Smem<D>::ROWF;
-        constexpr int OC = D / 4;
+        constexpr int OC = D / NCG;
         const int RPC = (QT + p.S - 1) / p.S;
         const uint32_t rank = cluster_rank();
         float *stage = reinterpret_cast<float *>(smem);
@@ -480,7 +487,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 stage[(size_t)row * ROWF + D + 1] = live ? sm_l : 0.f;
             }
             fence_async_smem();                           // staged rows visible to the asynchronous copy engine
-            asm volatile("bar.sync 1, 512;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
             if (trace && threadIdx.x == 64) trace[8] = global_ns();
             if (warp == 2 && lane < p.S) {
                 const uint32_t owner = (uint32_t)lane;
