@@ -513,3 +513,15 @@ def test_rounds_extreme_block_topk_budget(harness, block_B, topk, tree_N):
         run.round(p_m=(0.7 if r else None), check_draft=(r == 0))
     run.check_head_state()
     assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_rounds_batch2_sampling_two_layer_head(harness):
+    """Everything at once on two ragged sequences: sampling walk, two-layer two-tap head, root-entropy log."""
+    cfg = synth.CONFIGS["tiny"].replace(tree_N=16, block_B=6, topk=3, head_taps=(0, 1))
+    run = harness.ParityRun(cfg, batch=2, ctx_lens=[(70, 19), (140, 33)])
+    run.check_state()
+    for r in range(5):
+        run.round(p_m=(0.75 if r % 2 else None), check_draft=(r == 0), sample_seed=77)
+    run.check_head_state()
+    print("batch-2 sampling parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
