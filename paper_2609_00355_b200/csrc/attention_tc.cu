@@ -4,15 +4,20 @@
 // One CTA = (128 packed query rows of one kv head, one key split).  The G query heads that share a kv
 // head are packed into the row dimension (packed row = node * G + g), so each K/V page is fetched once
 // per CTA for all of them.  Per 64-key tile (= one KV page, TMA-loaded with 128-byte swizzle):
-//     S[128 x 64]  = Q K^T          tcgen05.mma, A = Q (K-major), B = K page (K-major), accumulator in TMEM
-//     P            = 2^(S' - m)     softmax warps read S from TMEM (four threads per row), apply the scale and
-//                                   the ancestor mask, write bf16 P into shared memory
-//     O[128 x d]  += P V            tcgen05.mma, A = P (K-major), B = V page (MN-major), accumulator in TMEM
+//     S[128 x 64]  = Q K^T          tcgen05.mma, A = Q (K-major, two bf16 terms hi + lo: the rounding of a query
+//                                   would otherwise reach every score of its row), B = K page (K-major),
+//                                   accumulator in TMEM
+//     P            = 2^(S' - m)     softmax warps read S from TMEM (two threads per row), apply the scale and
+//                                   the ancestor mask, write bf16 P back into TMEM over the scores
+//     O[128 x d]  += P V            tcgen05.mma, A = P in tensor memory, B = V page (MN-major), accumulator in TMEM
 // The running reference maximum m of a row is only raised when a tile exceeds it by more than 2^8 (the
 // accumulator is then rescaled in TMEM), so exponentials stay far inside fp32/bf16 range and O is almost
 // never touched between tiles.  Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
-// warps 2..17 = softmax / epilogue (a row's scores and outputs are split over four threads).  S and P are
-// double-buffered, so the next tile's scores and probabilities are produced while the previous P V runs.
+// warps 2..17 = softmax / epilogue.  The softmax warps form two groups: one takes the CTA's even key tiles, the
+// other the odd ones, each with two S/P buffers, its own running maximum, row sums and accumulator in TMEM.  The
+// scores of a group's next tile are issued a tile ahead into its other buffer, so a group goes from one tile
+// straight to the next, and one group's exponentials run while the tensor pipe works for the other; the two
+// accumulators are combined like two key splits when the loop ends.
 // The key splits of a tile form a thread-block cluster and are merged through distributed shared memory
 // (one asynchronous bulk copy per owner CTA, byte-counted on the owner's mbarrier).  Every mbarrier wait is
 // bounded; a wait that gives up records GLANCE_E_TIMEOUT.
@@ -27,7 +32,8 @@ using namespace tc;
 
 constexpr int QT = 128;          // packed query rows per CTA (UMMA M)
 constexpr int KT = kPage;        // keys per tile (UMMA N of S, K of P V)
-constexpr int KS = 3;             // K page ring (one deeper than V's: the next scores are issued a tile ahead)
+constexpr int KS = 3;             // K page ring: scores are issued tiles ahead, so a K slot frees soon after its page lands
+constexpr int VS = 2;             // V page ring: a V slot is held from the copy until the tile's second MMA
 constexpr int MAX_SPLITS = 8;     // the splits of a tile form one thread-block cluster
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 
@@ -36,27 +42,53 @@ __device__ __forceinline__ float ex2_approx(float x) {   // 2^x, hardware approx
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-constexpr int NCG = 4;           // column groups: threads per query row (a row's 64 scores and d outputs are split over them)
+constexpr int NG = 2;            // softmax groups (tile i belongs to group i % NG; S, P and O buffers are per group)
+constexpr int NCG = 2;           // column groups of a softmax group: threads per query row (a row's 64 scores are split over them)
 constexpr int KPT = KT / NCG;    // keys per thread and tile
-constexpr int NSOFT = 128 * NCG; // softmax / epilogue threads
+constexpr int GTHREADS = 128 * NCG;      // threads of one softmax group
+constexpr int NSOFT = NG * GTHREADS;     // softmax / epilogue threads
+constexpr int ECG = NSOFT / 128;         // column groups of the epilogue: a row's d outputs are split over them
 constexpr int NTHREADS = 64 + NSOFT;
+static_assert(NG == 2, "buffers are indexed by tile parity");
+static_assert(KPT == 32, "the visibility bit set of a thread's keys is one 32-bit word");
+static_assert(KPT % 32 == 0, "a thread writes its probabilities as 16-column chunks of bf16 pairs");
+
+// 16 accumulator columns of a row, combined over the softmax groups: sum_g w[g] * O_g.  Warp-collective.  Only the
+// first `groups` accumulators are read (a group without tiles never wrote its TMEM columns).
+__device__ __forceinline__ void load_combined(uint32_t tmem_O, uint32_t addr, int d, int groups, const float (&w)[NG], float (&out)[16]) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) out[j] = 0.f;
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi) {
+        if (gi < groups) {
+            uint32_t v[16];
+            tmem_ld16(tmem_O + (uint32_t)(gi * d) + addr, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j) out[j] = fmaf(w[gi], __uint_as_float(v[j]), out[j]);
+        }
+    }
+}
 
 template <int D>
 struct Smem {
     static constexpr int SLABS = D / 64;                 // 64-element (128-byte) column slabs of a d-wide tile
-    static constexpr int Q_BYTES = SLABS * QT * 128;     // 32 KB at d = 128
     static constexpr int KV_BYTES = SLABS * KT * 128;    // one K or V page: 16 KB at d = 128
-    static constexpr int P_BYTES = QT * 128;             // 128 rows x 64 keys bf16
-    static constexpr int OPER_BYTES = Q_BYTES + (KS + 2) * KV_BYTES + 2 * P_BYTES;   // P is double-buffered;   // operand buffers (and merge staging)
+    static constexpr int Q_BYTES = 2 * SLABS * QT * 128; // both query planes: 64 KB at d = 128
+    static constexpr int OPER_BYTES = Q_BYTES + (KS + VS) * KV_BYTES;   // Q, K ring, V ring (and merge staging)
     static constexpr int ROWF = D + 4;                   // floats per merged row: O, m, l, padding
     // split merge: rows received from the cluster's CTAs (each owner gets <= ceil(QT/S) rows from each of S CTAs)
     static constexpr int RECV_BYTES = (QT + MAX_SPLITS) * ROWF * 4;
     static constexpr int TOTAL = OPER_BYTES + RECV_BYTES + 1024;
-    static constexpr uint32_t TMEM_COLS = 256;           // two S buffers (2 x 64) + O (d)
+    // tensor memory columns: two S buffers per group (4 x 64; P overwrites the first half of its S), one O (d) per group
+    static constexpr uint32_t O_COL = 2 * NG * 64;
+    static constexpr uint32_t TMEM_COLS = 512;
+    static_assert(O_COL + NG * D <= TMEM_COLS, "tensor memory budget");
+    static_assert(ROWF * 4 * QT <= OPER_BYTES, "merge staging fits the operand buffers");
 };
 
 struct alignas(8) AttnBars {
-    uint64_t q_ready, k_full[KS], k_empty[KS], v_full[2], v_empty[2], s_full[2], p_full[2], o_done[2], merge;
+    uint64_t q_ready, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS], s_full[2 * NG], p_full[2 * NG], o_done[NG], all_done, v_zero, merge;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -67,13 +99,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     constexpr int CH = D / 8;                            // 16-byte chunks per row
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    unsigned char *sQ = smem;
+    unsigned char *sQ = smem;                                        // hi plane, lo plane
     unsigned char *sK = sQ + Smem<D>::Q_BYTES;                       // KS stages
-    unsigned char *sV = sK + KS * Smem<D>::KV_BYTES;                 // 2 stages
-    unsigned char *sP = sV + 2 * Smem<D>::KV_BYTES;
+    unsigned char *sV = sK + KS * Smem<D>::KV_BYTES;                 // VS stages
     __shared__ AttnBars bars;
-    __shared__ float red[2][NCG][QT];                       // cross-column-group exchange of row maxima / sums
-    __shared__ int quit[2][4];                            // per lane quarter: leave the tile loop (decided by one thread)
+    __shared__ float red[NG][2][NCG][QT];                 // per group: cross-column-group exchange of row maxima / sums
+    __shared__ int quit[NG][2][4];                        // per group and lane quarter: leave the tile loop (decided by one thread)
 
     unsigned long long *trace = (p.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? p.trace : nullptr;
     if (trace && threadIdx.x == 0) trace[0] = global_ns();
@@ -91,15 +122,17 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             mbar_init(&bars.k_full[b], 1);
             mbar_init(&bars.k_empty[b], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < VS; ++b) {
             mbar_init(&bars.v_full[b], 1);
             mbar_init(&bars.v_empty[b], 1);
+        }
+        for (int b = 0; b < 2 * NG; ++b) {
             mbar_init(&bars.s_full[b], 1);
+            mbar_init(&bars.p_full[b], GTHREADS / 32);   // one arrival per warp of the buffer's group
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&bars.p_full[b], NSOFT / 32);
-            mbar_init(&bars.o_done[b], 1);
-        }
+        for (int b = 0; b < NG; ++b) mbar_init(&bars.o_done[b], 1);
+        mbar_init(&bars.all_done, 1);
+        mbar_init(&bars.v_zero, 1);
         mbar_init(&bars.merge, 1);
         bars.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -118,10 +151,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     if (p.S > 1) cluster_sync_all();                     // peers' merge barriers exist before anybody can signal them
     else __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_S = bars.tmem_base, tmem_O = bars.tmem_base + 128;   // S is double-buffered: columns 0-63, 64-127
+    // S / P buffer of tile i: columns 64 (i & 3) (its parity is the group); O of group g: O_COL + d g
+    const uint32_t tmem_S = bars.tmem_base, tmem_O = bars.tmem_base + Smem<D>::O_COL;
     volatile int *abort_flag = &bars.abort_flag;
     bool sm_ok = true;                                   // softmax warps: state carried into the split merge
     float sm_m = -INFINITY, sm_l = 0.f;
+    float sm_w[NG] = {0.f, 0.f};                         // weights of the groups' accumulators in the combined row
 
     if (trace && threadIdx.x == 0) trace[1] = global_ns();
     // Sequence lengths and page tables only change in the commit kernel of the previous round, long finished:
@@ -142,7 +177,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     }
 
     if (warp == 0) {
-        // ---------------- TMA producer: K pages and V pages in separate two-slot rings ----------------
+        // ---------------- TMA producer: K pages and V pages in separate rings ----------------
+        int issued_k = 0, issued_v = 0;
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&map_kv) : "memory");
             bool waited = false;
@@ -163,40 +199,70 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 krow = ((page * 2 + 0) * p.geom.n_kv_heads + kvh) * KT;
                 vrow = ((page * 2 + 1) * p.geom.n_kv_heads + kvh) * KT;
             };
-            int issued_k = 0, issued_v = 0;
-            auto issue_k = [&](int i) -> bool {
-                int krow, vrow;
-                page_rows(i, krow, vrow);
-                const int st = i % KS;
-                if (!mbar_wait(&bars.k_empty[st], ((uint32_t)(i / KS) & 1u) ^ 1u, abort_flag, p.status)) return false;
-                mbar_expect_tx(&bars.k_full[st], (uint32_t)Smem<D>::KV_BYTES);
+            // K and V pages advance independently, each as far ahead as its ring allows: one thread polls both rings
+            uint64_t stall_t0 = 0;
+            uint32_t spins = 0;
+            while (issued_k < nt || issued_v < nt) {
+                bool progressed = false;
+                if (issued_k < nt && mbar_try_wait(&bars.k_empty[issued_k % KS], ((uint32_t)(issued_k / KS) & 1u) ^ 1u)) {
+                    int krow, vrow;
+                    page_rows(issued_k, krow, vrow);
+                    const int slot = issued_k % KS;
+                    mbar_expect_tx(&bars.k_full[slot], (uint32_t)Smem<D>::KV_BYTES);
 #pragma unroll
-                for (int sl = 0; sl < SLABS; ++sl)
-                    tma_load_2d(sK + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.k_full[st], sl * 64, krow);
-                issued_k = i + 1;
-                return true;
-            };
-            auto issue_v = [&](int i) -> bool {
-                int krow, vrow;
-                page_rows(i, krow, vrow);
-                const int st = i & 1;
-                if (!mbar_wait(&bars.v_empty[st], ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_flag, p.status)) return false;
-                mbar_expect_tx(&bars.v_full[st], (uint32_t)Smem<D>::KV_BYTES);
+                    for (int sl = 0; sl < SLABS; ++sl)
+                        tma_load_2d(sK + slot * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.k_full[slot], sl * 64, krow);
+                    ++issued_k;
+                    progressed = true;
+                }
+                if (issued_v < nt && mbar_try_wait(&bars.v_empty[issued_v % VS], ((uint32_t)(issued_v / VS) & 1u) ^ 1u)) {
+                    int krow, vrow;
+                    page_rows(issued_v, krow, vrow);
+                    const int slot = issued_v % VS;
+                    mbar_expect_tx(&bars.v_full[slot], (uint32_t)Smem<D>::KV_BYTES);
 #pragma unroll
-                for (int sl = 0; sl < SLABS; ++sl)
-                    tma_load_2d(sV + st * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.v_full[st], sl * 64, vrow);
-                issued_v = i + 1;
-                return true;
-            };
-            // K pages run KS - 1 tiles ahead of V pages: the scores of tile i + 1 are issued before P V of tile i,
-            // and a V slot only frees when P V of two tiles back has finished
-            bool pok = true;
-            for (int i = 0; i < KS - 1 && i < nt && pok; ++i) pok = issue_k(i);
-            for (int i = 0; i < nt && pok; ++i) {
-                if (i + KS - 1 < nt) pok = issue_k(i + KS - 1);
-                pok = pok && issue_v(i);
+                    for (int sl = 0; sl < SLABS; ++sl)
+                        tma_load_2d(sV + slot * Smem<D>::KV_BYTES + sl * KT * 128, &map_kv, &bars.v_full[slot], sl * 64, vrow);
+                    ++issued_v;
+                    progressed = true;
+                }
+                if (progressed) {
+                    stall_t0 = 0;
+                } else if ((++spins & 63u) == 0) {
+                    // bounded: no slot of either ring has come free for the whole limit, or another role gave up
+                    if (*abort_flag) break;
+                    const uint64_t now = global_ns();
+                    if (stall_t0 == 0) stall_t0 = now;
+                    else if (now - stall_t0 > kWaitLimitNs) {
+                        *abort_flag = 1;
+                        set_status(p.status, GLANCE_E_TIMEOUT);
+                        break;
+                    }
+                }
             }
             if (!waited) pdl_wait();
+        }
+        // The page that holds the last key may continue with rows that belong to nobody (any bits, NaN included):
+        // this warp zeroes them in the V slot once the page has landed, and tells the MMA issuer.  The wait is exact:
+        // this thread issued the copy, and no later copy can follow into the slot before that tile's second MMA.
+        const int last_valid = n_keys - (t_end - 1) * KT;       // keys of this CTA's last tile
+        if (nt > 0 && last_valid < KT) {
+            const int i = nt - 1, slot = i % VS;
+            int got = 0;
+            if (lane == 0) got = (issued_v == nt && mbar_wait(&bars.v_full[slot], (uint32_t)(i / VS) & 1u, abort_flag, p.status)) ? 1 : 0;
+            got = __shfl_sync(0xffffffffu, got, 0);
+            if (got) {
+                unsigned char *v = sV + slot * Smem<D>::KV_BYTES;
+                for (int it = lane; it < (KT - last_valid) * CH; it += 32) {
+                    const int r = last_valid + it / CH, c = it % CH;
+                    *reinterpret_cast<int4 *>(v + (c >> 3) * KT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = make_int4(0, 0, 0, 0);
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&bars.v_zero);
+            }
+        }
+        if (lane == 0) {
             if (*abort_flag) {
                 // copies already issued must land before the CTA may exit
                 for (int i = max(0, issued_k - KS); i < issued_k; ++i) {
@@ -204,77 +270,91 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     while (!mbar_try_wait(&bars.k_full[i % KS], (uint32_t)(i / KS) & 1u))
                         if (global_ns() - t0 > kWaitLimitNs) break;
                 }
-                for (int i = max(0, issued_v - 2); i < issued_v; ++i) {
+                for (int i = max(0, issued_v - VS); i < issued_v; ++i) {
                     const uint64_t t0 = global_ns();
-                    while (!mbar_try_wait(&bars.v_full[i & 1], (uint32_t)(i >> 1) & 1u))
+                    while (!mbar_try_wait(&bars.v_full[i % VS], (uint32_t)(i / VS) & 1u))
                         if (global_ns() - t0 > kWaitLimitNs) break;
                 }
             }
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        // S = Q K^T of tile i+1 is issued before P V of tile i, into the other S buffer, so that the softmax
-        // warps find the next scores ready when they finish a tile.
+        // Tile i uses S / P buffer i & 3 (so a group alternates between its two buffers) and the accumulator of
+        // group i & 1.  The scores of the first four tiles are issued up front; after P V of tile i the scores of
+        // tile i + 4 follow into the buffer that P V has just read.
         if (lane == 0 && nt > 0) {
             const uint32_t idesc_s = umma_idesc(KT);              // M 128, N 64 keys
             const uint32_t idesc_o = umma_idesc_bmn(D);           // M 128, N d, B = V is MN-major
+            const int planes = p.q_lo ? 2 : 1;
             auto issue_s = [&](int i) -> bool {
-                const int st = i & 1, ks_slot = i % KS;   // S buffer in TMEM / K page slot in shared memory
+                const int b = i & 3, ks_slot = i % KS;    // S buffer in TMEM / K page slot in shared memory
                 if (!mbar_wait(&bars.k_full[ks_slot], (uint32_t)(i / KS) & 1u, abort_flag, p.status)) return false;
                 tc_fence_after();
                 const uint32_t kbase = smem_u32(sK + ks_slot * Smem<D>::KV_BYTES);
+                for (int pl = 0; pl < planes; ++pl) {
+                    const uint32_t qbase = smem_u32(sQ) + (uint32_t)(pl * SLABS * QT * 128);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const int sl = ks >> 2, kk = ks & 3;
-                    umma_f16(tmem_S + (uint32_t)(st * 64), umma_desc(smem_u32(sQ) + sl * QT * 128) + (uint64_t)(kk * 2),
-                             umma_desc(kbase + sl * KT * 128) + (uint64_t)(kk * 2), idesc_s, ks > 0 ? 1u : 0u);
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const int sl = ks >> 2, kk = ks & 3;
+                        umma_f16(tmem_S + (uint32_t)(b * 64), umma_desc(qbase + sl * QT * 128) + (uint64_t)(kk * 2),
+                                 umma_desc(kbase + sl * KT * 128) + (uint64_t)(kk * 2), idesc_s, (pl | ks) > 0 ? 1u : 0u);
+                    }
                 }
                 umma_commit(&bars.k_empty[ks_slot]);      // K page free once these MMAs have read it
-                umma_commit(&bars.s_full[st]);
+                umma_commit(&bars.s_full[b]);
                 return true;
             };
             bool ok = mbar_wait(&bars.q_ready, 0, abort_flag, p.status);
-            ok = ok && issue_s(0);
+            for (int i = 0; i < 2 * NG && i < nt && ok; ++i) ok = issue_s(i);
             for (int i = 0; i < nt && ok; ++i) {
-                const int st = i & 1;
-                if (i + 1 < nt && !issue_s(i + 1)) { ok = false; break; }
-                if (!mbar_wait(&bars.p_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-                if (!mbar_wait(&bars.v_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+                const int b = i & 3, g = i & 1, vs = i % VS;
+                if (!mbar_wait(&bars.p_full[b], (uint32_t)(i >> 2) & 1u, abort_flag, p.status)) { ok = false; break; }
+                if (!mbar_wait(&bars.v_full[vs], (uint32_t)(i / VS) & 1u, abort_flag, p.status)) { ok = false; break; }
+                // the rows after the last key have been zeroed by the producer warp
+                if (i == nt - 1 && n_keys - (t_end - 1) * KT < KT && !mbar_wait(&bars.v_zero, 0, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t vbase = smem_u32(sV + st * Smem<D>::KV_BYTES);
+                const uint32_t vbase = smem_u32(sV + vs * Smem<D>::KV_BYTES);
 #pragma unroll
                 for (int kk = 0; kk < KT / 16; ++kk)
-                    umma_f16(tmem_O, umma_desc(smem_u32(sP) + st * Smem<D>::P_BYTES) + (uint64_t)(kk * 2), umma_desc_mn(vbase + kk * 16 * 128, KT * 128),
-                             idesc_o, (i > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(&bars.v_empty[st]);           // V page free once these MMAs have read it
-                umma_commit(&bars.o_done[st]);            // this P buffer free, O updated
+                    umma_f16_ts(tmem_O + (uint32_t)(g * D), tmem_S + (uint32_t)(b * 64 + kk * 8),
+                                umma_desc_mn(vbase + kk * 16 * 128, KT * 128), idesc_o, (i >= NG || kk > 0) ? 1u : 0u);
+                umma_commit(&bars.v_empty[vs]);           // V page free once these MMAs have read it
+                umma_commit(&bars.o_done[g]);             // this group's O updated
+                if (i + 2 * NG < nt && !issue_s(i + 2 * NG)) { ok = false; break; }
             }
+            if (ok) umma_commit(&bars.all_done);         // every MMA of this CTA has completed when this barrier flips
         }
     } else {
         // ---------------- softmax / epilogue warps ----------------
-        // 16 warps: warp (q, cg) serves the TMEM lane quarter q (32 query rows) and the column group cg;
-        // a row's 64 scores are split over four threads (16 keys each), its d output columns likewise.
+        // 16 warps in two groups of 8.  Inside a group warp (q, cg) serves the TMEM lane quarter q (32 query rows)
+        // and the column group cg: a row's 64 scores are split over NCG threads.  In the epilogue all 16 warps
+        // split a row's d output columns four ways.
         const int q = warp & 3;                           // TMEM lane quarter this warp may access
-        const int cg = (warp - 2) >> 2;                   // column group 0..NCG-1
+        const int sw = warp - 2;                          // 0..15
+        const int grp = sw / (4 * NCG);                   // softmax group: takes tiles i with i % NG == grp
+        const int cg = (sw % (4 * NCG)) >> 2;             // column group inside the softmax group
+        const int ecg = sw >> 2;                          // column group of the epilogue, 0..ECG-1
         const int row = q * 32 + lane;
-        const int tsm = threadIdx.x - 64;                 // 0..511
+        const int tsm = threadIdx.x - 64;                 // 0..NSOFT-1
         int pr = qt * QT + row;
         const bool row_valid = pr < PR;
         if (!row_valid) pr = PR - 1;
         const int node = pr / G, g = pr % G;
-        uint64_t anc0 = 0, anc1 = 0;
+        uint64_t anc0 = ~0ull, anc1 = ~0ull;               // no mask: every extra key is visible
         if (p.anc) {
             const uint64_t *a = p.anc + ((size_t)s * p.T + node) * p.W;
             anc0 = a[0];
             anc1 = p.W > 1 ? a[1] : 0ull;
         }
-        // Q tile -> shared memory in the K-major 128-byte-swizzled operand layout (async copies, all in flight)
-        for (int it = tsm; it < QT * CH; it += NSOFT) {
-            const int r = it / CH, c = it % CH;
+        // Q tile (both planes) -> shared memory in the K-major 128-byte-swizzled operand layout (async copies, all in flight)
+        for (int it = tsm; it < 2 * QT * CH; it += NSOFT) {
+            const int pl = it / (QT * CH), r = (it / CH) % QT, c = it % CH;
             int prr = qt * QT + r;
             if (prr >= PR) prr = PR - 1;
-            const bf16 *src = p.q + ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c * 8;
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(sQ + (c >> 3) * QT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4))), "l"(src));
+            const bf16 *src = pl == 0 ? p.q : p.q_lo;
+            if (src)
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(sQ + pl * SLABS * QT * 128 + (c >> 3) * QT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4))),
+                             "l"(src + ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c * 8));
         }
         asm volatile("cp.async.commit_group;" ::);
         asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -285,78 +365,68 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
 
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const float sl2 = rsqrtf((float)D) * 1.4426950408889634f;
-        constexpr int OC = D / NCG;                       // output columns per thread
-        float m_ref = -INFINITY, l_run = 0.f;             // l_run: this thread's share of the row sum
+        const uint32_t tmem_Og = tmem_O + (uint32_t)(grp * D);   // this group's accumulator
+        const int st = grp;                               // V slot and accumulator barrier of every tile of this group
+        float m_ref = -INFINITY, l_run = 0.f;             // l_run: this thread's share of the group's row sum
         bool ok = true;
-        for (int i = 0; i < nt; ++i) {
+        for (int i = grp; i < nt; i += NG) {
             const int t = t_begin + i;
-            const int st = i & 1;
+            const int u = i >> 1;                         // this group's tile count so far
+            const int sb = i & 3;                         // S / P buffer of the tile
+            const uint32_t sph = (uint32_t)(i >> 2) & 1u; // phase of that buffer's barriers
             const int key0 = t * KT;
-            const int valid_keys = min(KT, n_keys - key0);
-            if (valid_keys < KT) {
-                // rows of the page beyond the last key may hold anything (NaN bits included): zero them in V
-                ok = ok && mbar_wait(&bars.v_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status);
-                if (ok) {
-                    unsigned char *v = sV + st * Smem<D>::KV_BYTES;
-                    for (int it = tsm; it < (KT - valid_keys) * CH; it += NSOFT) {
-                        const int r = valid_keys + it / CH, c = it % CH;
-                        *reinterpret_cast<int4 *>(v + (c >> 3) * KT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4)) = make_int4(0, 0, 0, 0);
-                    }
-                    fence_async_smem();
-                }
-            }
-            ok = ok && mbar_wait(&bars.s_full[st], (uint32_t)(i >> 1) & 1u, abort_flag, p.status);
+            ok = ok && mbar_wait(&bars.s_full[sb], sph, abort_flag, p.status);
             ok = __all_sync(0xffffffffu, ok);             // TMEM accesses are warp-collective
             if (trace && threadIdx.x == 64 && i == 0) trace[4] = global_ns();
             tc_fence_after();
             float sc[KPT];
-#pragma unroll
-            for (int c = 0; c < KPT; c += 16) {
-                uint32_t v[16];
+            {
+                uint32_t v[KPT / 16][16];
                 if (ok) {
-                    tmem_ld16(tmem_S + lane_addr + (uint32_t)(st * 64 + cg * KPT + c), v);
-                    tmem_ld_wait();
-                } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0u;
+                    for (int c = 0; c < KPT / 16; ++c) tmem_ld16(tmem_S + lane_addr + (uint32_t)(sb * 64 + cg * KPT + c * 16), v[c]);
+                    tmem_ld_wait();
                 }
 #pragma unroll
-                for (int j = 0; j < 16; ++j) sc[c + j] = __uint_as_float(v[j]);
+                for (int c = 0; c < KPT / 16; ++c)
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) sc[c * 16 + j] = ok ? __uint_as_float(v[c][j]) : 0.f;
             }
             const bool need_mask = key0 + KT > P;
-            float mt = -INFINITY;
-#pragma unroll
-            for (int j = 0; j < KPT; ++j) {
-                float v = sc[j];                          // raw score: the scale is folded into the exponent below
-                if (need_mask) {
-                    const int key = key0 + cg * KPT + j;
-                    bool vis = key < P;
-                    if (!vis && key < n_keys) {
-                        const int b = key - P;
-                        const uint64_t w = (b >> 6) ? anc1 : anc0;
-                        vis = p.anc ? ((w >> (b & 63)) & 1ull) : true;
-                    }
-                    v = vis ? v : -INFINITY;
+            if (need_mask) {
+                // visibility of this thread's KPT keys as one bit set: committed keys (< P) are visible, keys past
+                // the last one are not, extra key b is visible if bit b of the row's ancestor set is (all of them
+                // without a mask).  b0 = index of the first key among the extra keys; negative inside the context.
+                const int b0 = key0 + cg * KPT - P;
+                uint32_t vis;
+                if (b0 >= 0) {
+                    const uint64_t lo = b0 >= 64 ? anc1 : anc0, hi = b0 >= 64 ? 0ull : anc1;
+                    const int sh = b0 & 63;
+                    vis = (uint32_t)(sh == 0 ? lo : ((lo >> sh) | (hi << (64 - sh))));
+                } else {
+                    const int nctx = -b0;                 // leading committed keys
+                    vis = nctx >= 32 ? 0xffffffffu : (((uint32_t)anc0 << nctx) | ((1u << nctx) - 1u));
                 }
-                sc[j] = v;
-                mt = fmaxf(mt, v);
-            }
-            // row maximum of the tile across the four column groups (in scaled log2 units: sl2 > 0 keeps the order)
-            mt *= sl2;
-            red[i & 1][cg][row] = mt;
-            // Leaving the loop must be decided once per quarter: its four warps meet at the barrier below every tile,
-            // and the abort flag can change between two warps' reads.  One thread samples it before the barrier.
-            if (cg == 0 && lane == 0) quit[i & 1][q] = *abort_flag;
-            asm volatile("bar.sync %0, %1;" ::"r"(2 + q), "n"(32 * NCG) : "memory");   // only the warps of this lane quarter share rows
-            if (quit[i & 1][q]) break;                    // a quarter that leaves stops arriving at p_full: every wait is bounded
-            mt = red[i & 1][0][row];
+                const int n_valid = p.T - b0;             // keys of this thread that exist
+                if (n_valid < 32) vis &= n_valid <= 0 ? 0u : ((1u << n_valid) - 1u);
 #pragma unroll
-            for (int c = 1; c < NCG; ++c) mt = fmaxf(mt, red[i & 1][c][row]);
-            if (i > 1) {
-                // this tile's P buffer was read by the second MMA of tile i-2
-                ok = ok && mbar_wait(&bars.o_done[st], (uint32_t)((i - 2) >> 1) & 1u, abort_flag, p.status);
-                ok = __all_sync(0xffffffffu, ok);
+                for (int j = 0; j < KPT; ++j) sc[j] = ((vis >> j) & 1u) ? sc[j] : -INFINITY;
             }
+            // raw scores: the scale is folded into the exponent below
+            float mt = fmaxf(sc[0], sc[1]);
+#pragma unroll
+            for (int j = 2; j < KPT; j += 2) mt = fmaxf(mt, fmaxf(sc[j], sc[j + 1]));
+            // row maximum of the tile across the column groups (in scaled log2 units: sl2 > 0 keeps the order)
+            mt *= sl2;
+            red[grp][u & 1][cg][row] = mt;
+            // Leaving the loop must be decided once per quarter: its warps meet at the barrier below every tile,
+            // and the abort flag can change between two warps' reads.  One thread samples it before the barrier.
+            if (cg == 0 && lane == 0) quit[grp][u & 1][q] = *abort_flag;
+            asm volatile("bar.sync %0, %1;" ::"r"(2 + grp * 4 + q), "n"(32 * NCG) : "memory");   // only the group's warps of this lane quarter share rows
+            if (quit[grp][u & 1][q]) break;               // a quarter that leaves stops arriving at p_full: every wait is bounded
+            mt = red[grp][u & 1][0][row];
+#pragma unroll
+            for (int c = 1; c < NCG; ++c) mt = fmaxf(mt, red[grp][u & 1][c][row]);
             float factor = 1.f;
             if (m_ref == -INFINITY) {
                 m_ref = mt;                               // nothing accumulated for this row yet
@@ -365,86 +435,106 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 m_ref = mt;
             }
             if (__any_sync(0xffffffffu, factor != 1.f)) {
-                // O may only be touched once the previous tile's second MMA has landed
-                if (i > 0) {
-                    ok = ok && mbar_wait(&bars.o_done[st ^ 1], (uint32_t)((i - 1) >> 1) & 1u, abort_flag, p.status);
+                if (i >= NG) {
+                    // the accumulator may only be touched once the second MMA of the group's previous tile has landed.
+                    // The parity wait is exact here: this tile's scores were issued behind the second MMA of the tile
+                    // before that, so the barrier is at most one phase behind the awaited one and cannot be ahead of it.
+                    ok = ok && mbar_wait(&bars.o_done[st], (uint32_t)(u - 1) & 1u, abort_flag, p.status);
                     ok = __all_sync(0xffffffffu, ok);
                 }
                 tc_fence_after();
                 if (ok) {
                     l_run *= factor;
+                    constexpr int RC = D / NCG;           // accumulator columns rescaled by this thread
 #pragma unroll
-                    for (int c = 0; c < OC; c += 16) {
+                    for (int c = 0; c < RC; c += 16) {
                         uint32_t v[16];
-                        tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                        tmem_ld16(tmem_Og + lane_addr + (uint32_t)(cg * RC + c), v);
                         tmem_ld_wait();
 #pragma unroll
                         for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * factor);
-                        tmem_st16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
+                        tmem_st16(tmem_Og + lane_addr + (uint32_t)(cg * RC + c), v);
                     }
                     tmem_st_wait();
                 }
             }
-            // P = 2^(S' - m_ref), bf16: this thread's 16 keys = two 16-byte chunks of its row of the A operand
+            // P = 2^(S' - m_ref) as bf16 pairs, written over the first half of this group's S columns (every thread of
+            // the row has its scores in registers since the barrier above): the A operand of the second MMA
             float rs = 0.f;
-            unsigned char *prow = sP + st * Smem<D>::P_BYTES + row * 128;
             const float m_sub = (m_ref == -INFINITY) ? 0.f : m_ref;   // a fully masked row keeps -inf - 0 = -inf -> 2^-inf = 0
 #pragma unroll
-            for (int c = 0; c < KPT / 8; ++c) {
-                uint32_t w[4];
+            for (int c = 0; c < KPT / 32; ++c) {
+                uint32_t w[16];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const float a = sc[c * 8 + 2 * j], b = sc[c * 8 + 2 * j + 1];
+                for (int j = 0; j < 16; ++j) {
+                    const float a = sc[c * 32 + 2 * j], b = sc[c * 32 + 2 * j + 1];
                     const float pa = ex2_approx(fmaf(a, sl2, -m_sub));
                     const float pb = ex2_approx(fmaf(b, sl2, -m_sub));
                     rs += pa + pb;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
                     w[j] = *reinterpret_cast<uint32_t *>(&h2);
                 }
-                *reinterpret_cast<uint4 *>(prow + (((cg * (KPT / 8) + c) ^ (row & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                if (ok) tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + cg * (KPT / 2) + c * 16), w);
             }
             l_run += rs;
-            fence_async_smem();
+            tmem_st_wait();
             tc_fence_before();
-            __syncwarp();                                 // 512 single arrivals would serialise on the barrier word
-            if (lane == 0) mbar_arrive(&bars.p_full[st]);  // always arrive: the MMA issuer counts one arrival per warp
+            __syncwarp();                                 // single arrivals of every thread would serialise on the barrier word
+            if (lane == 0) mbar_arrive(&bars.p_full[sb]);  // always arrive: the MMA issuer counts one arrival per warp
             if (trace && threadIdx.x == 64 && i == 0) trace[5] = global_ns();
         }
         if (trace && threadIdx.x == 64) trace[6] = global_ns();
+        // The accumulators are read below by every softmax thread.  The per-group barrier cannot be used here: a
+        // parity wait is only exact when the waiter is at most one phase behind, and a group does not observe every
+        // phase of its accumulator barrier.  The issuer commits a one-shot barrier after its last MMA instead.
         if (ok && nt > 0) {
-            ok = mbar_wait(&bars.o_done[(nt - 1) & 1], (uint32_t)((nt - 1) >> 1) & 1u, abort_flag, p.status);
+            ok = mbar_wait(&bars.all_done, 0, abort_flag, p.status);
             ok = __all_sync(0xffffffffu, ok);
             tc_fence_after();
         }
-        // row sums across the four column groups (fixed order)
+        // the groups' row sums and reference maxima meet here: every thread combines them in fixed order
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-        red[0][cg][row] = l_run;
+        red[grp][0][cg][row] = l_run;
+        red[grp][1][cg][row] = m_ref;
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
-        float l_row = red[0][0][row];
+        float gm[NG], gl[NG];
+        float m_all = -INFINITY;
 #pragma unroll
-        for (int c = 1; c < NCG; ++c) l_row += red[0][c][row];
+        for (int gi = 0; gi < NG; ++gi) {
+            gm[gi] = red[gi][1][0][row];
+            gl[gi] = red[gi][0][0][row];
+#pragma unroll
+            for (int c = 1; c < NCG; ++c) gl[gi] += red[gi][0][c][row];
+            m_all = fmaxf(m_all, gm[gi]);
+        }
+        float l_row = 0.f;
+#pragma unroll
+        for (int gi = 0; gi < NG; ++gi) {
+            // weight of the group's accumulator; a group without tiles, or with no visible key in this row, has none
+            sm_w[gi] = (gi < nt && gm[gi] != -INFINITY) ? ex2_approx(gm[gi] - m_all) : 0.f;
+            l_row += sm_w[gi] * gl[gi];
+        }
         ok = ok && (*abort_flag == 0);
         // ---------------- epilogue ----------------
         if (p.S == 1 && ok) {
+            constexpr int OC = D / ECG;
             const float inv = 1.f / l_row;
-            const size_t off = ((size_t)(s * p.T + node) * p.Hq + kvh * G + g) * D + cg * OC;
+            const size_t off = ((size_t)(s * p.T + node) * p.Hq + kvh * G + g) * D + ecg * OC;
 #pragma unroll
             for (int c = 0; c < OC; c += 16) {
-                uint32_t v[16];
-                tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
-                tmem_ld_wait();
+                float v[16];
+                load_combined(tmem_O, lane_addr + (uint32_t)(ecg * OC + c), D, min(nt, NG), sm_w, v);
                 if (row_valid) {
 #pragma unroll
                     for (int j = 0; j < 16; j += 4)
                         store_two_term(p.out + off + c + j, p.out_lo ? p.out_lo + off + c + j : nullptr,
-                                       make_float4(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv,
-                                                   __uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv));
+                                       make_float4(v[j] * inv, v[j + 1] * inv, v[j + 2] * inv, v[j + 3] * inv));
                 }
             }
         }
         tc_fence_before();
         sm_ok = ok;
-        sm_m = m_ref;
+        sm_m = m_all;
         sm_l = l_row;
     }
 
@@ -455,7 +545,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         // asynchronous shared-to-shared copy per owner ships that owner's band into the owner's receive region
         // and counts its bytes on the owner's merge barrier; the owner combines the S bands in split order.
         constexpr int ROWF = Smem<D>::ROWF;
-        constexpr int OC = D / NCG;
+        constexpr int OC = D / ECG;
         const int RPC = (QT + p.S - 1) / p.S;
         const uint32_t rank = cluster_rank();
         float *stage = reinterpret_cast<float *>(smem);
@@ -463,24 +553,23 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         if (trace && threadIdx.x == 64) trace[7] = global_ns();
         if (warp >= 2) {
             // this CTA's MMAs have all completed (o_done above) and every page it asked for has been consumed
-            const int q = warp & 3, cg = (warp - 2) >> 2;
+            const int q = warp & 3, cg = (warp - 2) >> 2;   // epilogue column group
             const int row = q * 32 + lane;
             const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
             const bool live = nt > 0 && sm_ok;
             float *dst = stage + (size_t)row * ROWF + cg * OC;
 #pragma unroll
             for (int c = 0; c < OC; c += 16) {
-                uint32_t v[16];
+                float v[16];
                 if (live) {
-                    tmem_ld16(tmem_O + lane_addr + (uint32_t)(cg * OC + c), v);
-                    tmem_ld_wait();
+                    load_combined(tmem_O, lane_addr + (uint32_t)(cg * OC + c), D, min(nt, NG), sm_w, v);
                 } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = 0u;
+                    for (int j = 0; j < 16; ++j) v[j] = 0.f;
                 }
 #pragma unroll
                 for (int j = 0; j < 16; j += 4)
-                    *reinterpret_cast<uint4 *>(dst + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    *reinterpret_cast<float4 *>(dst + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
             if (cg == 0) {
                 stage[(size_t)row * ROWF + D] = live ? sm_m : -INFINITY;

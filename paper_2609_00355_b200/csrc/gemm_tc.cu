@@ -470,13 +470,15 @@ __global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant_
                         out.z = va.z * cs.z + vb.z * sn.z; out.w = va.w * cs.w + vb.w * sn.w;
                     }
                 }
-                __nv_bfloat162 lo = __floats2bfloat162_rn(out.x, out.y), hi = __floats2bfloat162_rn(out.z, out.w);
-                uint2 ob;
-                ob.x = *reinterpret_cast<uint32_t *>(&lo);
-                ob.y = *reinterpret_cast<uint32_t *>(&hi);
                 if (is_q) {
-                    if (rr < a.Rq) *reinterpret_cast<uint2 *>(a.q + ((size_t)rr * a.Hq + h) * d + i) = ob;
+                    // queries keep two bf16 terms: their rounding error would otherwise reach every score of the row
+                    const size_t qo = ((size_t)rr * a.Hq + h) * d + i;
+                    if (rr < a.Rq) store_two_term(a.q + qo, a.q_lo ? a.q_lo + qo : nullptr, out);
                 } else {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(out.x, out.y), hi = __floats2bfloat162_rn(out.z, out.w);
+                    uint2 ob;
+                    ob.x = *reinterpret_cast<uint32_t *>(&lo);
+                    ob.y = *reinterpret_cast<uint32_t *>(&hi);
                     const long long base = it == 0 ? pre_kv[0] : it == 1 ? pre_kv[1] : a.kvrow[rr];
                     if (base >= 0)
                         *reinterpret_cast<uint2 *>(a.pool_layer + (size_t)base + (is_k ? 0 : a.v_off) + (size_t)kvh * a.head_stride + i) = ob;

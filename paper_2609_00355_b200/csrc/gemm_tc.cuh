@@ -41,7 +41,7 @@ struct TcGemmArgs {
     bf16 *xb, *xb_lo, *hidden_out;
     float *ssq_out;
     // mode 4 (rotary + K/V write): features are q heads, then k heads, then v heads, head_dim wide
-    bf16 *q;
+    bf16 *q, *q_lo;      // mode 4: rotated queries, and the second term of their two-term form (or nullptr)
     bf16 *pool_layer;
     const long long *kvrow;      // [R] element offset of the row's K slot for kv head 0 inside the layer, -1 = none
     size_t v_off, head_stride;

@@ -83,7 +83,7 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     const size_t R = d.Rmax, H = c.hidden;
     w.x = (float *)take(R * H * 4);
     w.xn = (bf16 *)take(2 * R * H * 2);                 // two planes: hi, lo
-    w.q = (bf16 *)take(R * d.qd * 2);
+    w.q = (bf16 *)take(2 * R * d.qd * 2);               // two planes
     w.attn = (bf16 *)take(2 * R * d.qd * 2);            // two planes
     w.act = (bf16 *)take(2 * R * (size_t)c.ffn * 2);    // two planes
     w.logits = (float *)take((size_t)d.Rlog * c.vocab * 4);
@@ -310,7 +310,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
         g.Nout = d.qkv_out; g.K = c.hidden; g.R = ps.R; g.S = choose_split(d.qkv_out, c.hidden, ps.R);
         with_row_scales(ctx, g);
         g.x_lo_row = 0;      // q, K, V are rounded to bf16 right after: the second term of x would buy nothing
-        g.q = ws.q; g.pool_layer = pool_layer; g.kvrow = ws.row_kvrow;
+        g.q = ws.q; g.q_lo = ws.q + (size_t)xr * d.qd; g.pool_layer = pool_layer; g.kvrow = ws.row_kvrow;
         g.v_off = (size_t)c.n_kv_heads * kPage * c.head_dim; g.head_stride = (size_t)kPage * c.head_dim;
         g.rope_cos = ws.rope_cos; g.rope_sin = ws.rope_sin;
         g.Hq = c.n_q_heads; g.Hkv = c.n_kv_heads; g.head_dim = c.head_dim; g.Rq = ps.Rq;
@@ -319,7 +319,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     if (ps.Rq == 0) return;
     AttnParams ap;
     ap.batch = ps.batch; ap.T = ps.T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
-    ap.q = ws.q; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
+    ap.q = ws.q; ap.q_lo = ws.q + (size_t)xr * d.qd; ap.pool_layer = pool_layer; ap.geom = geom; ap.page_table = page_table; ap.seq_len = seq_len;
     ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn; ap.out_lo = ws.attn + (size_t)xr * d.qd;
     ap.S = attention_tc_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch, c.head_dim);
     ap.status = ws.status;
@@ -714,7 +714,7 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     const KvGeom geom = geom_of(ctx, seqs);
     AttnParams ap;
     ap.batch = seqs->batch; ap.T = T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
-    ap.q = (const bf16 *)q; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
+    ap.q = (const bf16 *)q; ap.q_lo = nullptr; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
     ap.out = (bf16 *)out; ap.out_lo = nullptr; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
     ap.status = ctx->ws.status;

@@ -98,6 +98,7 @@ void launch_prefill_advance(int32_t *seq_len, int32_t *root, int32_t *feat_count
 struct AttnParams {
     int batch, T, Hq, Hkv, d;    // T = query rows per sequence = extra (uncommitted) keys per sequence
     const bf16 *q;               // [batch*T][Hq*d]
+    const bf16 *q_lo;            // second term of the two-term queries (same layout), or nullptr
     const bf16 *pool_layer;
     KvGeom geom;
     const int32_t *page_table;

@@ -168,7 +168,10 @@ def test_attention_random_inputs(harness, name, P, T):
         V = torch.randn(Ps[s] + T, Hkv, d, generator=g).to(torch.bfloat16)
         q = (torch.randn(T, Hq, d, generator=g) * 1.5).to(torch.bfloat16)
         eng.seq_len[s] = Ps[s]
-        _fill_cache(eng, s, 0, K.cuda(), V.cuda())
+        # the rest of the last page holds NaN bits: rows after the last key must never contribute
+        pad = (-(Ps[s] + T)) % cfg.page_size
+        poison = torch.full((pad, Hkv, d), float("nan"), dtype=torch.bfloat16)
+        _fill_cache(eng, s, 0, torch.cat([K, poison]).cuda(), torch.cat([V, poison]).cuda())
         refs.append(O.attention(q.float(), K.float(), V.float(), O.visibility(tree, Ps[s])))
         qs.append(q.reshape(T, Hq * d))
         ancs.append(torch.from_numpy(tree.anc.view(np.int64)))
@@ -178,6 +181,7 @@ def test_attention_random_inputs(harness, name, P, T):
     out2 = torch.zeros_like(out)
     eng.glance_debug_attention(0, torch.cat(qs).cuda().contiguous(), torch.stack(ancs).cuda().contiguous(), T, out2)
     assert torch.equal(out, out2)                       # split merge is order-fixed: run-to-run identical
+    assert torch.isfinite(out.float()).all()
     for s in range(2):
         got = out[s * T:(s + 1) * T].float().cpu().reshape(T, Hq, d)
         assert float((got - refs[s]).abs().max()) <= 2e-2 * float(refs[s].abs().max())
