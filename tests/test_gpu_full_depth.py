@@ -34,7 +34,10 @@ class LazyLayers:
         return {k: v.detach().cpu().float() for k, v in self.layers[i].items()}
 
 
-def test_verify_pass_7b_full_depth():
+@pytest.mark.parametrize("kv_seed", [11, 12])
+def test_verify_pass_7b_full_depth(kv_seed):
+    """Two seeds of the synthetic K/V context: the maximum error over 64 x 152064 logits varies by tens of per cent
+    from one context to the next (its rms does not), so one seed alone says little about the margin."""
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2609_00355_b200.binding import Engine
@@ -47,7 +50,7 @@ def test_verify_pass_7b_full_depth():
     P = cfg.ctx
 
     # committed state: the same seeded random K/V bits for both sides
-    g = torch.Generator(device=dev).manual_seed(11)
+    g = torch.Generator(device=dev).manual_seed(kv_seed)
     page = cfg.page_size
     pos = torch.arange(P, device=dev)
     pages = eng.page_table[0].long()[pos // page]
