@@ -56,18 +56,19 @@ static_assert(KPT % 32 == 0, "a thread writes its probabilities as 16-column chu
 // 16 accumulator columns of a row, combined over the softmax groups: sum_g w[g] * O_g.  Warp-collective.  Only the
 // first `groups` accumulators are read (a group without tiles never wrote its TMEM columns).
 __device__ __forceinline__ void load_combined(uint32_t tmem_O, uint32_t addr, int d, int groups, const float (&w)[NG], float (&out)[16]) {
+    uint32_t v[NG][16];
+#pragma unroll
+    for (int gi = 0; gi < NG; ++gi)
+        if (gi < groups) tmem_ld16(tmem_O + (uint32_t)(gi * d) + addr, v[gi]);
+    tmem_ld_wait();
 #pragma unroll
     for (int j = 0; j < 16; ++j) out[j] = 0.f;
 #pragma unroll
-    for (int gi = 0; gi < NG; ++gi) {
+    for (int gi = 0; gi < NG; ++gi)
         if (gi < groups) {
-            uint32_t v[16];
-            tmem_ld16(tmem_O + (uint32_t)(gi * d) + addr, v);
-            tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j) out[j] = fmaf(w[gi], __uint_as_float(v[j]), out[j]);
+            for (int j = 0; j < 16; ++j) out[j] = fmaf(w[gi], __uint_as_float(v[gi][j]), out[j]);
         }
-    }
 }
 
 template <int D>
@@ -340,23 +341,34 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
         const bool row_valid = pr < PR;
         if (!row_valid) pr = PR - 1;
         const int node = pr / G, g = pr % G;
+        // Q tile (both planes) -> shared memory in the K-major 128-byte-swizzled operand layout (async copies, all in
+        // flight).  A thread keeps one 16-byte chunk column and walks rows NSOFT / CH apart: the row's source offset
+        // (two integer divisions) is computed once per row and serves both planes.
+        {
+            static_assert(NSOFT % CH == 0 && QT % (NSOFT / CH) == 0, "a thread's chunks share one chunk column");
+            constexpr int RSTEP = NSOFT / CH;             // rows between a thread's consecutive chunks
+            const int c = tsm % CH;
+            const uint32_t dst0 = smem_u32(sQ) + (uint32_t)((c >> 3) * QT * 128);
+#pragma unroll
+            for (int k = 0; k < QT / RSTEP; ++k) {
+                const int r = tsm / CH + k * RSTEP;
+                int prr = qt * QT + r;
+                if (prr >= PR) prr = PR - 1;
+                const size_t off = ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c * 8;
+                const uint32_t dst = dst0 + (uint32_t)(r * 128 + (((c & 7) ^ (r & 7)) << 4));
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(p.q + off));
+                if (p.q_lo)
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)(SLABS * QT * 128)), "l"(p.q_lo + off));
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::);
+        // the row's ancestor words travel while the copies are in flight
         uint64_t anc0 = ~0ull, anc1 = ~0ull;               // no mask: every extra key is visible
         if (p.anc) {
             const uint64_t *a = p.anc + ((size_t)s * p.T + node) * p.W;
             anc0 = a[0];
             anc1 = p.W > 1 ? a[1] : 0ull;
         }
-        // Q tile (both planes) -> shared memory in the K-major 128-byte-swizzled operand layout (async copies, all in flight)
-        for (int it = tsm; it < 2 * QT * CH; it += NSOFT) {
-            const int pl = it / (QT * CH), r = (it / CH) % QT, c = it % CH;
-            int prr = qt * QT + r;
-            if (prr >= PR) prr = PR - 1;
-            const bf16 *src = pl == 0 ? p.q : p.q_lo;
-            if (src)
-                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(sQ + pl * SLABS * QT * 128 + (c >> 3) * QT * 128 + r * 128 + (((c & 7) ^ (r & 7)) << 4))),
-                             "l"(src + ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c * 8));
-        }
-        asm volatile("cp.async.commit_group;" ::);
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         fence_async_smem();
         __syncwarp();                                     // every lane's rows are written and fenced: one arrival per warp
