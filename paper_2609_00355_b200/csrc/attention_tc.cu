@@ -607,39 +607,44 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             const int tsm = threadIdx.x - 64;
             const float *rows = reinterpret_cast<const float *>(recv);
             const int my_rows = got ? max(0, min(own_rows, PR - qt * QT - row_lo)) : 0;
-            constexpr int SEG = D / 4;                    // 4-float segments per row
+            constexpr int SEG = D / 8;                    // items per row: two 4-float pieces, half a row apart
             for (int item = tsm; item < my_rows * SEG; item += NSOFT) {
-                const int lr = item / SEG, c0 = (item % SEG) * 4;
+                const int lr = item / SEG, c0 = (item % SEG) * 4, c1 = D / 2 + c0;
                 const float *rp0 = rows + (size_t)lr * ROWF;
                 const size_t sstride = (size_t)RPC * ROWF;      // floats between the same row of consecutive splits
                 // all loads first (the values of up to MAX_SPLITS splits), then the arithmetic
                 float ms[MAX_SPLITS], ls[MAX_SPLITS];
-                float4 vs[MAX_SPLITS];
+                float4 va[MAX_SPLITS], vb[MAX_SPLITS];
                 float M = -INFINITY;
 #pragma unroll
                 for (int sp = 0; sp < MAX_SPLITS; ++sp) {
-                    ms[sp] = -INFINITY; ls[sp] = 0.f; vs[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    ms[sp] = -INFINITY; ls[sp] = 0.f;
+                    va[sp] = vb[sp] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (sp < p.S) {
                         const float *rp = rp0 + sp * sstride;
                         ms[sp] = rp[D];
                         ls[sp] = rp[D + 1];
-                        vs[sp] = *reinterpret_cast<const float4 *>(rp + c0);
+                        va[sp] = *reinterpret_cast<const float4 *>(rp + c0);
+                        vb[sp] = *reinterpret_cast<const float4 *>(rp + c1);
                         M = fmaxf(M, ms[sp]);
                     }
                 }
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), bcc = acc;
                 float den = 0.f;
 #pragma unroll
                 for (int sp = 0; sp < MAX_SPLITS; ++sp) {  // split order: bit-reproducible
                     const float w = ex2_approx(ms[sp] - M);    // 2^-inf = 0 for an empty split
                     den += w * ls[sp];
-                    acc.x += w * vs[sp].x; acc.y += w * vs[sp].y; acc.z += w * vs[sp].z; acc.w += w * vs[sp].w;
+                    acc.x += w * va[sp].x; acc.y += w * va[sp].y; acc.z += w * va[sp].z; acc.w += w * va[sp].w;
+                    bcc.x += w * vb[sp].x; bcc.y += w * vb[sp].y; bcc.z += w * vb[sp].z; bcc.w += w * vb[sp].w;
                 }
                 const float inv = 1.f / den;
                 const int prr = qt * QT + row_lo + lr;
-                const size_t off = ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D + c0;
-                store_two_term(p.out + off, p.out_lo ? p.out_lo + off : nullptr,
+                const size_t off = ((size_t)(s * p.T + prr / G) * p.Hq + kvh * G + prr % G) * D;
+                store_two_term(p.out + off + c0, p.out_lo ? p.out_lo + off + c0 : nullptr,
                                make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv));
+                store_two_term(p.out + off + c1, p.out_lo ? p.out_lo + off + c1 : nullptr,
+                               make_float4(bcc.x * inv, bcc.y * inv, bcc.z * inv, bcc.w * inv));
             }
         }
     }
