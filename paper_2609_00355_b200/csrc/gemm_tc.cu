@@ -63,7 +63,7 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 // Modes 0, 1, 2 and 4 multiply each activation row's results by 1/rms(row) when a.ssq is given: the rows
 // they read are x * gain in bf16, and the row's sum of squares arrives as per-tile partial sums.
 template <int MODE>
-__global__ void __launch_bounds__(NTHR, 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+__global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                          const __grid_constant__ CUtensorMap map_x, TcGemmArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -630,14 +630,17 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     // The ring stays under half of an SM's shared memory so that two CTAs fit per SM: a GPC then offers enough
     // CTA slots for every cluster of a launch to be resident in one wave, and one CTA's prologue and epilogue
     // overlap the other's streaming.
-    int stages = (int)((100 * 1024) / stage_bytes);
+    const int tiles = mode == 1 ? (a.F + 63) / 64 : (a.Nout + BM - 1) / BM;
+    // The LM heads have a few more tiles than two CTAs per SM take in four rounds (1188 against 1184 at the 7B
+    // vocabulary): with a smaller ring three CTAs fit per SM and the last round is as full as the others.
+    const bool three = (mode == 0 || mode == 2) && tiles > 3 * 148;
+    int stages = (int)(((three ? 72 : 100) * 1024) / stage_bytes);
     stages = stages > 12 ? 12 : (stages < 2 ? 2 : stages);
     a.stages = stages;
     uint32_t cols = 32;
     while ((int)cols < nb) cols <<= 1;
     a.tmem_cols = cols;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
-    const int tiles = mode == 1 ? (a.F + 63) / 64 : (a.Nout + BM - 1) / BM;
     const int row_blocks = (a.R + 127) / 128;
     a.rows_fastest = row_blocks > 1 ? 1 : 0;
     dim3 grid(a.rows_fastest ? row_blocks : tiles, a.S, a.rows_fastest ? tiles : row_blocks);
