@@ -603,6 +603,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             const int own_rows = max(0, min(RPC, QT - row_lo));
             bool got = true;
             if (own_rows > 0) got = mbar_wait(&bars.merge, 0, abort_flag, p.status);
+            // Everything bound for this CTA has landed: that is all its peers need to know before they may leave
+            // (a CTA's staged rows are read by the copies it sent).  The matching wait is at the end of the kernel.
+            cluster_arrive();
             if (trace && threadIdx.x == 64) trace[10] = global_ns();
             const int tsm = threadIdx.x - 64;
             const float *rows = reinterpret_cast<const float *>(recv);
@@ -646,13 +649,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 store_two_term(p.out + off + c1, p.out_lo ? p.out_lo + off + c1 : nullptr,
                                make_float4(bcc.x * inv, bcc.y * inv, bcc.z * inv, bcc.w * inv));
             }
+        } else {
+            cluster_arrive();
         }
     }
     if (trace && threadIdx.x == 64) trace[11] = global_ns();
     if (p.trace && threadIdx.x == 64) atomicMax(p.trace + 15, (unsigned long long)global_ns());  // grid span: last end
     tc_fence_before();
     // no CTA leaves while its staged rows may still be read by a copy in flight, or a peer may still write to it
-    if (p.S > 1) cluster_sync_all();
+    if (p.S > 1) cluster_wait();
     else __syncthreads();
     if (warp == 1) {
         tc_fence_after();
