@@ -496,15 +496,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             if (trace && threadIdx.x == 64 && i == 0) trace[5] = global_ns();
         }
         if (trace && threadIdx.x == 64) trace[6] = global_ns();
-        // The accumulators are read below by every softmax thread.  The per-group barrier cannot be used here: a
-        // parity wait is only exact when the waiter is at most one phase behind, and a group does not observe every
-        // phase of its accumulator barrier.  The issuer commits a one-shot barrier after its last MMA instead.
-        if (ok && nt > 0) {
-            ok = mbar_wait(&bars.all_done, 0, abort_flag, p.status);
-            ok = __all_sync(0xffffffffu, ok);
-            tc_fence_after();
-        }
-        // the groups' row sums and reference maxima meet here: every thread combines them in fixed order
+        // the groups' row sums and reference maxima meet here: every thread combines them in fixed order (this needs
+        // no accumulator and runs while the last second MMA completes)
         asm volatile("bar.sync 1, %0;" ::"n"(NSOFT) : "memory");
         red[grp][0][cg][row] = l_run;
         red[grp][1][cg][row] = m_ref;
@@ -525,6 +518,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             // weight of the group's accumulator; a group without tiles, or with no visible key in this row, has none
             sm_w[gi] = (gi < nt && gm[gi] != -INFINITY) ? ex2_approx(gm[gi] - m_all) : 0.f;
             l_row += sm_w[gi] * gl[gi];
+        }
+        // The accumulators are read below by every softmax thread.  The per-group barrier cannot be used here: a
+        // parity wait is only exact when the waiter is at most one phase behind, and a group does not observe every
+        // phase of its accumulator barrier.  The issuer commits a one-shot barrier after its last MMA instead.
+        if (ok && nt > 0) {
+            ok = mbar_wait(&bars.all_done, 0, abort_flag, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            tc_fence_after();
         }
         ok = ok && (*abort_flag == 0);
         // ---------------- epilogue ----------------
