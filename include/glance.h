@@ -199,9 +199,11 @@ int32_t glance_poll_status(glance_ctx *ctx, int32_t *device_status);
 /* Test hook: the attention kernel alone.  q (device [batch*T][Hq*d] bf16) attends, per sequence, to cache
  * rows 0..seq_len-1 of target layer `layer` (all visible) and to rows seq_len..seq_len+T-1 under
  * anc (device [batch][T][(T+63)/64], or NULL = all visible); out (device [batch*T][Hq*d] bf16).
+ * q_lo and out_lo (same layouts, either may be NULL) are the second bf16 terms of the queries and of the
+ * outputs: the value is hi + lo, as between the kernels of a pass.
  * This is the masked attention of Definition 1's packed pass in isolation. */
 int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t layer, const void *q,
-                               const uint64_t *anc, int32_t T, void *out);
+                               const void *q_lo, const uint64_t *anc, int32_t T, void *out, void *out_lo);
 
 /* Test hook: the weight-streaming GEMM kernel alone (K % 64 == 0).  mode 0: Y[s][r][f] fp32 planes (S splits);
  * mode 1: W = [2F][K] (gate rows then up rows), act (device [R][F] bf16) = silu(gate) * up;

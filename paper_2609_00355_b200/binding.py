@@ -102,8 +102,8 @@ def load_library() -> C.CDLL:
     lib.glance_poll_status.restype = C.c_int32
     lib.glance_poll_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
     lib.glance_debug_attention.restype = C.c_int32
-    lib.glance_debug_attention.argtypes = [C.c_void_p, C.POINTER(Seqs), C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
-                                           C.c_void_p]
+    lib.glance_debug_attention.argtypes = [C.c_void_p, C.POINTER(Seqs), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                           C.c_int32, C.c_void_p, C.c_void_p]
     lib.glance_debug_gemm.restype = C.c_int32
     lib.glance_debug_gemm.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_int32, C.c_int32, C.c_int32, C.c_int32]
@@ -309,9 +309,10 @@ class Engine:
         _check(self.lib.glance_poll_status(self.ctx, C.byref(v)), "glance_poll_status")
         return v.value
 
-    def glance_debug_attention(self, layer: int, q: torch.Tensor, anc: Optional[torch.Tensor], T: int, out: torch.Tensor):
-        _check(self.lib.glance_debug_attention(self.ctx, C.byref(self.seqs), layer, _ptr(q), _ptr(anc), T, _ptr(out)),
-               "glance_debug_attention")
+    def glance_debug_attention(self, layer: int, q: torch.Tensor, anc: Optional[torch.Tensor], T: int, out: torch.Tensor,
+                               q_lo: Optional[torch.Tensor] = None, out_lo: Optional[torch.Tensor] = None):
+        _check(self.lib.glance_debug_attention(self.ctx, C.byref(self.seqs), layer, _ptr(q), _ptr(q_lo), _ptr(anc), T,
+                                               _ptr(out), _ptr(out_lo)), "glance_debug_attention")
 
     def glance_debug_gemm(self, mode: int, W, X, Y=None, act=None, argmax=None, S: int = 1):
         _check(self.lib.glance_debug_gemm(self.ctx, mode, _ptr(W), _ptr(X), _ptr(Y), _ptr(act), _ptr(argmax),

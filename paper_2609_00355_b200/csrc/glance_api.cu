@@ -705,7 +705,7 @@ int32_t glance_poll_status(glance_ctx *ctx, int32_t *device_status) {
 }
 
 int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t layer, const void *q,
-                               const uint64_t *anc, int32_t T, void *out) {
+                               const void *q_lo, const uint64_t *anc, int32_t T, void *out, void *out_lo) {
     int32_t rc = check_seqs(ctx, seqs);
     if (rc) return rc;
     const glance_config &c = ctx->cfg;
@@ -714,9 +714,9 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     const KvGeom geom = geom_of(ctx, seqs);
     AttnParams ap;
     ap.batch = seqs->batch; ap.T = T; ap.Hq = c.n_q_heads; ap.Hkv = c.n_kv_heads; ap.d = c.head_dim;
-    ap.q = (const bf16 *)q; ap.q_lo = nullptr; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
+    ap.q = (const bf16 *)q; ap.q_lo = (const bf16 *)q_lo; ap.pool_layer = (const bf16 *)seqs->kv_pool + (size_t)layer * geom.layer_stride();
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
-    ap.out = (bf16 *)out; ap.out_lo = nullptr; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
+    ap.out = (bf16 *)out; ap.out_lo = (bf16 *)out_lo; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
     ap.status = ctx->ws.status;
     attention(ctx, ap);
     return finish(ctx);

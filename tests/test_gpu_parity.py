@@ -195,6 +195,45 @@ def test_attention_random_inputs(harness, name, P, T):
         assert float((got - ref).abs().max()) <= 2e-2 * float(ref.abs().max())
 
 
+def test_attention_two_term_queries_and_outputs(harness):
+    """fp32 queries given as two bf16 terms, outputs read back as two terms: the only roundings left inside the
+    kernel are those of the probabilities and the fp32 accumulation, so the error against the oracle must sit far
+    below the one-term path's, whose queries alone are off by 2^-9."""
+    cfg = synth.CONFIGS["7b"].replace(n_layers=1, vocab=256, ffn=64, hidden=64, tree_N=64, n_img=2, n_txt=1, rounds=1)
+    P, T = 1536, 64
+    eng = make_engine(cfg, batch=1, max_len=P + T + 64)
+    rng = np.random.default_rng(17)
+    g = torch.Generator().manual_seed(17)
+    Hq, Hkv, d = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
+    tok, par, dep = synth.random_tree(T, 15, 1000, rng)
+    tree = O.tree_from_arrays(tok, par, dep)
+    K = (torch.randn(P + T, Hkv, d, generator=g) * 1.2).to(torch.bfloat16)
+    V = (torch.randn(P + T, Hkv, d, generator=g) * 1.2).to(torch.bfloat16)
+    q = torch.randn(T, Hq, d, generator=g) * 1.2                     # fp32: not representable in one bf16 term
+    eng.seq_len[0] = P
+    _fill_cache(eng, 0, 0, K.cuda(), V.cuda())
+    ref = O.attention(q, K.float(), V.float(), O.visibility(tree, P))
+    q_hi = q.to(torch.bfloat16)
+    q_lo = (q - q_hi.float()).to(torch.bfloat16)
+    anc = torch.from_numpy(tree.anc.view(np.int64)).cuda()[None].contiguous()
+
+    def run(lo):
+        out = torch.zeros(T, Hq * d, dtype=torch.bfloat16, device="cuda")
+        out_lo = torch.zeros_like(out)
+        eng.glance_debug_attention(0, q_hi.reshape(T, Hq * d).cuda().contiguous(), anc, T, out,
+                                   q_lo=lo.reshape(T, Hq * d).cuda().contiguous() if lo is not None else None, out_lo=out_lo)
+        eng.check_device_status()
+        got = (out.float() + out_lo.float()).cpu().reshape(T, Hq, d)
+        return float((got - ref).pow(2).mean().sqrt()), float((got - ref).abs().max())
+
+    rms1, max1 = run(None)
+    rms2, max2 = run(q_lo)
+    scale = float(ref.abs().max())
+    print(f"one-term q: rms {rms1:.3e} max {max1:.3e}; two-term q: rms {rms2:.3e} max {max2:.3e}; scale {scale:.3f}")
+    assert max2 <= 1e-2 * scale
+    assert rms2 < 0.75 * rms1                                        # the second term removes the queries' share
+
+
 # ------------------------------------------------------------------ tree builder (bit-exact)
 
 @pytest.mark.parametrize("name", ["tiny", "small", "7b", "long"])
