@@ -8,8 +8,10 @@
 //                                   would otherwise reach every score of its row), B = K page (K-major),
 //                                   accumulator in TMEM
 //     P            = 2^(S' - m)     softmax warps read S from TMEM (two threads per row), apply the scale and
-//                                   the ancestor mask, write bf16 P back into TMEM over the scores
-//     O[128 x d]  += P V            tcgen05.mma, A = P in tensor memory, B = V page (MN-major), accumulator in TMEM
+//                                   the ancestor mask, write P back into TMEM over the scores as two bf16 terms
+//                                   (hi in the first half of the tile's columns, lo in the second)
+//     O[128 x d]  += P V            tcgen05.mma, A = P_hi, then P_lo, in tensor memory, B = V page (MN-major),
+//                                   accumulator in TMEM
 // The running reference maximum m of a row is only raised when a tile exceeds it by more than 2^8 (the
 // accumulator is then rescaled in TMEM), so exponentials stay far inside fp32/bf16 range and O is almost
 // never touched between tiles.  Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocator + MMA issuer,
@@ -42,6 +44,7 @@ __device__ __forceinline__ float ex2_approx(float x) {   // 2^x, hardware approx
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+constexpr int P_TERMS = 2;       // bf16 terms of a probability (hi in the first half of the tile's S columns, lo in the second)
 constexpr int NG = 2;            // softmax groups (tile i belongs to group i % NG; S, P and O buffers are per group)
 constexpr int NCG = 2;           // column groups of a softmax group: threads per query row (a row's 64 scores are split over them)
 constexpr int KPT = KT / NCG;    // keys per thread and tile
@@ -316,9 +319,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 tc_fence_after();
                 const uint32_t vbase = smem_u32(sV + vs * Smem<D>::KV_BYTES);
 #pragma unroll
-                for (int kk = 0; kk < KT / 16; ++kk)
-                    umma_f16_ts(tmem_O + (uint32_t)(g * D), tmem_S + (uint32_t)(b * 64 + kk * 8),
-                                umma_desc_mn(vbase + kk * 16 * 128, KT * 128), idesc_o, (i >= NG || kk > 0) ? 1u : 0u);
+                for (int pt = 0; pt < P_TERMS; ++pt)
+#pragma unroll
+                    for (int kk = 0; kk < KT / 16; ++kk)
+                        umma_f16_ts(tmem_O + (uint32_t)(g * D), tmem_S + (uint32_t)(b * 64 + pt * (KT / 2) + kk * 8),
+                                    umma_desc_mn(vbase + kk * 16 * 128, KT * 128), idesc_o, (i >= NG || pt > 0 || kk > 0) ? 1u : 0u);
                 umma_commit(&bars.v_empty[vs]);           // V page free once these MMAs have read it
                 umma_commit(&bars.o_done[g]);             // this group's O updated
                 if (i + 2 * NG < nt && !issue_s(i + 2 * NG)) { ok = false; break; }
@@ -470,13 +475,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     tmem_st_wait();
                 }
             }
-            // P = 2^(S' - m_ref) as bf16 pairs, written over the first half of this group's S columns (every thread of
-            // the row has its scores in registers since the barrier above): the A operand of the second MMA
+            // P = 2^(S' - m_ref) as bf16 pairs, written over this tile's S columns (every thread of the row has its
+            // scores in registers since the barrier above): hi terms in the first half, lo terms (what the hi term
+            // lost to rounding) in the second; both are A operands of the second MMA
             float rs = 0.f;
             const float m_sub = (m_ref == -INFINITY) ? 0.f : m_ref;   // a fully masked row keeps -inf - 0 = -inf -> 2^-inf = 0
 #pragma unroll
             for (int c = 0; c < KPT / 32; ++c) {
-                uint32_t w[16];
+                uint32_t w[16], w2[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const float a = sc[c * 32 + 2 * j], b = sc[c * 32 + 2 * j + 1];
@@ -485,8 +491,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     rs += pa + pb;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
                     w[j] = *reinterpret_cast<uint32_t *>(&h2);
+                    if (P_TERMS > 1) {
+                        __nv_bfloat162 l2 = __floats2bfloat162_rn(pa - __low2float(h2), pb - __high2float(h2));
+                        w2[j] = *reinterpret_cast<uint32_t *>(&l2);
+                    }
                 }
-                if (ok) tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + cg * (KPT / 2) + c * 16), w);
+                if (ok) {
+                    tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + cg * (KPT / 2) + c * 16), w);
+                    if (P_TERMS > 1) tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + KT / 2 + cg * (KPT / 2) + c * 16), w2);
+                }
             }
             l_run += rs;
             tmem_st_wait();
