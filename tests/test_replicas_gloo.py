@@ -43,3 +43,21 @@ def test_single_replica_passthrough():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.combine_replica_stats(5.0, 7, 0.1, 3, None, "cpu") == (5.0, 7.0, 0.1, 3.0)
+
+
+def test_roofline_object_prefers_in_stream_durations():
+    """The roofline's launch duration: device timestamps when that pass ran, the event-bracketed figure otherwise,
+    and the event-bracketed figure is always kept beside the first."""
+    sys.path.insert(0, ROOT)
+    import bench
+    peak = 6000.0
+    # 100 launches of 120 MB each: 40 us per launch by events, 30 us per launch in the stream
+    r = bench.roofline_object({"gemm": [50, 1500.0], "attention": [10, 160.0]}, 4.0, 100 * 120e6, 100, 5.0, peak, "test", 121e6)
+    assert abs(r["avg_launch_us"] - 30.0) < 1e-9 and r["launches_timed"] == 50
+    assert abs(r["achieved"] - 120e6 / 30e-6 / 1e9) < 1e-6 and abs(r["frac"] - r["achieved"] / peak) < 1e-12
+    assert abs(r["event_bracketed"]["avg_launch_us"] - 40.0) < 1e-9
+    assert abs(r["event_bracketed"]["achieved"] - 120e6 / 40e-6 / 1e9) < 1e-6
+    assert r["attention_avg_launch_us"] == 16.0 and r["bound"] == "hbm" and r["traffic"] == 121e6
+    r2 = bench.roofline_object(None, 4.0, 100 * 120e6, 100, 5.0, peak, "test", None)
+    assert abs(r2["avg_launch_us"] - 40.0) < 1e-9 and "event_bracketed" not in r2
+    assert abs(r2["frac"] - (120e6 / 40e-6 / 1e9) / peak) < 1e-12
