@@ -151,7 +151,8 @@ def test_attention_mask_bits_one_hot(harness):
 
 
 @pytest.mark.parametrize("name,P,T", [("tiny", 300, 8), ("small", 704, 32), ("7b", 1536, 64), ("7b", 100, 128),
-                                      ("long", 8704, 128), ("7b", 0, 64), ("7b", 1, 1), ("tiny", 63, 2)])
+                                      ("long", 8704, 128), ("7b", 0, 64), ("7b", 1, 1), ("tiny", 63, 2),
+                                      ("7b", 191, 16), ("7b", 449, 33), ("7b", 3000, 64), ("small", 65, 32)])
 def test_attention_random_inputs(harness, name, P, T):
     base = synth.CONFIGS[name]
     cfg = base.replace(n_layers=1, vocab=256, ffn=64, hidden=64, tree_N=T, n_img=2, n_txt=1, rounds=1)
