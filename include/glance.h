@@ -14,9 +14,14 @@
  *     of the context (weights, pools, sequence state) or of the call (inputs and outputs).
  *     "host" pointers are ordinary process memory read during the call only.
  *   - The four round calls, glance_prefill and glance_commit_forced only enqueue work on the
- *     context's stream; they never synchronise and never allocate.  Faults detected on the device
- *     (capacity exceeded, bad index) are recorded in a device status word read by
- *     glance_poll_status(), which synchronises the stream.
+ *     context's stream; they never synchronise and never allocate device memory.  The first call that
+ *     meets a buffer it has not seen (a weight matrix, a pool layer, an activation buffer with a new row
+ *     count) encodes a TMA descriptor for it on the host and keeps it in the context (a few hundred bytes of
+ *     host memory, one driver call, no device work); later calls, CUDA-graph replays included, find it there.
+ *   - Faults detected on the device (capacity exceeded, bad index) are recorded in a device status word
+ *     read by glance_poll_status(), which synchronises the stream.  The page budget
+ *     seq_len + tree_N <= page_size * max_pages_per_seq is one of them (GLANCE_E_CAPACITY): seq_len lives in
+ *     device memory, so the host cannot check it before the launch.
  *   - bf16 = raw 16-bit brain-float; all matrices row-major; weights are [out_features, in_features].
  *   - Integer arrays are int32 unless stated.
  */
@@ -38,14 +43,15 @@ enum {
     GLANCE_E_CUDA = -4,        /* a CUDA runtime call failed */
     GLANCE_E_TIMEOUT = -5,     /* a bounded device-side wait gave up */
     GLANCE_E_BOUNDS = -6,      /* device-side index check failed */
-    GLANCE_E_STATE = -7        /* calls out of order */
+    GLANCE_E_STATE = -7        /* calls out of order (glance_profile_read before glance_profile_enable) */
 };
 
 typedef struct glance_ctx glance_ctx;
 
 /* Model and round shape.  Supported: head_dim in {64, 128}; hidden, ffn multiples of 64;
- * 2 <= block_B <= 16; 1 <= topk <= 16; 2 <= tree_N <= 128 (tree_N counts the root row: the
- * paper's budget is tree_N - 1); page_size = 64; n_q_heads a multiple of n_kv_heads. */
+ * 2 <= block_B <= 16; 1 <= topk <= min(16, vocab); 1 <= tree_N <= 128 (tree_N counts the root row: the
+ * paper's budget is tree_N - 1, and tree_N = 1 is plain one-token-per-pass decoding through the same calls);
+ * page_size = 64; n_q_heads a multiple of n_kv_heads. */
 #define GLANCE_MAX_HEAD_LAYERS 8
 typedef struct {
     int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
@@ -226,7 +232,8 @@ int32_t glance_debug_trace(glance_ctx *ctx, uint64_t *buffer, int32_t slots);
  * kernel kind (0 weight-streaming GEMM, 1 attention, 2 row setup, 3 top-k / tree / walk+commit, 4 everything
  * else): summed device time in milliseconds, summed algorithmic bytes (GEMM only: weights once +
  * activations in + results out) and launch count; then it resets the tally.  Disabling only pauses the
- * tally.  At most 32768 launches are tallied per read. */
+ * tally.  At most 32768 launches are tallied per read.  glance_profile_read on a context where profiling was
+ * never enabled returns GLANCE_E_STATE. */
 #define GLANCE_PROFILE_KINDS 5
 int32_t glance_profile_enable(glance_ctx *ctx, int32_t on);
 int32_t glance_profile_read(glance_ctx *ctx, double *ms, double *bytes, int64_t *launches);

@@ -1,7 +1,7 @@
 """Budget sweep on synthetic match probabilities: accepted length and round time against the verify budget N,
 chain against tree (the shape of the paper's budget tables: width saturates, the verify pass is flat in N).
 
-    python budget_sweep.py [--config 7b] [--steps 48] [--p-m 0.8 0.5]
+    python -m paper_2609_00355_b200.budget_sweep [--config 7b] [--steps 48] [--p-m 0.8 0.5]
 
 Candidates are calibrated: the true next token sits at rank r of its depth with the probability the controlled
 marginal gives that rank, so sibling branches can be hit.  Every (k, N) point builds its own engine on the same
@@ -13,9 +13,9 @@ import statistics
 
 import torch
 
-from bench import RoundBench
-from paper_2609_00355_b200 import build as glance_build
-from paper_2609_00355_b200 import synth
+from . import build as glance_build
+from . import synth
+from .round_driver import RoundBench
 
 
 def run_point(cfg, weights, dev, steps, warmup=3):
@@ -51,7 +51,7 @@ def main():
     ap.add_argument("--steps", type=int, default=48)
     ap.add_argument("--p-m", type=float, nargs="+", default=[0.8, 0.5])
     args = ap.parse_args()
-    assert torch.cuda.is_available(), "budget_sweep.py needs a CUDA device (there is no CPU fallback)"
+    assert torch.cuda.is_available(), "the budget sweep needs a CUDA device (there is no CPU fallback)"
     glance_build.build()
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)

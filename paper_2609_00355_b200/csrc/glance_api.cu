@@ -115,7 +115,7 @@ bool config_ok(const glance_config *c) {
     if (c->head_dim != 64 && c->head_dim != 128) return false;
     if (c->n_q_heads < 1 || c->n_kv_heads < 1 || c->n_q_heads % c->n_kv_heads) return false;
     if (c->vocab < 2) return false;
-    if (c->block_B < 2 || c->block_B > kMaxBlock || c->topk < 1 || c->topk > kMaxTopk) return false;
+    if (c->block_B < 2 || c->block_B > kMaxBlock || c->topk < 1 || c->topk > kMaxTopk || c->topk > c->vocab) return false;
     if (c->tree_N < 1 || c->tree_N > kMaxTreeN) return false;
     if (c->page_size != kPage || c->max_batch < 1 || c->max_batch > 64 || c->max_pages_per_seq < 1) return false;
     if (!(c->rms_eps > 0.f) || !(c->rope_theta > 1.f)) return false;
@@ -731,7 +731,9 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
     g.Nout = Nout; g.K = K; g.R = R; g.S = mode == 0 ? S : 1; g.Y = Y; g.ldy = Nout; g.split_stride = (size_t)R * Nout;
     g.act = (bf16 *)act; g.F = Nout / 2; g.argmax = argmax;
     gemm(ctx, mode, (const bf16 *)W, (const bf16 *)X, R, g);
-    ctx->maps.clear();          // the hook's operands are transient: do not keep their descriptors
+    // the hook's operands are transient: their two descriptors are dropped again, everybody else's stay
+    ctx->maps.erase(std::make_tuple((const void *)W, K, Nout, mode == 1 ? 64 : 128));
+    ctx->maps.erase(std::make_tuple((const void *)X, K, R, tc_row_pad(R)));
     return finish(ctx);
 }
 
@@ -758,6 +760,7 @@ int32_t glance_profile_enable(glance_ctx *ctx, int32_t on) {
 
 int32_t glance_profile_read(glance_ctx *ctx, double *ms, double *bytes, int64_t *launches) {
     if (!ctx || !ms || !bytes || !launches) return GLANCE_E_INVALID_ARG;
+    if (ctx->ev.empty()) return GLANCE_E_STATE;       // nothing was ever tallied: glance_profile_enable comes first
     if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return GLANCE_E_CUDA;
     for (int k = 0; k < KIND_COUNT; ++k) { ms[k] = 0.0; bytes[k] = 0.0; launches[k] = 0; }
     for (size_t i = 0; i < ctx->ev_used; ++i) {

@@ -1,4 +1,5 @@
-// Row setup, normalisation, rotary + paged K/V write, SwiGLU, argmax and top-k kernels of the round.
+// Row setup kernels of the verify and draft passes (embedding gather, rotary table, paged row offsets, first
+// norm statistics) and the two-stage per-offset top-k + log-softmax of the draft pass.
 #include "kernels.cuh"
 #include "tc_ptx.cuh"
 
@@ -101,10 +102,12 @@ __global__ void __launch_bounds__(128) setup_verify_kernel(VerifySetup p) {
     int depth = prefill ? i : p.depth[r];
     if (!prefill && (depth < 0 || depth > kMaxBlock)) depth = 0;
     if (threadIdx.x == 0) {
-        if (P < 0 || P + p.N > p.capacity) set_status(p.status, GLANCE_E_CAPACITY);
+        // a sequence without room for its N rows is reported once, as a capacity fault, and writes no K/V at all
+        const bool fits = P >= 0 && P + p.N <= p.capacity;
+        if (!fits) set_status(p.status, GLANCE_E_CAPACITY);
         p.meta.seq[r] = s;
         p.meta.pos[r] = P + depth;
-        p.meta.kvrow[r] = (P >= 0) ? kv_row_offset(p.geom, p.page_table, s, P + i, p.status) : -1;
+        p.meta.kvrow[r] = fits ? kv_row_offset(p.geom, p.page_table, s, P + i, p.status) : -1;
     }
     fill_rope_row(p.meta, r, P + depth, p.d, p.theta);
     const bf16 *src = nullptr;

@@ -47,7 +47,8 @@ extern "C" int32_t glance_topk_static(const float *logits, int32_t batch, int32_
     const size_t warps = (size_t)glance::topk_warps(vocab);
     const size_t cand_bytes = (rows * warps * k * 8 + 255) / 256 * 256;
     const size_t ml_bytes = rows * warps * 2 * 4;
-    if (cand_bytes + ml_bytes > kStaticScratchBytes) return GLANCE_E_CAPACITY;   // beyond the fixed array: refuse, launch nothing
+    // beyond the fixed array, or more rows than one launch dimension holds: refuse, launch nothing
+    if (cand_bytes + ml_bytes > kStaticScratchBytes || rows > 65535) return GLANCE_E_CAPACITY;
     void *base = nullptr;
     const int32_t rc = scratch_for_current_device(&base);
     if (rc != GLANCE_OK) return rc;
@@ -55,6 +56,7 @@ extern "C" int32_t glance_topk_static(const float *logits, int32_t batch, int32_
     // has to be cleared between calls even though the array keeps the previous call's contents
     auto *cand = reinterpret_cast<unsigned long long *>(base);
     auto *ml = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(base) + cand_bytes);
+    (void)cudaGetLastError();      // an earlier, unrelated launch error is not this call's failure
     glance::launch_topk(logits, batch, block_B, vocab, k, topk_ids, topk_lp, cand, ml, (cudaStream_t)cuda_stream);
     return cudaPeekAtLastError() == cudaSuccess ? GLANCE_OK : GLANCE_E_CUDA;
 }

@@ -95,19 +95,19 @@ __global__ void __launch_bounds__(32) build_tree_kernel(int N, int L, int k, con
         GLANCE_SLOTS(GLANCE_BEST_OP)
         // warp arg-best: hardware max over the score image, then (rarely) over the halves of the tie word
         const uint32_t m1 = __reduce_max_sync(0xffffffffu, bu >= 0 ? bsk : 0u);
-        uint32_t live = __ballot_sync(0xffffffffu, bu >= 0 && bsk == m1);
-        if (__popc(live) > 1) {
-            const bool in = (live >> lane) & 1u;
+        uint32_t cand = __ballot_sync(0xffffffffu, bu >= 0 && bsk == m1);
+        if (__popc(cand) > 1) {
+            const bool in = (cand >> lane) & 1u;
             const uint32_t m2 = __reduce_max_sync(0xffffffffu, in ? (uint32_t)(bt >> 32) : 0u);
-            live = __ballot_sync(0xffffffffu, in && (uint32_t)(bt >> 32) == m2);
-            if (__popc(live) > 1) {
-                const bool in2 = (live >> lane) & 1u;
+            cand = __ballot_sync(0xffffffffu, in && (uint32_t)(bt >> 32) == m2);
+            if (__popc(cand) > 1) {
+                const bool in2 = (cand >> lane) & 1u;
                 const uint32_t m3 = __reduce_max_sync(0xffffffffu, in2 ? (uint32_t)bt : 0u);
-                live = __ballot_sync(0xffffffffu, in2 && (uint32_t)bt == m3);
+                cand = __ballot_sync(0xffffffffu, in2 && (uint32_t)bt == m3);
             }
         }
         // (score, depth, key) identifies a candidate uniquely: exactly one lane is left; everybody takes its entry
-        const int wl = __ffs(live) - 1;
+        const int wl = __ffs(cand) - 1;
         uint32_t bmeta = 0u;
         float bps = 0.f;
 #define GLANCE_META_OP(u, sk, tw, me, ps) if (bu == u) { bmeta = me; bps = ps; }

@@ -1,0 +1,134 @@
+"""Round driver shared by the benchmark and the budget sweep: prefilled sequences, controlled-match candidate trees
+against the model's own greedy continuation (an untimed look-ahead of single-node rounds, then a state rollback),
+and the four calls of a round -- plain launches or one CUDA-graph replay.  Marshalling and input generation only:
+every step of the round runs in the CUDA library."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import synth
+
+
+def to_device(w, dev):
+    if isinstance(w, dict):
+        return {k: to_device(v, dev) for k, v in w.items()}
+    if isinstance(w, list):
+        return [to_device(v, dev) for v in w]
+    return w.to(dev)
+
+
+class RoundBench:
+    """Drives rounds of the library at controlled p_m.  All method arithmetic runs in the CUDA library."""
+
+    def __init__(self, cfg, device, rank=0, weights=None, max_new=None):
+        """max_new: tokens the sequences may grow by over the engine's life (default: cfg.rounds full blocks)."""
+        from .binding import Engine, TreeBuffers
+        self.cfg, self.dev, self.rank = cfg, device, rank
+        self.no_lookahead = False
+        self.calibrated = False      # true token at rank r with the marginal's probability (budget sweeps)
+        self.sample_seed = None      # set: sampling mode at temperature 1 (draws instead of arg-max decisions)
+        self.tw, self.hw = weights if weights is not None else synth.make_weights(cfg, device)
+        self.stream = torch.cuda.Stream(device)      # the library's stream; also made torch's current stream
+        torch.cuda.set_stream(self.stream)
+        max_len = None
+        if max_new is not None:
+            longest = max(synth.batch_context_lengths(cfg)) if cfg.batch > 1 else cfg.ctx
+            max_len = longest + max_new + 2 * cfg.tree_N + cfg.page_size
+        self.eng = Engine(cfg, self.tw, self.hw, batch=cfg.batch, stream=self.stream, max_len=max_len)
+        self.graph = None
+        eng = self.eng
+        # round log for the entropy law: every verify pass leaves the root entropy of each sequence here
+        self.root_entropy = torch.zeros(cfg.batch, dtype=torch.float32, device=device)
+        eng.glance_log_root_entropy(self.root_entropy)
+        lens = [cfg.ctx] * cfg.batch
+        if cfg.batch > 1:
+            lens = synth.batch_context_lengths(cfg)
+            self.p_ms = synth.batch_match_probs(cfg)
+        else:
+            self.p_ms = [cfg.p_m]
+        for s in range(cfg.batch):
+            n_img = cfg.n_img if cfg.batch == 1 else int(lens[s] * 0.75)
+            n_txt = lens[s] - n_img
+            img, ids = synth.make_context(cfg, device, seed=1 + s + 100 * rank, n_img=n_img, n_txt=n_txt)
+            eng.prefill_context(s, img, ids)
+        eng.check_device_status()
+        # single-node trees for the look-ahead (plain greedy steps through the same library)
+        self.ar_tree = TreeBuffers(cfg.batch, cfg.tree_N, device)
+        N, W = cfg.tree_N, (cfg.tree_N + 63) // 64
+        anc = np.zeros((N, W), dtype=np.uint64)
+        for i in range(N):
+            anc[i, i >> 6] = np.uint64(1) << np.uint64(i & 63)
+        self.ar_tree.anc.copy_(torch.from_numpy(anc.view(np.int64))[None].expand(cfg.batch, N, W))
+        self.rng = np.random.default_rng(3 + rank)
+        L, k = cfg.L, cfg.topk
+        self.lp_host = torch.from_numpy(np.stack([synth.controlled_marginals(p, k, L) for p in self.p_ms])).pin_memory()
+        self.ids_host = torch.zeros(cfg.batch, L, k, dtype=torch.int32).pin_memory()
+        self.cand_ids = torch.zeros(cfg.batch, L, k, dtype=torch.int32, device=device)
+        self.cand_lp = self.lp_host.to(device)
+        self.res_host = torch.zeros(cfg.batch, 1 + cfg.block_B, dtype=torch.int32).pin_memory()
+        self.res_dev = torch.zeros(cfg.batch, 1 + cfg.block_B, dtype=torch.int32, device=device)
+
+    def lookahead(self):
+        """Untimed: the next L greedy tokens after the pending root (single-node rounds, then rollback)."""
+        eng, cfg = self.eng, self.cfg
+        if self.no_lookahead:
+            return self.rng.integers(0, cfg.vocab, size=(cfg.batch, cfg.L))
+        snap = eng.snapshot_state()
+        ys = []
+        for _ in range(cfg.L):
+            self.ar_tree.token[:, 0].copy_(eng.root)
+            self.verify(self.ar_tree)
+            eng.glance_accept_commit(tree=self.ar_tree)
+            ys.append(eng.root.clone())
+        eng.restore_state(snap)
+        return torch.stack(ys, dim=1).cpu().numpy()      # [batch][L]
+
+    def make_candidates(self, Y, round_index=None):
+        """Candidate ids of one round around the true continuation Y.  With `round_index` the hit pattern and the
+        filler ids are drawn from a generator seeded by (rank, round_index) alone, so two arms of a benchmark that
+        number their rounds alike meet the same pattern; without it they come from the driver's running generator."""
+        cfg = self.cfg
+        if round_index is not None:
+            self.rng = np.random.default_rng((3, self.rank, int(round_index)))
+        for s in range(cfg.batch):
+            gen = synth.calibrated_candidates if self.calibrated else synth.controlled_candidates
+            self.ids_host[s] = torch.from_numpy(gen(list(Y[s]), self.p_ms[s], cfg.topk, cfg.L, cfg.vocab, self.rng))
+
+    def capture_round(self):
+        """One CUDA graph for the four calls of a round (ragged lengths live in device memory)."""
+        snap = self.eng.snapshot_state()
+        self.graph = self.eng.capture(self.round_calls)
+        self.eng.restore_state(snap)
+
+    def round_device(self):
+        """One round, inputs already on the device: graph replay when captured, else the four calls."""
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.round_calls()
+
+    def verify(self, tree=None):
+        if self.sample_seed is None:
+            self.eng.glance_verify_tree(tree=tree)
+        else:
+            self.eng.glance_verify_tree_sample(self.sample_seed, 1.0, tree=tree)
+
+    def round_calls(self):
+        eng = self.eng
+        eng.glance_draft_block()
+        eng.glance_build_tree(self.cand_ids, self.cand_lp)
+        self.verify()
+        eng.glance_accept_commit()
+
+    def round_e2e(self):
+        """Same round with this step's inputs copied from pinned host memory and the result read back."""
+        eng = self.eng
+        self.cand_ids.copy_(self.ids_host, non_blocking=True)
+        self.cand_lp.copy_(self.lp_host, non_blocking=True)
+        self.round_device()
+        self.res_dev[:, 0].copy_(eng.accept_len)
+        self.res_dev[:, 1:].copy_(eng.out_tokens)
+        self.res_host.copy_(self.res_dev, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return self.res_host[:, 0].clone()

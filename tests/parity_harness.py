@@ -2,7 +2,7 @@
 
 Because bf16 kernels and the fp32 oracle can disagree at near-ties, every round is compared stage by
 stage on the same inputs, and the GPU is put back on the oracle's path whenever a near-tie sent it
-elsewhere (the event is counted).  Tolerances (stated by the benchmark spec):
+elsewhere (the event is counted).  Tolerances:
   * logits, hidden states, log-probabilities, K/V rows: max-abs error <= 2e-2 x max|oracle tensor|
   * token ids (argmax, top-k): identical wherever the oracle's deciding margin exceeds 0.05
   * tree arrays, accepted path/length, emitted tokens, sequence state, compacted KV bytes: bit-exact

@@ -51,6 +51,12 @@ def test_workspace_sizing_and_shape_validation(lib):
     assert lib.glance_workspace_bytes(C.byref(bad)) == 0
     bad = binding.make_config(synth.CONFIGS["tiny"].replace(page_size=32), 1, 8)
     assert lib.glance_workspace_bytes(C.byref(bad)) == 0
+    # more candidates per offset than the vocabulary holds
+    bad = binding.make_config(synth.CONFIGS["tiny"].replace(vocab=8, topk=9), 1, 8)
+    assert lib.glance_workspace_bytes(C.byref(bad)) == 0
+    # a one-row budget is plain decoding and is supported
+    ok = binding.make_config(synth.CONFIGS["tiny"].replace(tree_N=1), 1, 8)
+    assert lib.glance_workspace_bytes(C.byref(ok)) > 0
     # multi-layer head: taps must be distinct target layers; deeper heads need more workspace
     one = lib.glance_workspace_bytes(C.byref(binding.make_config(synth.CONFIGS["tiny"], 1, 8)))
     two = lib.glance_workspace_bytes(C.byref(binding.make_config(synth.CONFIGS["tiny"].replace(head_taps=(0, 1)), 1, 8)))

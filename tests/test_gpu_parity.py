@@ -261,6 +261,33 @@ def test_build_tree_bit_exact(harness, tiny_run, name):
             harness.assert_tree_bits(harness.tree_from_device(eng.tree, s), O.build_tree(5 + s, ids[s], lp[s], N))
 
 
+@pytest.mark.parametrize("block_B,topk,tree_N", [(4, 1, 8), (3, 2, 16), (2, 3, 8), (5, 1, 128), (3, 3, 100)])
+def test_build_tree_exhausted_frontier_bit_exact(harness, block_B, topk, tree_N):
+    """Budgets the candidate trie cannot fill (sum_l k^l < N - 1): the frontier runs empty, n_nodes < N, and the
+    rows from n_nodes on are padding (token 0, parent -1, visible to themselves only) -- all bit for bit."""
+    cfg = synth.CONFIGS["tiny"].replace(block_B=block_B, topk=topk, tree_N=tree_N, n_img=2, n_txt=1, rounds=1, vocab=256)
+    eng = make_engine(cfg, batch=2)
+    rng = np.random.default_rng(23)
+    L, k, N = cfg.L, cfg.topk, cfg.tree_N
+    prefixes = sum(k ** l for l in range(1, L + 1))
+    assert prefixes < N - 1
+    for trial in range(4):
+        ids = np.zeros((2, L, k), dtype=np.int32)
+        lp = np.zeros((2, L, k), dtype=np.float32)
+        for s in range(2):
+            ids[s], lp[s] = synth.random_topk(L, k, 1000, rng, ties=(trial % 2 == 1))
+        roots = torch.tensor([5, 6], dtype=torch.int32, device="cuda")
+        eng.glance_build_tree(torch.from_numpy(ids).cuda(), torch.from_numpy(lp).cuda(), root=roots)
+        eng.check_device_status()
+        for s in range(2):
+            got = harness.tree_from_device(eng.tree, s)
+            want = O.build_tree(5 + s, ids[s], lp[s], N)
+            assert want.n_nodes == prefixes + 1
+            harness.assert_tree_bits(got, want)
+            assert int(eng.tree.n_nodes[s]) == prefixes + 1
+            assert all(int(v) == -1 for v in eng.tree.parent[s, prefixes + 1:].cpu())
+
+
 # ------------------------------------------------------------------ walk + commit (bit-exact)
 
 def test_walk_commit_examples_and_compaction_hazard(harness):
@@ -318,13 +345,24 @@ def test_commit_forced_and_bad_path_is_reported(harness):
     assert eng.glance_poll_status() == 0
 
 
+def test_profile_read_before_enable_is_a_state_error(harness):
+    eng = make_engine(synth.CONFIGS["tiny"], batch=1)
+    import ctypes as C
+    ms, by, n = (C.c_double * 5)(), (C.c_double * 5)(), (C.c_int64 * 5)()
+    assert eng.lib.glance_profile_read(eng.ctx, ms, by, n) == -7          # GLANCE_E_STATE
+    assert eng.lib.glance_status_string(-7) == b"invalid call order"
+    eng.glance_profile_enable(True)
+    assert eng.lib.glance_profile_read(eng.ctx, ms, by, n) == 0
+
+
 def test_capacity_overflow_sets_status_not_fault(harness):
     cfg = synth.CONFIGS["tiny"]
     run = harness.ParityRun(cfg, ctx_lens=[(20, 5)])
     eng = run.eng
     eng.seq_len[0] = eng.pages_per_seq * 64 - 2          # P + N exceeds the page budget
     eng.glance_verify_tree()
-    assert eng.glance_poll_status() in (-3, -6)
+    assert eng.glance_poll_status() == -3                 # GLANCE_E_CAPACITY, from the row setup kernel
+    assert eng.glance_poll_status() == 0
 
 
 # ------------------------------------------------------------------ the whole round, stage by stage
@@ -545,7 +583,8 @@ def test_graph_replay_equals_plain_launches(harness):
     assert len(set(accepts)) > 1, accepts
 
 
-@pytest.mark.parametrize("block_B,topk,tree_N", [(2, 16, 2), (2, 1, 2), (16, 16, 128), (3, 2, 7), (16, 2, 33)])
+@pytest.mark.parametrize("block_B,topk,tree_N", [(2, 16, 2), (2, 1, 2), (16, 16, 128), (3, 2, 7), (16, 2, 33),
+                                                 (4, 1, 8), (3, 2, 16)])
 def test_rounds_extreme_block_topk_budget(harness, block_B, topk, tree_N):
     """Corners of the supported shapes: the shortest block (L = 1), the widest top-k, the smallest and the largest
     verify budget, budgets that the candidate trie cannot fill (n_nodes < N) and budgets that are not multiples of

@@ -486,6 +486,59 @@ def test_draft_block_single_key_closed_form(tiny):
     assert np.abs(dl - ref).max() <= 1e-4 * np.abs(ref).max()
 
 
+def test_head_context_kv_stated_reading_in_float64(tiny):
+    """The head's context keys/values for committed positions (Section 3.2: they are the target's hidden states, read
+    here as projections of the normalised features through the head layer's own W_k / W_v): written out row by row
+    in float64 numpy with a NON-unit context gain,
+        K[p] = rotate(W_k (f_p / rms(f_p) * g_ctx), p),     V[p] = W_v (f_p / rms(f_p) * g_ctx)   (not rotated).
+    Dropping the norm, the gain or the key rotation, rotating the values, or reading the q rows of W_qkv instead of
+    the k / v rows moves the result by O(1) of its scale; the pin allows 1e-4."""
+    sh = tiny.sh
+    Hq, Hkv, d, H = sh.n_q_heads, sh.n_kv_heads, sh.head_dim, sh.hidden
+    half = d // 2
+    rng = np.random.default_rng(41)
+    hw = dict(tiny.hw)
+    g_ctx = rng.uniform(0.5, 1.5, size=H)
+    hw["ctx_norm"] = torch.from_numpy(g_ctx).float()
+    n = 5
+    feats = torch.from_numpy(rng.normal(0.0, 3.0, size=(n, H))).float()       # far from unit rms: the norm matters
+    pos = torch.tensor([0, 3, 17, 300, 1234])
+    K, V = O.head_context_kv(sh, hw, feats, pos)
+    assert K.shape == (n, Hkv, d) and V.shape == (n, Hkv, d)
+    Wqkv = hw["wqkv"].double().numpy()
+    Wk, Wv = Wqkv[Hq * d:(Hq + Hkv) * d], Wqkv[(Hq + Hkv) * d:]
+    inv_freq = np.array([sh.rope_theta ** (-(2.0 * i) / d) for i in range(half)])
+    g64 = hw["ctx_norm"].double().numpy()
+    for r in range(n):
+        f = feats[r].double().numpy()
+        hn = f / np.sqrt(np.mean(f * f) + sh.rms_eps) * g64
+        k = (Wk @ hn).reshape(Hkv, d)
+        v = (Wv @ hn).reshape(Hkv, d)
+        ang = float(pos[r]) * inv_freq
+        c, s_ = np.cos(ang), np.sin(ang)
+        k_rot = np.concatenate([k[:, :half] * c - k[:, half:] * s_, k[:, half:] * c + k[:, :half] * s_], axis=1)
+        assert np.abs(K[r].double().numpy() - k_rot).max() <= 1e-4 * np.abs(k_rot).max()
+        assert np.abs(V[r].double().numpy() - v).max() <= 1e-4 * np.abs(v).max()
+        # the pin has teeth: each plausible mistake is far outside the allowance
+        if r > 0:
+            assert np.abs(k - k_rot).max() > 1e-2 * np.abs(k_rot).max()                        # rotation dropped
+        no_gain = (Wv @ (f / np.sqrt(np.mean(f * f) + sh.rms_eps))).reshape(Hkv, d)
+        assert np.abs(no_gain - v).max() > 1e-2 * np.abs(v).max()                              # gain dropped
+        no_norm = (Wv @ (f * g64)).reshape(Hkv, d)
+        assert np.abs(no_norm - v).max() > 1e-1 * np.abs(v).max()                              # norm dropped
+
+
+def test_prefill_and_commit_store_head_context_kv_of_the_tapped_features(tiny):
+    """The state a round leaves is this function applied to the stored features: after prefill and after rounds,
+    hK / hV of every committed position equal head_context_kv(feat[p], p)."""
+    st = _fresh(tiny)
+    for _ in range(3):
+        O.spec_round(tiny.sh, tiny.tw, tiny.hw, st, tiny.cfg.block_B, tiny.cfg.topk, tiny.cfg.tree_N)
+    P = st.P
+    K, V = O.head_context_kv(tiny.sh, tiny.hw, st.feat[:P], torch.arange(P))
+    assert torch.allclose(st.hK[:P], K, atol=1e-6) and torch.allclose(st.hV[:P], V, atol=1e-6)
+
+
 def test_draft_block_context_order_invariance(tiny):
     """No mask inside [context ; block]: permuting the context rows (keys and values together) changes nothing,
     while breaking the pairing of keys and values does."""

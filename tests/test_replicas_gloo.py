@@ -39,6 +39,27 @@ def test_replica_statistics_max_time_sum_tokens():
         assert abs(e2e_s - 0.04) < 1e-12 and e2e_committed == 101.0
 
 
+def test_bench_gpus_2_without_a_launcher_spawns_two_ranks():
+    """`python bench.py --gpus 2` run as one plain process must become two ranks (here: gloo on CPU, made-up
+    statistics) and report their combined figures -- never one replica's work under n_gpus = 2."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--replica-selftest"],
+                         capture_output=True, text=True, timeout=300, env=env, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                           # rank 0 alone prints
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["world"] == 2
+    assert line["total_ms"] == 11.0 and line["committed"] == 300.0   # slowest replica's time, both replicas' tokens
+    # a launcher that gave another number of ranks than --gpus is refused
+    env_bad = dict(env, WORLD_SIZE="1", RANK="0")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--replica-selftest"],
+                         capture_output=True, text=True, timeout=120, env=env_bad, cwd=ROOT)
+    assert res.returncode == 2 and "WORLD_SIZE" in res.stderr
+
+
 def test_single_replica_passthrough():
     sys.path.insert(0, ROOT)
     import bench
@@ -53,6 +74,11 @@ def test_roofline_object_prefers_in_stream_durations():
     peak = 6000.0
     # 100 launches of 120 MB each: 40 us per launch by events, 30 us per launch in the stream
     r = bench.roofline_object({"gemm": [50, 1500.0], "attention": [10, 160.0]}, 4.0, 100 * 120e6, 100, 5.0, peak, "test", 121e6)
+    assert abs(r["frac_with_activations"] - r["frac"]) < 1e-12          # no weights-only figure given: the two agree
+    rw = bench.roofline_object({"gemm": [50, 1500.0], "attention": [10, 160.0]}, 4.0, 100 * 120e6, 100, 5.0, peak, "test", 121e6,
+                               weight_bytes_per_launch=90e6)
+    assert abs(rw["achieved"] - 90e6 / 30e-6 / 1e9) < 1e-6 and abs(rw["frac_with_activations"] - r["frac"]) < 1e-12
+    assert rw["traffic_note"] and abs(rw["event_bracketed"]["achieved"] - 90e6 / 40e-6 / 1e9) < 1e-6
     assert abs(r["avg_launch_us"] - 30.0) < 1e-9 and r["launches_timed"] == 50
     assert abs(r["achieved"] - 120e6 / 30e-6 / 1e9) < 1e-6 and abs(r["frac"] - r["achieved"] / peak) < 1e-12
     assert abs(r["event_bracketed"]["avg_launch_us"] - 40.0) < 1e-9

@@ -1,20 +1,25 @@
-"""glance_topk_static: the workspace-free top-k entry point against the regular draft path (GPU).
+"""glance_topk_static: the workspace-free top-k entry point (GPU).
 
 Some callers may not allocate device memory (their process gave the whole GPU to its own arena, or they run
 inside a callback where allocation calls are forbidden), so this entry point keeps its scratch in a fixed
 array inside the library.  The test drives it through the C ABI twice in a row -- the array keeps the first
-call's contents -- and compares with what glance_draft_block returned for the same logits.
-Collected last on purpose: a failure here leaves every other test's result intact.
+call's contents -- and compares its output (a) with what glance_draft_block returned for the same logits and
+(b) with the oracle's per-offset top-k and log-softmax of those logits.
 """
+import numpy as np
 import pytest
 import torch
 
+from oracle import glance_oracle as O
 from paper_2609_00355_b200 import synth
 
 pytestmark = pytest.mark.gpu
 
+MARGIN = 0.05          # ids are compared where consecutive ranks are further apart than this
+TOL = 2e-2             # of the logit scale
 
-def test_topk_static_matches_draft_block_twice():
+
+def test_topk_static_matches_draft_block_and_oracle_twice():
     if not torch.cuda.is_available():
         pytest.skip("no CUDA device")
     from paper_2609_00355_b200 import binding
@@ -38,7 +43,21 @@ def test_topk_static_matches_draft_block_twice():
         # which is well inside the 2e-2 (relative to the logit scale) tolerance of the other parity tests
         assert torch.equal(ids, ids_ref)
         assert torch.equal(lp, lp_ref)
-        assert float((lp - lp_ref).abs().max()) <= 2e-2 * float(logits.abs().max())
+        scale = float(logits.abs().max())
+        assert float((lp - lp_ref).abs().max()) <= TOL * scale
+        # against the oracle on the same logits: log-probabilities within the tolerance, ids identical wherever
+        # the oracle's gap between consecutive ranks exceeds the margin
+        lg_cpu = logits.cpu()
+        for s in range(2):
+            oid, olp = O.topk_logprobs(lg_cpu[s], k)
+            assert float(np.abs(lp[s].cpu().numpy() - olp).max()) <= TOL * scale
+            for j in range(L):
+                srt = np.sort(lg_cpu[s, j + 1].numpy())[::-1][:k + 1]
+                for r in range(k):
+                    clear_above = r == 0 or srt[r - 1] - srt[r] > MARGIN
+                    clear_below = srt[r] - srt[r + 1] > MARGIN
+                    if clear_above and clear_below:
+                        assert int(ids[s, j, r]) == int(oid[j, r]), (call, s, j, r)
         # move the state on so that the second call sees different logits and stale scratch from the first
         eng.glance_build_tree()
         eng.glance_verify_tree()
@@ -48,4 +67,7 @@ def test_topk_static_matches_draft_block_twice():
     lib = binding.load_library()
     rc = lib.glance_topk_static(big.data_ptr(), 64, 16, 1 << 24, 16, ids.data_ptr(), lp.data_ptr(), None)
     assert rc == -3 and lib.glance_status_string(rc) == b"capacity exceeded"
+    # so is one with more rows than a launch dimension takes, although its scratch would fit
+    rc = lib.glance_topk_static(big.data_ptr(), 65536, 2, 8, 1, ids.data_ptr(), lp.data_ptr(), None)
+    assert rc == -3
     assert lib.glance_topk_static(None, 1, 2, 8, 1, ids.data_ptr(), lp.data_ptr(), None) == -1
