@@ -108,6 +108,113 @@ def test_verify_pass_7b_full_depth(kv_seed):
             assert am[i] == int(oam[i]), f"node {i}: arg-max differs at margin {margin[i]:.3g}"
 
 
+def _verify_pass_against_oracle(cfg, lens, kv_seed, kv_std=0.5):
+    """One verify pass of `cfg` over len(lens) sequences with committed lengths `lens`, every layer's committed K/V
+    rows seeded random bf16 values given to both sides; returns the worst relative errors (logits, hidden) and the
+    number of clear arg-max decisions that were compared (all of which must agree)."""
+    from paper_2609_00355_b200.binding import Engine
+    from tests import parity_harness as H
+
+    dev = torch.device("cuda:0")
+    batch = len(lens)
+    tw, hw = synth.make_weights(cfg, dev)
+    eng = Engine(cfg, tw, hw, batch=batch, max_len=max(lens) + 2 * cfg.tree_N + cfg.page_size)
+    g = torch.Generator(device=dev).manual_seed(kv_seed)
+    page = cfg.page_size
+    Ks, Vs = [[] for _ in range(batch)], [[] for _ in range(batch)]
+    for s, P in enumerate(lens):
+        pos = torch.arange(P, device=dev)
+        pages = eng.page_table[s].long()[pos // page]
+        for l in range(cfg.n_layers):
+            K = (torch.randn(P, cfg.n_kv_heads, cfg.head_dim, generator=g, device=dev) * kv_std).to(torch.bfloat16)
+            V = (torch.randn(P, cfg.n_kv_heads, cfg.head_dim, generator=g, device=dev) * kv_std).to(torch.bfloat16)
+            eng.kv_pool[l, pages, 0, :, pos % page, :] = K
+            eng.kv_pool[l, pages, 1, :, pos % page, :] = V
+            Ks[s].append(K.cpu())
+            Vs[s].append(V.cpu())
+        eng.seq_len[s] = P
+        eng.root[s] = 1234 + 17 * s
+    rng = np.random.default_rng(5)
+    ids = np.zeros((batch, cfg.L, cfg.topk), dtype=np.int32)
+    lp = np.zeros((batch, cfg.L, cfg.topk), dtype=np.float32)
+    for s in range(batch):
+        ids[s], lp[s] = synth.random_topk(cfg.L, cfg.topk, cfg.vocab, rng)
+    eng.glance_build_tree(torch.from_numpy(ids).to(dev), torch.from_numpy(lp).to(dev))
+    vlog = torch.zeros(batch, cfg.tree_N, cfg.vocab, dtype=torch.float32, device=dev)
+    eng.glance_verify_tree(logits_dbg=vlog)
+    eng.check_device_status()
+    torch.cuda.synchronize()
+
+    otw = {"embed": tw["embed"].cpu().float(), "lm_head": tw["lm_head"].cpu().float(),
+           "final_norm": tw["final_norm"].cpu().float(), "layers": LazyLayers(tw["layers"])}
+    worst_l = worst_h = 0.0
+    compared = 0
+    for s, P in enumerate(lens):
+        root = 1234 + 17 * s
+        tree = O.build_tree(root, ids[s], lp[s], cfg.tree_N)
+        H.assert_tree_bits(H.tree_from_device(eng.tree, s), tree)
+        cap = P + cfg.tree_N + 8
+        st = O.SeqState(P, root, [], [], torch.zeros(1), torch.zeros(1), torch.zeros(1))
+        for l in range(cfg.n_layers):
+            Kc = torch.zeros(cap, cfg.n_kv_heads, cfg.head_dim)
+            Kc[:P] = Ks[s][l].float()
+            st.K.append(Kc)
+            Vc = torch.zeros(cap, cfg.n_kv_heads, cfg.head_dim)
+            Vc[:P] = Vs[s][l].float()
+            st.V.append(Vc)
+        ol, oh = O.verify_tree(O.Shape.of(cfg), otw, st, tree)
+        n = tree.n_nodes
+        assert n == cfg.tree_N
+        scale = float(ol[:n].abs().max())
+        err = float((vlog[s, :n].cpu() - ol[:n]).abs().max())
+        assert err <= H.REL_TOL * scale, f"sequence {s}: logits max-abs error {err:.4g} > {H.REL_TOL} x {scale:.4g}"
+        hscale = float(oh[:n].abs().max())
+        herr = float((eng.hidden[0, s, :n].float().cpu() - oh[:n]).abs().max()) if eng.hidden.dim() == 4 else \
+            float((eng.hidden[s, :n].float().cpu() - oh[:n]).abs().max())
+        assert herr <= H.REL_TOL * hscale, f"sequence {s}: hidden max-abs error {herr:.4g} > {H.REL_TOL} x {hscale:.4g}"
+        worst_l, worst_h = max(worst_l, err / scale), max(worst_h, herr / hscale)
+        oam = O.argmax_lowest(ol)
+        top2 = torch.topk(ol, 2, dim=-1).values
+        margin = (top2[:, 0] - top2[:, 1]).numpy()
+        am = eng.argmax[s].cpu().numpy()
+        for i in range(n):
+            if margin[i] > H.MARGIN:
+                assert am[i] == int(oam[i]), f"sequence {s} node {i}: arg-max differs at margin {margin[i]:.3g}"
+                compared += 1
+        # the tree rows' K/V of the first and the last layer, as written into the paged cache
+        for l in (0, cfg.n_layers - 1):
+            Kg, Vg = eng.gather_kv(s, l, P + n)
+            kscale = float(st.K[l][P:P + n].abs().max())
+            assert float((Kg[P:].float().cpu() - st.K[l][P:P + n]).abs().max()) <= H.REL_TOL * kscale
+            vscale = float(st.V[l][P:P + n].abs().max())
+            assert float((Vg[P:].float().cpu() - st.V[l][P:P + n]).abs().max()) <= H.REL_TOL * vscale
+    return worst_l, worst_h, compared
+
+
+def test_verify_pass_long_full_depth():
+    """The long-context configuration at full depth: 28 layers, N = 128 tree rows (two mask words, 256-column MMA
+    tiles with the two-term activations) against 8704 committed positions."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    cfg = synth.CONFIGS["long"]
+    wl, wh, compared = _verify_pass_against_oracle(cfg, [cfg.ctx], kv_seed=31)
+    print(f"long full depth: logits {wl:.3e}, hidden {wh:.3e} of scale; {compared} clear arg-max rows compared")
+    assert compared > 0
+
+
+def test_verify_pass_batch8_7b_widths_four_row_blocks():
+    """Eight ragged sequences (1024-4096 committed positions) at the 7B widths: 512 verify rows = four 128-row
+    blocks per weight tile, per-sequence trees, contexts and page tables; three target layers and the full LM head."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    cfg = synth.CONFIGS["batch8"].replace(n_layers=3)
+    lens = synth.batch_context_lengths(cfg)
+    assert len(lens) == 8 and min(lens) >= 1024 and max(lens) <= 4096
+    wl, wh, compared = _verify_pass_against_oracle(cfg, lens, kv_seed=37)
+    print(f"batch 8, 3 layers: logits {wl:.3e}, hidden {wh:.3e} of scale; {compared} clear arg-max rows compared")
+    assert compared > 0
+
+
 def test_draft_pass_7b_full_vocabulary():
     """The draft pass at the benchmark's widths and full vocabulary (head layer 3584 / 18944, LM head over 152064
     ids, top-8 of every block slot) against the oracle, on a seeded synthetic head context of 1536 positions.
