@@ -378,6 +378,8 @@ def main():
     ap.add_argument("--no-ar", action="store_true", help="skip the plain greedy-decoding comparison arm")
     ap.add_argument("--no-stream-spans", action="store_true", help="skip the device-timestamp pass behind roofline_in_stream")
     ap.add_argument("--no-graph", action="store_true", help="launch the round's kernels one by one instead of replaying a CUDA graph")
+    ap.add_argument("--attn-terms", type=int, nargs=2, default=None, metavar=("LO_SKIP", "MIN_KEYS"),
+                    help="override which second bf16 terms the attention drops on pure-context key tiles (tuning)")
     ap.add_argument("--replica-selftest", action="store_true",
                     help="CPU-only check of the replica launcher and of the statistics reduction (gloo ranks, no GPU work)")
     args = ap.parse_args()
@@ -445,6 +447,8 @@ def main():
     # every timed, profiled and end-to-end round may commit a whole block
     rounds_total = 2 * (warmup + args.steps) + min(args.steps, 16) + 2
     bench = RoundBench(cfg, dev, rank, max_new=max(rounds_total, cfg.rounds) * cfg.block_B)
+    if args.attn_terms:
+        bench.eng.glance_debug_attention_terms(*args.attn_terms)
     bench.no_lookahead = args.no_lookahead
     bench.sample_seed = args.sample_seed
     eng = bench.eng

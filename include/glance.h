@@ -211,6 +211,13 @@ int32_t glance_poll_status(glance_ctx *ctx, int32_t *device_status);
 int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t layer, const void *q,
                                const void *q_lo, const uint64_t *anc, int32_t T, void *out, void *out_lo);
 
+/* Test hook / tuning knob: second bf16 terms of the attention on key tiles that lie entirely inside the committed
+ * context (tiles holding tree or block keys always keep both terms).  lo_skip bit 0: such a tile's score MMAs use the
+ * queries' first term only; bit 1: its P V MMAs use the probabilities' first term only; applied to sequences with at
+ * least min_keys committed positions.  Host call; takes effect from the next enqueued pass (a captured CUDA graph
+ * keeps the setting it was captured with). */
+int32_t glance_debug_attention_terms(glance_ctx *ctx, int32_t lo_skip, int32_t min_keys);
+
 /* Test hook: the weight-streaming GEMM kernel alone (K % 64 == 0).  mode 0: Y[s][r][f] fp32 planes (S splits);
  * mode 1: W = [2F][K] (gate rows then up rows), act (device [R][F] bf16) = silu(gate) * up;
  * mode 2: argmax (device [R] int32) over f of X W^T with ties to the lowest f, Y (device [R][Nout] fp32) optional. */

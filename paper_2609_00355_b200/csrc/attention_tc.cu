@@ -175,6 +175,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
     const int t_end = (int)(((long long)(split + 1) * n_tiles + p.S - 1) / p.S);
     const int nt = t_end - t_begin;
     const int32_t *pt = p.page_table + (size_t)s * p.geom.max_pages_per_seq;
+    // second terms of queries / probabilities on pure-context tiles (see AttnParams::lo_skip)
+    const bool skip_q_lo = (p.lo_skip & 1) && P >= p.lo_skip_min_keys;
+    const bool skip_p_lo = (p.lo_skip & 2) && P >= p.lo_skip_min_keys;
     if (warp != 0) {
         pdl_wait();                                      // q, the tree rows' K/V and the outputs belong to other kernels
         if (trace && threadIdx.x == 64) trace[2] = global_ns();
@@ -292,10 +295,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
             const int planes = p.q_lo ? 2 : 1;
             auto issue_s = [&](int i) -> bool {
                 const int b = i & 3, ks_slot = i % KS;    // S buffer in TMEM / K page slot in shared memory
+                const int planes_i = (skip_q_lo && (t_begin + i + 1) * KT <= P) ? 1 : planes;
                 if (!mbar_wait(&bars.k_full[ks_slot], (uint32_t)(i / KS) & 1u, abort_flag, p.status)) return false;
                 tc_fence_after();
                 const uint32_t kbase = smem_u32(sK + ks_slot * Smem<D>::KV_BYTES);
-                for (int pl = 0; pl < planes; ++pl) {
+                for (int pl = 0; pl < planes_i; ++pl) {
                     const uint32_t qbase = smem_u32(sQ) + (uint32_t)(pl * SLABS * QT * 128);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
@@ -318,8 +322,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                 if (i == nt - 1 && n_keys - (t_end - 1) * KT < KT && !mbar_wait(&bars.v_zero, 0, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t vbase = smem_u32(sV + vs * Smem<D>::KV_BYTES);
-#pragma unroll
-                for (int pt = 0; pt < P_TERMS; ++pt)
+                const int p_terms = (skip_p_lo && (t_begin + i + 1) * KT <= P) ? 1 : P_TERMS;
+                for (int pt = 0; pt < p_terms; ++pt)
 #pragma unroll
                     for (int kk = 0; kk < KT / 16; ++kk)
                         umma_f16_ts(tmem_O + (uint32_t)(g * D), tmem_S + (uint32_t)(b * 64 + pt * (KT / 2) + kk * 8),
@@ -410,6 +414,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     for (int j = 0; j < 16; ++j) sc[c * 16 + j] = ok ? __uint_as_float(v[c][j]) : 0.f;
             }
             const bool need_mask = key0 + KT > P;
+            const bool two_p = P_TERMS > 1 && !(skip_p_lo && !need_mask);   // this tile's probabilities keep their second term
             if (need_mask) {
                 // visibility of this thread's KPT keys as one bit set: committed keys (< P) are visible, keys past
                 // the last one are not, extra key b is visible if bit b of the row's ancestor set is (all of them
@@ -491,14 +496,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc_kernel(const __grid_const
                     rs += pa + pb;
                     __nv_bfloat162 h2 = __floats2bfloat162_rn(pa, pb);
                     w[j] = *reinterpret_cast<uint32_t *>(&h2);
-                    if (P_TERMS > 1) {
+                    if (two_p) {
                         __nv_bfloat162 l2 = __floats2bfloat162_rn(pa - __low2float(h2), pb - __high2float(h2));
                         w2[j] = *reinterpret_cast<uint32_t *>(&l2);
                     }
                 }
                 if (ok) {
                     tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + cg * (KPT / 2) + c * 16), w);
-                    if (P_TERMS > 1) tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + KT / 2 + cg * (KPT / 2) + c * 16), w2);
+                    if (two_p) tmem_st16(tmem_S + lane_addr + (uint32_t)(sb * 64 + KT / 2 + cg * (KPT / 2) + c * 16), w2);
                 }
             }
             l_run += rs;
@@ -733,14 +738,18 @@ int max_active_clusters(int cs) {
 int attention_tc_q_tiles(int T, int G) { return (T * G + QT - 1) / QT; }
 
 // Key splits per (sequence, kv head, q tile): the splits of a tile form a cluster, and all clusters of the
-// launch should be resident at once (a second wave would double the kernel's latency).
+// launch should be resident at once (a second wave would double the kernel's latency).  A launch that cannot fit
+// one wave split (several sequences) gets two splits: that halves the longest sequence's loop, which sets the
+// launch's duration, while larger clusters lose more than they gain once clusters queue for SMs (a cluster starts
+// only when enough SMs of one GPC are free together: 8 sequences of 1024-4096 positions took 100 / 84 / 102 / 154 us
+// per layer with 1 / 2 / 4 / 8 splits).
 int attention_tc_splits(int T, int G, int Hkv, int batch, int d) {
     const int base = attention_tc_q_tiles(T, G) * Hkv * batch;
     for (int s = MAX_SPLITS; s > 1; --s) {
         const int fit = d == 128 ? max_active_clusters<128>(s) : max_active_clusters<64>(s);
         if (base <= fit) return s;
     }
-    return 1;
+    return base <= 148 ? 2 : 1;
 }
 
 cudaError_t launch_attention_tc(const AttnParams &p, const CUtensorMap &map_kv, cudaStream_t st) {

@@ -19,10 +19,30 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 // split-K factor of a weight-streaming GEMM: as many CTAs as fit one wave at two CTAs per SM (one CTA per SM
 // keeps too few weight bytes in flight to cover the HBM latency), at least 7 k-tiles per split
 // The splits of one tile form a thread-block cluster (<= 8 CTAs) that reduces them through shared memory.
-int choose_split(int Nout, int K, int rows) {
+// With more than one 128-row block the launch is tensor-bound, not latency-bound: every (tile, row block) item is a
+// long main loop, and splitting K only pays where it evens out the last wave over the 148 SMs -- each split adds a
+// cluster epilogue of a few microseconds per item.
+int choose_split(int Nout, int K, int rows, bool two_term) {
     const int tiles = (Nout + 127) / 128;
     const int ktiles = K / 64;
-    (void)rows;
+    const int row_blocks = (rows + 127) / 128;
+    if (row_blocks > 1) {
+        // Two CTAs per SM keep about 200 KB of operands in flight, which is what the tensor rate needs from L2; one
+        // CTA per SM runs at about half of it.  So a wave is 296 items wide, each item running at half an SM's rate.
+        const double step_us = two_term ? 0.45 : 0.225;       // one 128 x 128-row x 64 k-step at an SM's tensor rate
+        const double unit_us = ktiles * step_us;               // one unsplit item with the SM to itself
+        const int smax = std::max(1, std::min(8, ktiles / 7));
+        int best = 1;
+        double best_us = 1e30;
+        for (int s = 1; s <= smax; ++s) {
+            const double waves = std::ceil((double)tiles * row_blocks * s / 296.0);
+            // cluster epilogue per wave; clusters of a later wave also wait for enough SMs of one GPC to come free together
+            const double epilogue_us = s == 1 ? 0.0 : (waves > 1.0 ? 10.0 : 3.0);
+            const double us = waves * (2.0 * unit_us / s + epilogue_us);
+            if (us < best_us - 1e-9) { best_us = us; best = s; }
+        }
+        return best;
+    }
     int s = (2 * 148) / tiles;
     s = std::min(s, std::max(1, ktiles / 7));
     s = std::max(1, std::min(s, 8));
@@ -162,6 +182,8 @@ struct glance_ctx {
     // test hook: phase timestamps of successive GEMM launches, 16 words each, ring of trace_slots launches
     unsigned long long *trace = nullptr;
     int trace_slots = 0, trace_next = 0;
+    // attention: which second bf16 terms the pure-context key tiles drop, and from which context length on
+    int attn_lo_skip = 0, attn_lo_min_keys = 0;
 };
 
 namespace {
@@ -307,7 +329,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     const int xr = d.Rmax;                             // rows allocated behind every activation buffer
     {
         TcGemmArgs g{};
-        g.Nout = d.qkv_out; g.K = c.hidden; g.R = ps.R; g.S = choose_split(d.qkv_out, c.hidden, ps.R);
+        g.Nout = d.qkv_out; g.K = c.hidden; g.R = ps.R; g.S = choose_split(d.qkv_out, c.hidden, ps.R, false);
         with_row_scales(ctx, g);
         g.x_lo_row = 0;      // q, K, V are rounded to bf16 right after: the second term of x would buy nothing
         g.q = ws.q; g.q_lo = ws.q + (size_t)xr * d.qd; g.pool_layer = pool_layer; g.kvrow = ws.row_kvrow;
@@ -323,11 +345,12 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     ap.anc = ps.anc; ap.W = (ps.T + 63) / 64; ap.out = ws.attn; ap.out_lo = ws.attn + (size_t)xr * d.qd;
     ap.S = attention_tc_splits(ps.T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, ps.batch, c.head_dim);
     ap.status = ws.status;
+    ap.lo_skip = ctx->attn_lo_skip; ap.lo_skip_min_keys = ctx->attn_lo_min_keys;
     attention(ctx, ap);
     const int R = ps.Rq;
     {
         TcGemmArgs g{};
-        g.Nout = c.hidden; g.K = d.qd; g.R = R; g.S = choose_split(c.hidden, d.qd, R);
+        g.Nout = c.hidden; g.K = d.qd; g.R = R; g.S = choose_split(c.hidden, d.qd, R, true);
         g.x = ws.x; g.gain = w.ln2; g.xb = ws.xn; g.xb_lo = ws.xn + (size_t)xr * c.hidden; g.ssq_out = ws.ssq;
         g.ssq_stride = d.Rmax; g.x_lo_row = xr;
         gemm(ctx, 3, w.wo, ws.attn, xr, g);
@@ -341,7 +364,7 @@ void run_layer(glance_ctx *ctx, const LayerW &w, bf16 *pool_layer, const PassInf
     }
     {
         TcGemmArgs g{};
-        g.Nout = c.hidden; g.K = c.ffn; g.R = R; g.S = choose_split(c.hidden, c.ffn, R);
+        g.Nout = c.hidden; g.K = c.ffn; g.R = R; g.S = choose_split(c.hidden, c.ffn, R, true);
         g.x = ws.x; g.gain = next_gain; g.xb = ws.xn; g.xb_lo = ws.xn + (size_t)xr * c.hidden; g.hidden_out = hidden_out;
         g.ssq_out = ws.ssq; g.ssq_stride = d.Rmax; g.x_lo_row = xr;
         gemm(ctx, 3, w.wd, ws.act, xr, g);
@@ -718,6 +741,7 @@ int32_t glance_debug_attention(glance_ctx *ctx, const glance_seqs *seqs, int32_t
     ap.geom = geom; ap.page_table = seqs->page_table; ap.seq_len = seqs->seq_len; ap.anc = anc; ap.W = (T + 63) / 64;
     ap.out = (bf16 *)out; ap.out_lo = (bf16 *)out_lo; ap.S = attention_tc_splits(T, c.n_q_heads / c.n_kv_heads, c.n_kv_heads, seqs->batch, c.head_dim);
     ap.status = ctx->ws.status;
+    ap.lo_skip = ctx->attn_lo_skip; ap.lo_skip_min_keys = ctx->attn_lo_min_keys;
     attention(ctx, ap);
     return finish(ctx);
 }
@@ -735,6 +759,13 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
     ctx->maps.erase(std::make_tuple((const void *)W, K, Nout, mode == 1 ? 64 : 128));
     ctx->maps.erase(std::make_tuple((const void *)X, K, R, tc_row_pad(R)));
     return finish(ctx);
+}
+
+int32_t glance_debug_attention_terms(glance_ctx *ctx, int32_t lo_skip, int32_t min_keys) {
+    if (!ctx || lo_skip < 0 || lo_skip > 3 || min_keys < 0) return GLANCE_E_INVALID_ARG;
+    ctx->attn_lo_skip = lo_skip;
+    ctx->attn_lo_min_keys = min_keys;
+    return GLANCE_OK;
 }
 
 int32_t glance_debug_trace(glance_ctx *ctx, uint64_t *buffer, int32_t slots) {

@@ -108,6 +108,11 @@ struct AttnParams {
     bf16 *out;                   // [batch*T][Hq*d]
     bf16 *out_lo;                // second term of the two-term output, or nullptr
     int S;                       // key splits (= cluster size)
+    // Second bf16 terms on key tiles that lie entirely inside the committed context: bit 0 set = the score MMAs of
+    // such a tile use the queries' first term only, bit 1 set = its P V MMAs use the probabilities' first term only.
+    // Applied to sequences with at least lo_skip_min_keys committed positions (tiles that hold tree / block keys
+    // always keep both terms).
+    int lo_skip, lo_skip_min_keys;
     int32_t *status;
     unsigned long long *trace;   // test hook: phase timestamps of the first CTA, or nullptr
 };

@@ -108,7 +108,7 @@ def test_verify_pass_7b_full_depth(kv_seed):
             assert am[i] == int(oam[i]), f"node {i}: arg-max differs at margin {margin[i]:.3g}"
 
 
-def _verify_pass_against_oracle(cfg, lens, kv_seed, kv_std=0.5):
+def _verify_pass_against_oracle(cfg, lens, kv_seed, kv_std=0.5, attn_terms=None):
     """One verify pass of `cfg` over len(lens) sequences with committed lengths `lens`, every layer's committed K/V
     rows seeded random bf16 values given to both sides; returns the worst relative errors (logits, hidden) and the
     number of clear arg-max decisions that were compared (all of which must agree)."""
@@ -119,6 +119,8 @@ def _verify_pass_against_oracle(cfg, lens, kv_seed, kv_std=0.5):
     batch = len(lens)
     tw, hw = synth.make_weights(cfg, dev)
     eng = Engine(cfg, tw, hw, batch=batch, max_len=max(lens) + 2 * cfg.tree_N + cfg.page_size)
+    if attn_terms is not None:
+        eng.glance_debug_attention_terms(*attn_terms)
     g = torch.Generator(device=dev).manual_seed(kv_seed)
     page = cfg.page_size
     Ks, Vs = [[] for _ in range(batch)], [[] for _ in range(batch)]
