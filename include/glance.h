@@ -224,6 +224,15 @@ int32_t glance_debug_attention_terms(glance_ctx *ctx, int32_t lo_skip, int32_t m
 int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const void *X, float *Y, void *act,
                              int32_t *argmax, int32_t Nout, int32_t K, int32_t R, int32_t S);
 
+/* Test hook for the bounded device waits (every mbarrier wait of the tcgen05 kernels gives up after a limit, records
+ * GLANCE_E_TIMEOUT in the status word, lets the CTA drain the copies it has in flight, free its tensor memory and
+ * return).  One shot: in the NEXT glance_debug_gemm launch the TMA producer never fills the ring slot of k-step
+ * `kstep` (0-based, of every CTA's own K range) and every wait of that launch gives up after wait_limit_ns
+ * (1 us .. 1 s) instead of the regular second, so the MMA issuer's wait on that slot runs out.  Nothing faults and
+ * nothing is left in flight; the launch's results are undefined, the status word reads GLANCE_E_TIMEOUT, and the
+ * context stays usable. */
+int32_t glance_debug_stall_next_gemm(glance_ctx *ctx, int32_t kstep, uint64_t wait_limit_ns);
+
 /* Test hook: phase timestamps of the GEMM kernel.  While a buffer (device, slots x 16 uint64) is set, the
  * n-th GEMM launch after this call makes its first CTA write nanosecond timestamps (entry, set-up done,
  * predecessor finished, first tile landed, accumulator ready, cluster barrier 1, tile shipped, cluster

@@ -20,7 +20,7 @@ EXPORTS = [
     "glance_verify_tree_sample", "glance_log_root_entropy",
     "glance_accept_commit", "glance_commit_forced", "glance_poll_status", "glance_launch_count",
     "glance_debug_attention", "glance_debug_gemm", "glance_profile_enable", "glance_profile_read",
-    "glance_topk_static", "glance_debug_trace", "glance_debug_attention_terms",
+    "glance_topk_static", "glance_debug_trace", "glance_debug_attention_terms", "glance_debug_stall_next_gemm",
 ]
 
 
@@ -113,6 +113,8 @@ def load_library() -> C.CDLL:
     lib.glance_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.glance_debug_attention_terms.restype = C.c_int32
     lib.glance_debug_attention_terms.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
+    lib.glance_debug_stall_next_gemm.restype = C.c_int32
+    lib.glance_debug_stall_next_gemm.argtypes = [C.c_void_p, C.c_int32, C.c_uint64]
     lib.glance_debug_trace.restype = C.c_int32
     lib.glance_debug_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
     lib.glance_topk_static.restype = C.c_int32
@@ -322,6 +324,9 @@ class Engine:
 
     def glance_debug_attention_terms(self, lo_skip: int, min_keys: int = 0):
         _check(self.lib.glance_debug_attention_terms(self.ctx, lo_skip, min_keys), "glance_debug_attention_terms")
+
+    def glance_debug_stall_next_gemm(self, kstep: int, wait_limit_ns: int):
+        _check(self.lib.glance_debug_stall_next_gemm(self.ctx, kstep, wait_limit_ns), "glance_debug_stall_next_gemm")
 
     def glance_debug_trace(self, buffer: Optional[torch.Tensor]):
         slots = 0 if buffer is None else buffer.numel() // 16

@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
     const int kt0 = (int)((long long)split * ktiles / a.S), kt1 = (int)((long long)(split + 1) * ktiles / a.S);
     const int nk = kt1 - kt0;
     const uint32_t tmem_cols = a.tmem_cols;
+    const uint64_t wait_limit = a.wait_limit_ns ? a.wait_limit_ns : kWaitLimitNs;
 
     // optional phase timestamps of CTA (0,0,0) (test hook; a.trace is nullptr in normal use)
     unsigned long long *trace = (a.trace && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0) ? a.trace : nullptr;
@@ -135,6 +136,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
             // weights do not depend on earlier kernels: fill the ring with them before waiting on the predecessor
             const int pre = min(nk, stages);
             for (int i = 0; i < pre; ++i) {
+                if (i + 1 == a.stall_kstep1) continue;        // test hook: this slot is never filled
                 mbar_expect_tx(&bars.full[i], (uint32_t)stage_bytes);
                 load_w(i, smem + (size_t)i * stage_bytes, &bars.full[i]);
             }
@@ -142,6 +144,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
             if (trace) trace[2] = global_ns();
             for (int i = 0; i < pre; ++i)
             {
+                if (i + 1 == a.stall_kstep1) continue;
                 unsigned char *xs = smem + (size_t)i * stage_bytes + BM * 128;
                 tma_load_2d(xs, &map_x, &bars.full[i], (kt0 + i) * BK, r0);
                 if (NB > NP) tma_load_2d(xs + NP * 128, &map_x, &bars.full[i], (kt0 + i) * BK, a.x_lo_row + r0);
@@ -150,7 +153,8 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
             for (int i = pre; i < nk; ++i) {
                 const int s = i % stages;
                 const uint32_t ph = (uint32_t)(i / stages) & 1u;
-                if (!mbar_wait(&bars.empty[s], ph ^ 1u, abort_flag, a.status)) break;
+                if (!mbar_wait(&bars.empty[s], ph ^ 1u, abort_flag, a.status, wait_limit)) break;
+                if (i + 1 == a.stall_kstep1) continue;        // test hook (nothing issued: `issued` keeps its value)
                 unsigned char *slot = smem + (size_t)s * stage_bytes;
                 mbar_expect_tx(&bars.full[s], (uint32_t)stage_bytes);
                 load_w(i, slot, &bars.full[s]);
@@ -161,9 +165,10 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
             if (*abort_flag) {
                 // copies already issued must land before the CTA may exit
                 for (int i = max(0, issued - stages); i < issued; ++i) {
+                    if (i + 1 == a.stall_kstep1) continue;    // never issued
                     const uint64_t t0 = global_ns();
                     while (!mbar_try_wait(&bars.full[i % stages], (uint32_t)(i / stages) & 1u))
-                        if (global_ns() - t0 > kWaitLimitNs) break;
+                        if (global_ns() - t0 > wait_limit) break;
                 }
             }
         }
@@ -175,7 +180,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
             for (int i = 0; i < nk && mok; ++i) {
                 const int s = i % stages;
                 const uint32_t ph = (uint32_t)(i / stages) & 1u;
-                if (!mbar_wait(&bars.full[s], ph, abort_flag, a.status)) { mok = false; break; }
+                if (!mbar_wait(&bars.full[s], ph, abort_flag, a.status, wait_limit)) { mok = false; break; }
                 if (trace && i == 0) trace[3] = global_ns();
                 tc_fence_after();
                 const uint32_t slot = smem_u32(smem + (size_t)s * stage_bytes);
@@ -201,7 +206,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
             }
             if (t < 128) inv_rms[t] = inv;
         }
-        if (nk > 0) ok = mbar_wait(&bars.acc_ready, 0, abort_flag, a.status);
+        if (nk > 0) ok = mbar_wait(&bars.acc_ready, 0, abort_flag, a.status, wait_limit);
         ok = __all_sync(0xffffffffu, ok);                // tcgen05.ld is warp-collective: decide as a warp
         tc_fence_after();
         asm volatile("bar.sync 1, 256;" ::: "memory");   // inv_rms visible to all epilogue warps

@@ -48,6 +48,11 @@ struct TcGemmArgs {
     const float *rope_cos, *rope_sin;   // [R][head_dim/2]
     int Hq, Hkv, head_dim, Rq;
     unsigned long long *trace;   // test hook: 16 phase timestamps (ns) of CTA (0,0,0), or nullptr
+    // test hook for the bounded waits: every wait of the launch gives up after wait_limit_ns (0 = the regular limit),
+    // and the producer never fills the ring slot of k-step stall_kstep1 - 1 (0 = none), so the consumer's wait on it
+    // runs out
+    unsigned long long wait_limit_ns;
+    int stall_kstep1;
     // filled by launch_gemm_tc
     int np, stages, rows_fastest;
     uint32_t tmem_cols;

@@ -184,6 +184,9 @@ struct glance_ctx {
     int trace_slots = 0, trace_next = 0;
     // attention: which second bf16 terms the pure-context key tiles drop, and from which context length on
     int attn_lo_skip = 0, attn_lo_min_keys = 0;
+    // test hook, one shot: the next glance_debug_gemm launch withholds one ring slot and waits at most this long
+    int stall_kstep1 = 0;
+    unsigned long long stall_limit_ns = 0;
 };
 
 namespace {
@@ -754,11 +757,20 @@ int32_t glance_debug_gemm(glance_ctx *ctx, int32_t mode, const void *W, const vo
     TcGemmArgs g{};
     g.Nout = Nout; g.K = K; g.R = R; g.S = mode == 0 ? S : 1; g.Y = Y; g.ldy = Nout; g.split_stride = (size_t)R * Nout;
     g.act = (bf16 *)act; g.F = Nout / 2; g.argmax = argmax;
+    g.stall_kstep1 = ctx->stall_kstep1; g.wait_limit_ns = ctx->stall_limit_ns;
+    ctx->stall_kstep1 = 0; ctx->stall_limit_ns = 0;      // one shot
     gemm(ctx, mode, (const bf16 *)W, (const bf16 *)X, R, g);
     // the hook's operands are transient: their two descriptors are dropped again, everybody else's stay
     ctx->maps.erase(std::make_tuple((const void *)W, K, Nout, mode == 1 ? 64 : 128));
     ctx->maps.erase(std::make_tuple((const void *)X, K, R, tc_row_pad(R)));
     return finish(ctx);
+}
+
+int32_t glance_debug_stall_next_gemm(glance_ctx *ctx, int32_t kstep, uint64_t wait_limit_ns) {
+    if (!ctx || kstep < 0 || wait_limit_ns < 1000 || wait_limit_ns > 1000ull * 1000ull * 1000ull) return GLANCE_E_INVALID_ARG;
+    ctx->stall_kstep1 = kstep + 1;
+    ctx->stall_limit_ns = wait_limit_ns;
+    return GLANCE_OK;
 }
 
 int32_t glance_debug_attention_terms(glance_ctx *ctx, int32_t lo_skip, int32_t min_keys) {

@@ -60,6 +60,28 @@ def test_gemm_tc_planes(gemm_eng, Nout, K, R, S):
     assert torch.equal(Y, Y2)
 
 
+def test_bounded_wait_runs_out_and_the_context_stays_usable(gemm_eng):
+    """Failure detection on the device, without a fault: one ring slot of a tiny GEMM is never filled (chosen on the
+    host), the MMA issuer's bounded wait on it gives up after 100 us, the CTA drains the copies it has in flight,
+    frees its tensor memory and returns; the host reads GLANCE_E_TIMEOUT, and the next launch is correct."""
+    eng = gemm_eng
+    g = torch.Generator(device="cuda").manual_seed(99)
+    W = (torch.randn(128, 512, generator=g, device="cuda") * 0.05).to(torch.bfloat16)
+    X = torch.randn(16, 512, generator=g, device="cuda").to(torch.bfloat16)
+    ref = X.double() @ W.double().T
+    for kstep in (2, 6):                                   # inside the first ring fill, and in a re-used slot
+        Y = torch.zeros(1, 16, 128, device="cuda")
+        eng.glance_debug_stall_next_gemm(kstep, 100_000)
+        eng.glance_debug_gemm(0, W, X, Y=Y, S=1)
+        assert eng.glance_poll_status() == -5              # GLANCE_E_TIMEOUT
+        assert eng.glance_poll_status() == 0               # cleared by the read
+        # the hook was one shot: the same launch again is a normal one
+        Y2 = torch.full((1, 16, 128), float("nan"), device="cuda")
+        eng.glance_debug_gemm(0, W, X, Y=Y2, S=1)
+        assert eng.glance_poll_status() == 0
+        assert float((Y2[0].double() - ref).abs().max()) <= 1e-4 * float(ref.abs().max()) + 1e-5
+
+
 @pytest.mark.parametrize("F,K,R", [(704, 256, 8), (2816, 1024, 32), (18944, 3584, 64), (320, 128, 130)])
 def test_gemm_tc_swiglu(gemm_eng, F, K, R):
     eng = gemm_eng
