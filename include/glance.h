@@ -144,8 +144,9 @@ int32_t glance_seq_truncate(glance_ctx *ctx, const glance_seqs *seqs, int32_t se
  * slots 1..L masked (L = block_B - 1); every slot attends to all committed context K/V and all
  * block slots.  Also refreshes the head's context K/V for the feat_count rows committed last.
  * Outputs (device): topk_ids [batch][L][k] and topk_lp [batch][L][k] = logit - logsumexp over
- * the full vocabulary, ordered by (logit desc, id asc).  logits_dbg (device [batch][block_B][V]
- * fp32) may be NULL. */
+ * the full vocabulary, ordered by (logit desc, id asc).  The selection and the log-sum-exp run inside the
+ * LM head's epilogue (per 128-feature tile) and one small merge launch; the block's logits are written only on
+ * request: logits_dbg (device [batch][block_B][V] fp32) may be NULL. */
 int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *topk_ids, float *topk_lp,
                            float *logits_dbg);
 

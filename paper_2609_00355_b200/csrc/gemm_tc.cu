@@ -60,10 +60,11 @@ __device__ __forceinline__ float gumbel_from_word(uint32_t w) {
 // MODE 0: fp32 planes              MODE 1: SwiGLU (64 gate + 64 up rows per tile)   MODE 2: arg-max (+ optional logits)
 // MODE 3: split-K over a cluster, residual add + bf16 copy scaled by the next norm's gain + sum of squares
 // MODE 4: split-K over a cluster, rotary embedding + q / paged K,V write
+// MODE 5: per-row top-k candidates + log-sum-exp share of every 128-feature tile (draft LM head; + optional logits)
 // Modes 0, 1, 2 and 4 multiply each activation row's results by 1/rms(row) when a.ssq is given: the rows
 // they read are x * gain in bf16, and the row's sum of squares arrives as per-tile partial sums.
 template <int MODE>
-__global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
+__global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2 || MODE == 5) ? 3 : 2) gemm_tc_kernel(const __grid_constant__ CUtensorMap map_w,
                                                          const __grid_constant__ CUtensorMap map_x, TcGemmArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = reinterpret_cast<unsigned char *>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -72,7 +73,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
 
     // MODE 1 stacks 64 gate rows and the matching 64 up rows into one 128-row weight tile (two TMA boxes)
     constexpr int FT = (MODE == 1) ? 64 : BM;            // output features per CTA
-    constexpr bool CLUSTERED = (MODE >= 3);
+    constexpr bool CLUSTERED = (MODE == 3 || MODE == 4);
     const int NP = a.np;                                 // activation rows per CTA, padded to 16
     // With two-term activations (x = hi + lo, both bf16) the lo rows ride along as NP more rows of the B
     // operand: the accumulator gets NP more columns, which the epilogue adds to the first NP.
@@ -327,7 +328,7 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
     }
     if (warp >= 2 && ok) {
         const float *tile = reinterpret_cast<const float *>(smem);
-        if (MODE == 0 || MODE == 2) {
+        if (MODE == 0 || MODE == 2 || MODE == 5) {
             const bool vec = (a.ldy & 3) == 0;
             for (int r = ew; r < my_rows; r += NEPI) {
                 const int rr = r0 + r;
@@ -335,6 +336,96 @@ __global__ void __launch_bounds__(NTHR, (MODE == 0 || MODE == 2) ? 3 : 2) gemm_t
                 const float sc = inv_rms[r];
                 v.x *= sc; v.y *= sc; v.z *= sc; v.w *= sc;
                 const int f = f0 + fo;
+                if (MODE == 5) {
+                    // Block slot 0 of every sequence is the root: its row is not a prediction (Section 3.2).
+                    // Per row and tile: (max, sum of exponentials) for the log-sum-exp over the vocabulary, and the
+                    // packed (value, id) keys that can still be among the row's k largest.  A key qualifies if it
+                    // reaches a threshold that at least k entries of the row are known to reach.  The row keeps k
+                    // running maxima in global memory, one per residue class of the tile index modulo k (every tile
+                    // raises its class's maximum with atomicMax): the smallest of the k is such a threshold -- k
+                    // entries of k different tiles reach it -- and with ~150 tiles per class it sits close to the
+                    // row's true k-th largest value.  While a class is still empty, or if too many entries of this
+                    // tile reach the bound, the tile falls back to its own bound, the k-th largest of its 32 lane
+                    // maxima.  Which tiles emit what depends on timing; the merged result (the k largest keys,
+                    // unique by id) does not.
+                    if (rr % a.tk_B != 0) {
+                        const bool in0 = f < a.Nout, in1 = f + 1 < a.Nout, in2 = f + 2 < a.Nout, in3 = f + 3 < a.Nout;
+                        float m = -INFINITY;
+                        if (in0) m = v.x;
+                        if (in1) m = fmaxf(m, v.y);
+                        if (in2) m = fmaxf(m, v.z);
+                        if (in3) m = fmaxf(m, v.w);
+                        const float lane_max = m;
+                        m = warp_max(m);
+                        float e = 0.f;
+                        if (in0) e += __expf(v.x - m);
+                        if (in1) e += __expf(v.y - m);
+                        if (in2) e += __expf(v.z - m);
+                        if (in3) e += __expf(v.w - m);
+                        e = warp_sum(e);
+                        const size_t slot = (size_t)tile_idx * a.R + rr;
+                        if (lane == 0) {
+                            a.tk_ml[2 * slot] = m;
+                            a.tk_ml[2 * slot + 1] = e;
+                        }
+                        const uint32_t k0 = in0 ? float_key(v.x) : 0u, k1 = in1 ? float_key(v.y) : 0u;
+                        const uint32_t k2 = in2 ? float_key(v.z) : 0u, k3 = in3 ? float_key(v.w) : 0u;
+                        uint32_t T = lane < a.tk_k ? __ldcg(a.tk_thr + (size_t)rr * kTopkTileCap + lane) : 0xffffffffu;
+                        T = __reduce_min_sync(0xffffffffu, T);
+                        if (lane == 0 && m != -INFINITY) atomicMax(a.tk_thr + (size_t)rr * kTopkTileCap + tile_idx % a.tk_k, float_key(m));
+                        auto count_at = [&](uint32_t t) {
+                            return __popc(__ballot_sync(0xffffffffu, k0 >= t && in0)) + __popc(__ballot_sync(0xffffffffu, k1 >= t && in1)) +
+                                   __popc(__ballot_sync(0xffffffffu, k2 >= t && in2)) + __popc(__ballot_sync(0xffffffffu, k3 >= t && in3));
+                        };
+                        int nhit = T ? count_at(T) : kTopkTileCap + 1;
+                        if (nhit > kTopkTileCap) {
+                            // the running bound is unset or loose: this tile's own bound, the k-th largest lane maximum
+                            // (at least k entries of the tile reach it; k <= 16 <= 32 lanes)
+                            uint32_t cur = lane_max == -INFINITY ? 0u : float_key(lane_max), tl = 0u;
+                            for (int t = 0; t < a.tk_k; ++t) {
+                                tl = __reduce_max_sync(0xffffffffu, cur);
+                                const uint32_t holders = __ballot_sync(0xffffffffu, cur == tl);
+                                if (lane == __ffs(holders) - 1) cur = 0u;
+                            }
+                            if (tl > T) T = tl;
+                            nhit = T ? count_at(T) : kTopkTileCap + 1;
+                        }
+                        unsigned long long *out = a.tk_cand + slot * kTopkTileCap;
+                        if (nhit <= kTopkTileCap) {
+                            int at = 0;
+                            const uint32_t below = (1u << lane) - 1u;
+#define GLANCE_EMIT(kk, inb, val, id)                                                        \
+                            {                                                                \
+                                const bool hit = (inb) && (kk) >= T;                         \
+                                const uint32_t hits = __ballot_sync(0xffffffffu, hit);       \
+                                if (hit) out[at + __popc(hits & below)] = pack_val_id(val, id); \
+                                at += __popc(hits);                                          \
+                            }
+                            GLANCE_EMIT(k0, in0, v.x, f) GLANCE_EMIT(k1, in1, v.y, f + 1) GLANCE_EMIT(k2, in2, v.z, f + 2) GLANCE_EMIT(k3, in3, v.w, f + 3)
+#undef GLANCE_EMIT
+                            if (lane == 0) a.tk_cnt[slot] = nhit;
+                        } else {
+                            // more than the slots hold (a tile full of equal values, or fewer than k entries): exact selection
+                            const unsigned long long q0 = in0 ? pack_val_id(v.x, f) : 0ull, q1 = in1 ? pack_val_id(v.y, f + 1) : 0ull;
+                            const unsigned long long q2 = in2 ? pack_val_id(v.z, f + 2) : 0ull, q3 = in3 ? pack_val_id(v.w, f + 3) : 0ull;
+                            unsigned long long prev = ~0ull;
+                            int n = 0;
+                            for (int t = 0; t < a.tk_k; ++t) {
+                                unsigned long long best = 0ull;
+                                if (q0 < prev && q0 > best) best = q0;
+                                if (q1 < prev && q1 > best) best = q1;
+                                if (q2 < prev && q2 > best) best = q2;
+                                if (q3 < prev && q3 > best) best = q3;
+                                best = warp_max_u64(best);
+                                if (best == 0ull) break;
+                                if (lane == 0) out[t] = best;
+                                prev = best;
+                                ++n;
+                            }
+                            if (lane == 0) a.tk_cnt[slot] = n;
+                        }
+                    }
+                }
                 if (MODE == 0 || a.Y) {
                     float *dst = a.Y + (MODE == 0 ? (size_t)split * a.split_stride : 0) + (size_t)rr * a.ldy + f;
                     if (vec && f + 3 < a.Nout) *reinterpret_cast<float4 *>(dst) = v;
@@ -599,7 +690,7 @@ cudaError_t launch_mode(const TcGemmArgs &a, const CUtensorMap &mw, const CUtens
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = (MODE >= 3) ? grid.y : 1;     // the K splits of one tile form a cluster
+    attr[0].val.clusterDim.y = (MODE == 3 || MODE == 4) ? grid.y : 1;     // the K splits of one tile form a cluster
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
@@ -638,7 +729,7 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     const int tiles = mode == 1 ? (a.F + 63) / 64 : (a.Nout + BM - 1) / BM;
     // The LM heads have a few more tiles than two CTAs per SM take in four rounds (1188 against 1184 at the 7B
     // vocabulary): with a smaller ring three CTAs fit per SM and the last round is as full as the others.
-    const bool three = (mode == 0 || mode == 2) && tiles > 3 * 148;
+    const bool three = (mode == 0 || mode == 2 || mode == 5) && tiles > 3 * 148;
     int stages = (int)(((three ? 72 : 100) * 1024) / stage_bytes);
     stages = stages > 12 ? 12 : (stages < 2 ? 2 : stages);
     a.stages = stages;
@@ -649,7 +740,7 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     const int row_blocks = (a.R + 127) / 128;
     a.rows_fastest = row_blocks > 1 ? 1 : 0;
     dim3 grid(a.rows_fastest ? row_blocks : tiles, a.S, a.rows_fastest ? tiles : row_blocks);
-    if (mode >= 3) {
+    if (mode == 3 || mode == 4) {
         // every CTA's ring must hold S planes of ceil(np/S) rows, and a cluster has at most 8 CTAs
         const size_t rp = (a.np + a.S - 1) / a.S;
         if (a.S > 8 || (size_t)a.S * rp * BM * 4 > (size_t)stages * stage_bytes) return cudaErrorInvalidValue;
@@ -658,6 +749,7 @@ cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, con
     if (mode == 1) return launch_mode<1>(a, map_w, map_x, smem, grid, st);
     if (mode == 2) return launch_mode<2>(a, map_w, map_x, smem, grid, st);
     if (mode == 3) return launch_mode<3>(a, map_w, map_x, smem, grid, st);
+    if (mode == 5) return launch_mode<5>(a, map_w, map_x, smem, grid, st);
     return launch_mode<4>(a, map_w, map_x, smem, grid, st);
 }
 

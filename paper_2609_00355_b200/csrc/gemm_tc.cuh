@@ -6,6 +6,8 @@
 
 namespace glance {
 
+constexpr int kTopkTileCap = 16;     // candidate keys a (tile, row) pair may emit (>= the largest k)
+
 struct TcGemmArgs {
     int Nout, K, R, S;          // W [Nout][K], X [R][K]; S = split-K factor (modes 0, 3, 4; 1 otherwise)
     int x_lo_row;               // > 0: X is two-term (hi + lo, both bf16); the lo plane starts at this row of the X map
@@ -31,7 +33,17 @@ struct TcGemmArgs {
     // sequence r / ent_N to ent_out; ent_out == nullptr: off
     float *ent_part, *ent_out;
     int ent_N, ent_batch;
-    // row scales (modes 0, 1, 2, 4): row r is multiplied by rsqrt(sum_i ssq[i*ssq_stride + r] / K + eps); nullptr = 1
+    // mode 5 (top-k of the draft block): rows r with r % tk_B != 0 leave, per 128-feature tile, (max, sum exp) in
+    // tk_ml [tiles][R][2], up to kTopkTileCap packed (value, id) keys in tk_cand [tiles][R][kTopkTileCap] and their
+    // number in tk_cnt [tiles][R]; tk_thr [R][kTopkTileCap] holds, per row, the order-preserving images of tk_k running
+    // maxima (class c = tiles with index % tk_k == c; 0 = empty; raised with atomicMax, re-armed by the merge kernel):
+    // their minimum is a bound that at least tk_k entries of the row reach
+    int tk_k, tk_B;
+    uint32_t *tk_thr;
+    float *tk_ml;
+    int32_t *tk_cnt;
+    unsigned long long *tk_cand;
+    // row scales (modes 0, 1, 2, 4, 5): row r is multiplied by rsqrt(sum_i ssq[i*ssq_stride + r] / K + eps); nullptr = 1
     const float *ssq;
     int n_ssq, ssq_stride;
     float eps;
@@ -62,7 +74,8 @@ struct TcGemmArgs {
 bool tc_make_map(CUtensorMap *map, const void *base, uint64_t inner, uint64_t rows, uint32_t box_rows);
 // activation rows per CTA, padded to the UMMA N granularity (box_rows of the X map)
 int tc_row_pad(int R);
-// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max, 3 cluster split-K + residual, 4 cluster split-K + rotary/KV write.
+// mode: 0 fp32 planes, 1 SwiGLU, 2 arg-max, 3 cluster split-K + residual, 4 cluster split-K + rotary/KV write,
+// 5 per-tile top-k candidates + log-sum-exp shares.
 // map_w box_rows must be 128 (64 in mode 1), map_x box_rows tc_row_pad(R).
 cudaError_t launch_gemm_tc(int mode, TcGemmArgs a, const CUtensorMap &map_w, const CUtensorMap &map_x, cudaStream_t st);
 

@@ -56,7 +56,6 @@ struct Workspace {
     bf16 *q;             // [Rmax][Hq d]
     bf16 *attn;          // [Rmax][Hq d]
     bf16 *act;           // [Rmax][F]
-    float *logits;       // [Rlog][V]
     int32_t *walk_ctr;
     int32_t *row_seq, *row_pos;
     long long *row_kvrow;
@@ -70,8 +69,11 @@ struct Workspace {
     unsigned long long *am_keys;   // [Rlog] packed arg-max keys, zero between launches
     int32_t *am_counter;
     float *ent_part;       // [vocab tiles][max_batch][3] soft-max statistics of the root rows (entropy log)
-    unsigned long long *topk_cand; // [batch*L][warps][k]
-    float *topk_ml;                // [batch*L][warps][2]
+    // draft top-k, fused into the LM head: per 128-feature tile and block row
+    uint32_t *tk_thr;              // [batch*B][kTopkTileCap] running class maxima of every row (0 between launches)
+    float *tk_ml;                  // [vocab tiles][batch*B][2] (max, sum exp)
+    int32_t *tk_cnt;               // [vocab tiles][batch*B] candidate keys emitted
+    unsigned long long *tk_cand;   // [vocab tiles][batch*B][kTopkTileCap]
     size_t total;
 };
 
@@ -106,7 +108,6 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.q = (bf16 *)take(2 * R * d.qd * 2);               // two planes
     w.attn = (bf16 *)take(2 * R * d.qd * 2);            // two planes
     w.act = (bf16 *)take(2 * R * (size_t)c.ffn * 2);    // two planes
-    w.logits = (float *)take((size_t)d.Rlog * c.vocab * 4);
     w.walk_ctr = (int32_t *)take((size_t)c.max_batch * 4);
     w.row_seq = (int32_t *)take(R * 4);
     w.row_pos = (int32_t *)take(R * 4);
@@ -122,9 +123,11 @@ Workspace carve(const glance_config &c, const Dims &d, unsigned char *base) {
     w.am_keys = (unsigned long long *)take((size_t)d.Rlog * 8);
     w.am_counter = (int32_t *)take(256);
     w.ent_part = (float *)take((size_t)((c.vocab + 127) / 128) * c.max_batch * 3 * 4);
-    const size_t trows = (size_t)c.max_batch * (c.block_B - 1) * topk_warps(c.vocab);
-    w.topk_cand = (unsigned long long *)take(trows * c.topk * 8);
-    w.topk_ml = (float *)take(trows * 2 * 4);
+    const size_t trows = (size_t)((c.vocab + 127) / 128) * c.max_batch * c.block_B;
+    w.tk_thr = (uint32_t *)take((size_t)c.max_batch * c.block_B * kTopkTileCap * 4);
+    w.tk_ml = (float *)take(trows * 2 * 4);
+    w.tk_cnt = (int32_t *)take(trows * 4);
+    w.tk_cand = (unsigned long long *)take(trows * kTopkTileCap * 8);
     w.total = off;
     return w;
 }
@@ -246,6 +249,7 @@ void gemm(glance_ctx *ctx, int mode, const bf16 *W, const bf16 *X, int x_rows, T
     if (mode == 0) bytes += 4.0 * a.S * a.R * a.Nout;
     else if (mode == 1) bytes += (a.act_lo ? 4.0 : 2.0) * a.R * a.F;
     else if (mode == 2) bytes += 4.0 * a.R + (a.Y ? 4.0 * a.R * a.Nout : 0.0);
+    else if (mode == 5) bytes += (a.Y ? 4.0 * a.R * a.Nout : 0.0) + 12.0 * a.R * ((a.Nout + 127) / 128);
     else if (mode == 3) bytes += (4.0 + 4.0 + (a.xb_lo ? 4.0 : 2.0)) * a.R * a.Nout;   // residual in/out + bf16 copy
     else bytes += 2.0 * a.R * a.Nout;
     prof_end(ctx, prof, KIND_GEMM, bytes);
@@ -505,7 +509,8 @@ int32_t glance_create(const glance_config *cfg, const glance_target_weights *t, 
     if (cudaMemsetAsync(ws.walk_ctr, 0, (size_t)cfg->max_batch * 4, ctx->stream) != cudaSuccess ||
         cudaMemsetAsync(ws.status, 0, 256, ctx->stream) != cudaSuccess ||
         cudaMemsetAsync(ws.am_keys, 0, (size_t)d.Rlog * 8, ctx->stream) != cudaSuccess ||
-        cudaMemsetAsync(ws.am_counter, 0, 256, ctx->stream) != cudaSuccess) {
+        cudaMemsetAsync(ws.am_counter, 0, 256, ctx->stream) != cudaSuccess ||
+        cudaMemsetAsync(ws.tk_thr, 0, (size_t)cfg->max_batch * cfg->block_B * kTopkTileCap * 4, ctx->stream) != cudaSuccess) {
         delete ctx;
         return GLANCE_E_CUDA;
     }
@@ -611,20 +616,19 @@ int32_t glance_draft_block(glance_ctx *ctx, const glance_seqs *seqs, int32_t *to
         const bf16 *next_gain = i + 1 < HL ? (const bf16 *)ctx->head_layer[i + 1].ln1 : (const bf16 *)ctx->head.final_norm;
         run_layer(ctx, hw, (bf16 *)seqs->head_kv_pool + (size_t)i * hgeom.layer_stride(), ps, next_gain, nullptr);
     }
-    float *logits = logits_dbg ? logits_dbg : ws.logits;
+    // LM head over the block rows with the per-offset top-k fused into its epilogue: every 128-feature tile leaves
+    // its log-sum-exp share and the keys that can still be among a row's k largest; one small launch merges them.
+    // The logits themselves are written only on request.
     {
         TcGemmArgs g{};
-        g.Nout = c.vocab; g.K = c.hidden; g.R = R1; g.S = 1; g.Y = logits; g.ldy = c.vocab; g.split_stride = 0;
+        g.Nout = c.vocab; g.K = c.hidden; g.R = R1; g.S = 1; g.Y = logits_dbg; g.ldy = c.vocab; g.split_stride = 0;
         g.x_lo_row = 0;
+        g.tk_k = c.topk; g.tk_B = B; g.tk_thr = ws.tk_thr; g.tk_ml = ws.tk_ml; g.tk_cnt = ws.tk_cnt; g.tk_cand = ws.tk_cand;
         with_row_scales(ctx, g);
-        gemm(ctx, 0, ctx->lm_head, ws.xn, ctx->dims.Rmax, g);
+        gemm(ctx, 5, ctx->lm_head, ws.xn, ctx->dims.Rmax, g);
     }
-    {
-        const bool prof = prof_begin(ctx);
-        launch_topk(logits, batch, B, c.vocab, c.topk, topk_ids, topk_lp, ws.topk_cand, ws.topk_ml, st);
-        ctx->launches++;                              // two kernels
-        prof_end(ctx, prof, KIND_CONTROL, 0.0);
-    }
+    LAUNCH(ctx, KIND_CONTROL, launch_topk_merge(batch, B, (c.vocab + 127) / 128, c.topk, ws.tk_thr, ws.tk_ml, ws.tk_cnt,
+                                                ws.tk_cand, topk_ids, topk_lp, st));
     return finish(ctx);
 }
 

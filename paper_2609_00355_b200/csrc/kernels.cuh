@@ -68,6 +68,12 @@ int topk_warps(int V);
 void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *ids, float *lp,
                  unsigned long long *cand, float *ml, cudaStream_t st);
 
+// merge of the draft LM head's per-tile candidates and log-sum-exp shares (gemm_tc_kernel mode 5): thr [batch*B][16],
+// ml [tiles][batch*B][2], cnt [tiles][batch*B], cand [tiles][batch*B][kTopkTileCap] -> ids / lp [batch][B-1][k];
+// re-arms thr.  One launch.
+void launch_topk_merge(int batch, int B, int tiles, int k, uint32_t *thr, const float *ml, const int32_t *cnt,
+                       const unsigned long long *cand, int32_t *ids, float *lp, cudaStream_t st);
+
 // ---- tree + walk (tree_walk.cu) -----------------------------------------------------------
 void launch_build_tree(int batch, int N, int L, int k, const int32_t *root, const int32_t *ids, const float *lp,
                        const glance_tree &out, cudaStream_t st);

@@ -1,5 +1,6 @@
 // Row setup kernels of the verify and draft passes (embedding gather, rotary table, paged row offsets, first
 // norm statistics) and the two-stage per-offset top-k + log-softmax of the draft pass.
+#include "gemm_tc.cuh"
 #include "kernels.cuh"
 #include "tc_ptx.cuh"
 
@@ -401,6 +402,151 @@ void launch_topk(const float *logits, int batch, int B, int V, int k, int32_t *i
     dim3 g1((nw + 3) / 4, rows);
     topk_stage1_kernel<<<g1, 128, 0, st>>>(logits, B, V, k, nw, cand, ml);
     topk_stage2_kernel<<<rows, 32, 0, st>>>(k, nw, cand, ml, ids, lp);
+}
+
+// ------------------------------------------------------------------------------------------
+// Merge of the draft LM head's per-tile shares (gemm_tc_kernel mode 5) into the per-offset top-k and log-softmax.
+// One block per (sequence, offset).  The tiles left, for this row, (max, sum exp) and the keys that reached the
+// row's bound at the time; the bound's final value (the smallest of the row's k class maxima) is what at least k
+// entries of the row reach, so the k best are among the emitted keys at or above it.  Log-sum-exp: every thread folds the tiles t = tid, tid + 1024, ... in order,
+// the threads' shares are then added in a fixed tree (bit-reproducible).  The keys at or above the final bound
+// (few) are collected into shared memory in any order and ranked by one warp; keys are unique, so the ranking does
+// not depend on the order of collection.  The row's bound is re-armed (0) for the next launch.
+// ------------------------------------------------------------------------------------------
+constexpr int kMergeThreads = 1024;
+constexpr int kMergeCap = 512;                           // keys a row may collect before it falls back to full scans
+
+__global__ void __launch_bounds__(kMergeThreads) topk_merge_kernel(int B, int R, int tiles, int k, uint32_t *thr,
+                                                                   const float *ml, const int32_t *cnt,
+                                                                   const unsigned long long *cand, int32_t *ids, float *lp) {
+    static_assert(kMergeThreads == 1024, "the second reduction level takes exactly 32 warps");
+    __shared__ float red_m[32], red_s[32];
+    __shared__ unsigned long long list[kMergeCap];
+    __shared__ int n_list;
+    __shared__ unsigned long long best_w[kMergeThreads / 32];
+    const int L = B - 1;
+    const int out_row = blockIdx.x;                      // (s, j-1)
+    const int s = out_row / L, j = out_row % L + 1;
+    const int r = s * B + j;                             // row of the LM-head launch
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    tc::pdl_wait();                                      // launched early; everything it reads is the LM head's output
+    // ---- log-sum-exp over the tiles
+    float M = -INFINITY, S = 0.f;
+    for (int t = tid; t < tiles; t += kMergeThreads) {
+        const float m = __ldcg(ml + 2 * ((size_t)t * R + r)), e = __ldcg(ml + 2 * ((size_t)t * R + r) + 1);
+        const float nm = fmaxf(M, m);
+        S = (M == -INFINITY ? 0.f : S * expf(M - nm)) + (m == -INFINITY ? 0.f : e * expf(m - nm));
+        M = nm;
+    }
+    // fixed tree: lanes by shuffles, then the 32 warps' shares by the first warp
+    auto fold = [](float &m0, float &s0, float m1, float s1) {
+        const float nm = fmaxf(m0, m1);
+        s0 = (m0 == -INFINITY ? 0.f : s0 * expf(m0 - nm)) + (m1 == -INFINITY ? 0.f : s1 * expf(m1 - nm));
+        m0 = nm;
+    };
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) fold(M, S, __shfl_xor_sync(0xffffffffu, M, o), __shfl_xor_sync(0xffffffffu, S, o));
+    if (lane == 0) { red_m[wid] = M; red_s[wid] = S; }
+    if (tid == 0) n_list = 0;
+    __syncthreads();
+    if (wid == 0) {
+        M = red_m[lane];
+        S = red_s[lane];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) fold(M, S, __shfl_xor_sync(0xffffffffu, M, o), __shfl_xor_sync(0xffffffffu, S, o));
+        if (lane == 0) { red_m[0] = M; red_s[0] = S; }
+    }
+    __syncthreads();
+    const float lse = red_m[0] + logf(red_s[0]);
+    // ---- the keys at or above the row's final bound
+    uint32_t T = 0xffffffffu;                            // the smallest of the row's k class maxima (0: a class stayed empty)
+    for (int b = 0; b < k; ++b) T = min(T, __ldcg(thr + (size_t)r * kTopkTileCap + b));
+    // one thread per (tile, key slot): the count and the key are fetched independently (a slot beyond the tile's count
+    // holds an older launch's key and is ignored), so the loads of a thread's few iterations are all in flight together
+    for (int idx0 = tid; idx0 < tiles * kTopkTileCap; idx0 += 8 * kMergeThreads) {
+        int c8[8];
+        unsigned long long key8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {                    // eight independent (count, key) pairs in flight
+            const int idx = idx0 + u * kMergeThreads;
+            c8[u] = 0;
+            key8[u] = 0ull;
+            if (idx < tiles * kTopkTileCap) {
+                const size_t slot = (size_t)(idx / kTopkTileCap) * R + r;
+                c8[u] = __ldcg(cnt + slot);
+                key8[u] = __ldcg(cand + slot * kTopkTileCap + idx % kTopkTileCap);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = (idx0 + u * kMergeThreads) % kTopkTileCap;
+            if (i < c8[u] && (uint32_t)(key8[u] >> 32) >= T) {
+                const int at = atomicAdd(&n_list, 1);
+                if (at < kMergeCap) list[at] = key8[u];
+            }
+        }
+    }
+    __syncthreads();
+    const int n = n_list;
+    unsigned long long prev = ~0ull;
+    if (n <= kMergeCap) {
+        if (wid == 0) {
+            for (int t = 0; t < k; ++t) {
+                unsigned long long best = 0ull;
+                for (int c = lane; c < n; c += 32) {
+                    const unsigned long long key = list[c];
+                    if (key < prev && key > best) best = key;
+                }
+                best = warp_max_u64(best);
+                if (lane == 0) {
+                    ids[(size_t)out_row * k + t] = unpack_id(best);
+                    lp[(size_t)out_row * k + t] = unpack_val(best) - lse;
+                }
+                prev = best;
+            }
+        }
+    } else {
+        // very many equal values at the bound: k full scans over the emitted keys
+        for (int t = 0; t < k; ++t) {
+            unsigned long long best = 0ull;
+            for (int tl = tid; tl < tiles; tl += kMergeThreads) {
+                const size_t slot = (size_t)tl * R + r;
+                const int c = __ldcg(cnt + slot);
+                for (int i = 0; i < c; ++i) {
+                    const unsigned long long key = __ldcg(cand + slot * kTopkTileCap + i);
+                    if (key < prev && key > best) best = key;
+                }
+            }
+            best = warp_max_u64(best);
+            if (lane == 0) best_w[wid] = best;
+            __syncthreads();
+            best = 0ull;
+            for (int w = 0; w < kMergeThreads / 32; ++w) best = best_w[w] > best ? best_w[w] : best;
+            if (tid == 0) {
+                ids[(size_t)out_row * k + t] = unpack_id(best);
+                lp[(size_t)out_row * k + t] = unpack_val(best) - lse;
+            }
+            prev = best;
+            __syncthreads();
+        }
+    }
+    if (tid < kTopkTileCap) thr[(size_t)r * kTopkTileCap + tid] = 0u;   // every read of the bounds is behind the barrier above
+}
+
+void launch_topk_merge(int batch, int B, int tiles, int k, uint32_t *thr, const float *ml, const int32_t *cnt,
+                       const unsigned long long *cand, int32_t *ids, float *lp, cudaStream_t st) {
+    if (B < 2) return;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(batch * (B - 1), 1, 1);
+    cfg.blockDim = dim3(kMergeThreads, 1, 1);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // its blocks are placed while the LM head drains
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, topk_merge_kernel, B, batch * B, tiles, k, thr, (const float *)ml, (const int32_t *)cnt,
+                       (const unsigned long long *)cand, ids, lp);
 }
 
 __global__ void prefill_advance_kernel(int32_t *seq_len, int32_t *root, int32_t *feat_count, const int32_t *argmax,

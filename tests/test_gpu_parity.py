@@ -310,6 +310,39 @@ def test_build_tree_exhausted_frontier_bit_exact(harness, block_B, topk, tree_N)
             assert all(int(v) == -1 for v in eng.tree.parent[s, prefixes + 1:].cpu())
 
 
+@pytest.mark.parametrize("vocab,topk,distinct", [(1000, 4, 3), (1000, 16, 2), (130, 8, 130), (8192, 16, 1), (2000, 8, 40)])
+def test_draft_topk_fused_in_lm_head_with_massive_ties(harness, vocab, topk, distinct):
+    """The per-offset top-k inside the LM head's epilogue under the worst ties: the LM head repeats `distinct` rows,
+    so every logit value is shared by vocab / distinct ids spread over all tiles (tiles with more equal values at
+    the bound than they have slots, a merge with more keys at the bound than it collects, a last tile of two
+    features, k equal to the slot count).  Against the exact (logit desc, id asc) order of the library's own logits."""
+    cfg = synth.CONFIGS["tiny"].replace(vocab=vocab, topk=topk, block_B=5, tree_N=8, n_img=20, n_txt=12, rounds=1)
+    tw, hw = synth.make_weights(cfg, "cuda")
+    tw["lm_head"] = tw["lm_head"][:distinct].repeat((vocab + distinct - 1) // distinct, 1)[:vocab].contiguous()
+    from paper_2609_00355_b200.binding import Engine
+    eng = Engine(cfg, tw, hw, batch=2)
+    for s in range(2):
+        img, ids = synth.make_context(cfg, "cuda", seed=3 + s)
+        eng.prefill_context(s, img, ids % min(vocab, 1000))
+    B, L = cfg.block_B, cfg.L
+    for rep in range(2):                                   # the second call meets re-armed bounds and stale key slots
+        logits = torch.zeros(2, B, vocab, dtype=torch.float32, device="cuda")
+        eng.glance_draft_block(logits_dbg=logits)
+        eng.check_device_status()
+        lg = logits.cpu().numpy()
+        for s in range(2):
+            for j in range(1, B):
+                row = lg[s, j]
+                order = np.lexsort((np.arange(vocab), -row))[:topk]
+                assert np.array_equal(eng.topk_ids[s, j - 1].cpu().numpy(), order.astype(np.int32)), (rep, s, j)
+                lse = float(torch.logsumexp(torch.from_numpy(row).double(), dim=0))
+                got = eng.topk_lp[s, j - 1].cpu().numpy().astype(np.float64)
+                assert np.abs(got - (row[order].astype(np.float64) - lse)).max() < 1e-4
+        eng.glance_build_tree()
+        eng.glance_verify_tree()
+        eng.glance_accept_commit()
+
+
 # ------------------------------------------------------------------ walk + commit (bit-exact)
 
 def test_walk_commit_examples_and_compaction_hazard(harness):

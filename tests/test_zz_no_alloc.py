@@ -39,12 +39,14 @@ def test_topk_static_matches_draft_block_and_oracle_twice():
         lp = torch.full((2, L, k), float("nan"), dtype=torch.float32, device="cuda")
         assert binding.glance_topk_static(logits, k, ids, lp) == 0
         torch.cuda.synchronize()
-        # same kernels, same inputs, fixed reduction order: ids identical and log-probabilities bit-equal,
-        # which is well inside the 2e-2 (relative to the logit scale) tolerance of the other parity tests
+        # Same logits on both sides (the draft pass exported the ones its fused top-k worked on): both select the k
+        # largest under (logit desc, id asc), so the ids are identical; the log-sum-exp is added up in a different
+        # order (1024-entry spans here, 128-feature tiles there), so the log-probabilities agree to rounding --
+        # checked within the 2e-2 (relative to the logit scale) tolerance of the other parity tests, and far tighter
         assert torch.equal(ids, ids_ref)
-        assert torch.equal(lp, lp_ref)
         scale = float(logits.abs().max())
         assert float((lp - lp_ref).abs().max()) <= TOL * scale
+        assert float((lp - lp_ref).abs().max()) <= 1e-4
         # against the oracle on the same logits: log-probabilities within the tolerance, ids identical wherever
         # the oracle's gap between consecutive ranks exceeds the margin
         lg_cpu = logits.cpu()
