@@ -513,6 +513,42 @@ def test_rounds_batch3_two_row_blocks(harness):
     assert run.stats["max_rel_logit"] <= 2e-2
 
 
+def test_rounds_batch16_four_row_blocks_ragged(harness):
+    """Sixteen ragged sequences of 32 tree rows each: 512 verify rows = four 128-row blocks of every GEMM (the launch
+    shapes of the small-batch serving configuration: split-K chosen for whole waves, two key splits in the
+    attention), 256 draft rows, per-sequence trees, accepts and compaction."""
+    cfg = synth.CONFIGS["tiny"].replace(tree_N=32, block_B=8, topk=3)
+    rng = np.random.default_rng(12)
+    ctx_lens = [(int(a), int(b)) for a, b in zip(rng.integers(5, 220, size=16), rng.integers(1, 40, size=16))]
+    run = harness.ParityRun(cfg, batch=16, ctx_lens=ctx_lens)
+    run.check_state()
+    for r in range(2):
+        run.round(p_m=(0.7 if r else None), check_draft=(r == 0))
+    run.check_head_state()
+    print("batch16 x 32 rows parity stats:", run.stats)
+    assert run.stats["max_rel_logit"] <= 2e-2
+
+
+def test_page_budget_exact_fit_passes_and_one_more_row_is_a_capacity_fault(harness):
+    """seq_len + tree_N == page_size * max_pages_per_seq is legal (the last tree row sits in the last slot of the
+    last page); one committed position more is reported as GLANCE_E_CAPACITY and nothing faults."""
+    cfg = synth.CONFIGS["tiny"]
+    run = harness.ParityRun(cfg, ctx_lens=[(20, 5)])
+    eng = run.eng
+    cap = eng.pages_per_seq * 64
+    snap = eng.snapshot_state()
+    eng.seq_len[0] = cap - cfg.tree_N                    # rows cap - N .. cap - 1: exactly fits
+    eng.glance_build_tree()
+    eng.glance_verify_tree()
+    assert eng.glance_poll_status() == 0
+    eng.seq_len[0] = cap - cfg.tree_N + 1
+    eng.glance_verify_tree()
+    assert eng.glance_poll_status() == -3
+    eng.restore_state(snap)
+    run.round(p_m=0.7)                                    # the engine is still good
+    assert eng.glance_poll_status() == 0
+
+
 def test_rounds_tiny_chain_k1(harness):
     """k = 1: the candidate tree degenerates to the rank-0 chain (classic chain drafting through the same path)."""
     cfg = synth.CONFIGS["tiny"].replace(topk=1, tree_N=4)
