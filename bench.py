@@ -458,7 +458,6 @@ def main():
 
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
     from paper_2609_00355_b200 import build as glance_build
-    glance_build.build()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
@@ -466,6 +465,11 @@ def main():
         import torch.distributed as dist_mod
         dist_mod.init_process_group("nccl", device_id=dev)
         dist = dist_mod
+        # one rank per node compiles (if the library is stale at all); the others load what it built
+        if local_rank == 0:
+            glance_build.build()
+        dist.barrier()
+    glance_build.build()
     torch.manual_seed(0)
     # every timed, profiled and end-to-end round may commit a whole block
     rounds_total = 2 * (warmup + args.steps) + min(args.steps, 16) + 2
