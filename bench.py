@@ -609,7 +609,7 @@ def main():
                 "tau": e2e_committed / (args.steps * cfg.batch * world) if e2e_s > 0 else None,
                 "value_at_expected_tau": (expected_tau * cfg.batch * world / (e2e_s / args.steps)) if (e2e_s > 0 and cfg.batch == 1) else None,
                 "note": "same seeded hit pattern per round as the device-resident arm; compare ms_per_step",
-                "h2d_bytes_per_step": int(bench.ids_host.numel() * 4 + bench.lp_host.numel() * 4),
+                "h2d_bytes_per_step": int(bench.in_host.numel() * 4),
                 "d2h_bytes_per_step": int(bench.res_host.numel() * 4)},
         "gpu_launches": int(launches_per_round * args.steps),
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],

@@ -69,12 +69,24 @@ class RoundBench:
         self.ar_tree.anc.copy_(torch.from_numpy(anc.view(np.int64))[None].expand(cfg.batch, N, W))
         self.rng = np.random.default_rng(3 + rank)
         L, k = cfg.L, cfg.topk
-        self.lp_host = torch.from_numpy(np.stack([synth.controlled_marginals(p, k, L) for p in self.p_ms])).pin_memory()
-        self.ids_host = torch.zeros(cfg.batch, L, k, dtype=torch.int32).pin_memory()
-        self.cand_ids = torch.zeros(cfg.batch, L, k, dtype=torch.int32, device=device)
-        self.cand_lp = self.lp_host.to(device)
-        self.res_host = torch.zeros(cfg.batch, 1 + cfg.block_B, dtype=torch.int32).pin_memory()
-        self.res_dev = torch.zeros(cfg.batch, 1 + cfg.block_B, dtype=torch.int32, device=device)
+        # Host <-> device staging of the end-to-end step, one copy each way: the step's inputs (candidate ids, int32,
+        # then their log-probabilities, fp32 bits) sit in ONE pinned buffer mirrored by one device buffer of which
+        # cand_ids / cand_lp are views; the step's result (accepted lengths, then emitted tokens) is ONE device buffer
+        # that the engine's accept_len / out_tokens are views of, mirrored by one pinned buffer.
+        n_in = cfg.batch * L * k
+        self.in_host = torch.zeros(2 * n_in, dtype=torch.int32).pin_memory()
+        self.in_dev = torch.zeros(2 * n_in, dtype=torch.int32, device=device)
+        self.ids_host = self.in_host[:n_in].view(cfg.batch, L, k)
+        self.lp_host = self.in_host[n_in:].view(torch.float32).view(cfg.batch, L, k)
+        self.lp_host.copy_(torch.from_numpy(np.stack([synth.controlled_marginals(p, k, L) for p in self.p_ms])))
+        self.cand_ids = self.in_dev[:n_in].view(cfg.batch, L, k)
+        self.cand_lp = self.in_dev[n_in:].view(torch.float32).view(cfg.batch, L, k)
+        self.in_dev.copy_(self.in_host)
+        B = cfg.block_B
+        self.res_dev = torch.zeros(cfg.batch * (1 + B), dtype=torch.int32, device=device)
+        self.res_host = torch.zeros(cfg.batch * (1 + B), dtype=torch.int32).pin_memory()
+        eng.accept_len = self.res_dev[:cfg.batch]
+        eng.out_tokens = self.res_dev[cfg.batch:].view(cfg.batch, B)
 
     def lookahead(self):
         """Untimed: the next L greedy tokens after the pending root (single-node rounds, then rollback)."""
@@ -131,12 +143,8 @@ class RoundBench:
     def e2e_calls(self):
         """The round as a caller with host buffers issues it: this step's inputs from pinned host memory, the four
         calls, the result (accepted lengths and emitted tokens) back to pinned host memory."""
-        eng = self.eng
-        self.cand_ids.copy_(self.ids_host, non_blocking=True)
-        self.cand_lp.copy_(self.lp_host, non_blocking=True)
+        self.in_dev.copy_(self.in_host, non_blocking=True)
         self.round_calls()
-        self.res_dev[:, 0].copy_(eng.accept_len)
-        self.res_dev[:, 1:].copy_(eng.out_tokens)
         self.res_host.copy_(self.res_dev, non_blocking=True)
 
     def capture_round_e2e(self):
@@ -151,14 +159,10 @@ class RoundBench:
         if self.graph_e2e is not None:
             self.graph_e2e.replay()
         elif self.graph is not None:
-            eng = self.eng
-            self.cand_ids.copy_(self.ids_host, non_blocking=True)
-            self.cand_lp.copy_(self.lp_host, non_blocking=True)
+            self.in_dev.copy_(self.in_host, non_blocking=True)
             self.graph.replay()
-            self.res_dev[:, 0].copy_(eng.accept_len)
-            self.res_dev[:, 1:].copy_(eng.out_tokens)
             self.res_host.copy_(self.res_dev, non_blocking=True)
         else:
             self.e2e_calls()
         torch.cuda.current_stream().synchronize()
-        return self.res_host[:, 0].clone()
+        return self.res_host[:self.cfg.batch].clone()
